@@ -1,0 +1,232 @@
+/*
+ * epara.h -- C ABI of the B200 categorized serving step.
+ *
+ * One "step" executes, on one GPU, the forward passes of every admitted request of every
+ * co-resident model: the single-GPU combination of the paper's allocation operators
+ * batching (BS), multi-task (MT) and multi-frame (MF) (paper Section 3.1, "Allocation
+ * operators") for the two categories that need no multi-GPU collaboration (Section 3.1,
+ * "Performing operators to categories", first and third case).
+ *
+ * Ownership: the caller owns every byte of device memory (weights, KV pool, inputs,
+ * outputs, workspace) and the CUDA stream.  The library borrows the pointers; they must
+ * stay valid until the request is collected (weights/KV/workspace: until epara_destroy).
+ * The library owns only host structures and its pinned descriptor buffers.
+ *
+ * Pointers named "device" are CUDA device pointers, 16-byte aligned; "host" pointers are
+ * ordinary host memory read during the call only.  All tensors are row-major.  bf16 means
+ * the upper 16 bits of an IEEE fp32.
+ *
+ * Errors: every function returns an epara_status; nothing throws, aborts or prints.
+ * A context is not thread-safe: one host thread per context.
+ */
+#ifndef EPARA_H
+#define EPARA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct epara_ctx epara_ctx;
+
+/* Task categories (Section 3.1, "Task categories"): sensitivity (latency / frequency) x
+ * resource need (<1 GPU / >1 GPU).  The >1 GPU categories need model parallelism and are
+ * rejected by epara_submit with EPARA_E_UNSUPPORTED. */
+enum {
+  EPARA_CAT_LS_LT1 = 0, /* latency-sensitive, fits one GPU: BS + MT */
+  EPARA_CAT_FS_LT1 = 1, /* frequency-sensitive, fits one GPU: MF + MT + BS */
+  EPARA_CAT_LS_GT1 = 2,
+  EPARA_CAT_FS_GT1 = 3
+};
+
+/* Status codes.  TIMEOUT and RESOURCE are two of the request handler's answers
+ * (Section 3.2: "timeout", "resource insufficiency"). */
+enum {
+  EPARA_OK = 0,
+  EPARA_PENDING = 1,
+  EPARA_E_INVALID = -1,
+  EPARA_E_UNSUPPORTED = -2,
+  EPARA_E_TIMEOUT = -3,
+  EPARA_E_RESOURCE = -4,
+  EPARA_E_DEVICE = -5,
+  EPARA_E_CUDA = -6
+};
+
+enum { EPARA_MODEL_MLP = 0, EPARA_MODEL_VIT = 1, EPARA_MODEL_DECODER = 2 };
+
+enum { EPARA_GEMM_TCGEN05 = 0, EPARA_GEMM_SIMT = 1 };
+
+#define EPARA_KV_PAGE 16 /* tokens per KV page */
+
+typedef struct {
+  int device;             /* CUDA device ordinal; made current by every call */
+  void* workspace;        /* device, caller-owned scratch for activations and descriptors */
+  size_t workspace_bytes;
+  int cap_ls;             /* BS cap of a latency-sensitive group per model per step (0 -> 4) */
+  int cap_fs;             /* BS cap of a frequency-sensitive group (0 -> 256) */
+  int mf_max;             /* MF: max inter-frame count per stream; 0 = plain oldest-first batching */
+  int gemm_impl;          /* EPARA_GEMM_TCGEN05 (default) or EPARA_GEMM_SIMT (plain CUDA-core comparator) */
+  int max_queue;          /* queued requests per (model, category) before RESOURCE (0 -> 4096) */
+  int profile;            /* 1: bracket every launch with CUDA events (see epara_step_profile) */
+} epara_config;
+
+/* Model description.  `tensors` is a host array of device pointers to bf16 tensors in this order:
+ *  MLP     : W_0 [dims[1], dims[0]], b_0 [dims[1]], W_1, b_1, ...          (GELU between layers,
+ *            none after the last)
+ *  VIT     : W_pe [d, 3*patch*patch], b_pe [d], cls [d], pos [T, d], then per layer
+ *            ln1_g, ln1_b, Wqkv [3d, d] (rows q;k;v), bqkv, Wo [d,d], bo, ln2_g, ln2_b,
+ *            W1 [ffn, d], b1, W2 [d, ffn], b2, then lnf_g, lnf_b, Whead [vocab, d], bhead.
+ *            T = (img/patch)^2 + 1; pre-LN encoder, LayerNorm eps 1e-6, exact-erf GELU.
+ *  DECODER : Emb [vocab, d], then per layer g1 [d], Wqkv [(Hq+2Hkv)*hd, d] (rows q;k;v),
+ *            Wo [d, Hq*hd], g2 [d], Wgu [2*ffn, d] (row 2j = gate j, row 2j+1 = up j),
+ *            Wd [d, ffn], then gf [d], Wlm [vocab, d].  RMSNorm eps 1e-5, interleaved-pair
+ *            RoPE base 10000, SwiGLU.
+ * Every weight matrix is [out_features, in_features] with in_features contiguous and a
+ * multiple of 8.  kv_pool (decoder): bf16 [n_layers][kv_pages][2 (K,V)][Hkv][16][hd]. */
+typedef struct {
+  int kind;
+  int n_layers;
+  int d;
+  int n_heads;      /* query heads */
+  int n_kv_heads;   /* decoder only */
+  int head_dim;
+  int ffn;
+  int vocab;        /* decoder vocabulary / ViT class count / ignored for MLP */
+  int img, patch;   /* ViT only */
+  const int* mlp_dims;          /* host, n_layers + 1 entries, MLP only */
+  const void* const* tensors;   /* host array of device pointers */
+  int n_tensors;
+  void* kv_pool;                /* device, decoder only */
+  long long kv_pages;
+  int max_kv_len;               /* decoder: longest cached length a request may have */
+  int max_batch;                /* rows reserved in the workspace (0 -> cap_ls + cap_fs) */
+} epara_model_desc;
+
+/* One request.  Unused fields are ignored for the model's kind. */
+typedef struct {
+  const void* input;        /* device: MLP bf16 [dims[0]]; VIT bf16 [3, img, img]; DECODER: NULL */
+  int token;                /* decoder: id of the token being decoded */
+  int kv_len;               /* decoder: cached tokens L; the new token is written at slot L and
+                               attention runs over L + 1 tokens */
+  const int32_t* block_table; /* device int32 [n_blocks], page ids; needs n_blocks >= L/16 + 1 */
+  int n_blocks;
+  long long deadline_ns;    /* absolute time after which the request is dropped; 0 = none */
+  long long arrival_ns;
+  int stream;               /* frequency-sensitive stream id (MF groups frames per stream) */
+  void* out_logits;         /* device bf16 [n_out] (MLP: last width; VIT/DECODER: vocab) */
+  int32_t* out_argmax;      /* device int32 [1]; lowest index wins ties; may be NULL */
+} epara_inputs;
+
+typedef struct {
+  uint64_t step_id;
+  int admitted[2];          /* per category */
+  int dropped[2];           /* timed out at admission */
+  int launches;             /* kernels launched by this step */
+  int gemm_groups;
+  double gemm_flops;        /* 2 M N K over all GEMM groups */
+  double weight_bytes;      /* bytes of weight matrices the step streams */
+  double kv_bytes;          /* bytes of cached K/V the step reads */
+  int device_error;         /* filled by epara_collect when a kernel reported a bounded-wait failure */
+} epara_step_info;
+
+typedef struct {
+  int status;               /* EPARA_OK, EPARA_E_TIMEOUT (dropped), EPARA_E_DEVICE */
+  uint64_t step_id;
+  void* logits;             /* the request's out_logits */
+  int n_out;
+  int32_t* argmax;
+} epara_output;
+
+/* Kinds of kernels a step launches (index into epara_step_profile arrays). */
+enum {
+  EPARA_K_GATHER = 0, EPARA_K_NORM = 1, EPARA_K_GEMM = 2, EPARA_K_ROPE = 3, EPARA_K_ATTN_DEC = 4,
+  EPARA_K_ATTN_COMBINE = 5, EPARA_K_ATTN_ENC = 6, EPARA_K_ASSEMBLE = 7, EPARA_K_OUTPUT = 8,
+  EPARA_K_COUNT = 9
+};
+
+/* Creates a context on cfg->device.  Returns INVALID (null/unaligned workspace), CUDA. */
+int epara_init(const epara_config* cfg, epara_ctx** out);
+
+/* "Placement" of a service on this GPU (the paper pre-places models because loading is slow,
+ * Section 3.3): records the pointers, reserves activation workspace for max_batch rows and
+ * builds the TMA tensor maps.  RESOURCE if the workspace is too small, INVALID on bad dims. */
+int epara_register_model(epara_ctx*, const epara_model_desc* m, int* model_id);
+
+/* Queues one request (host only, no device work).  UNSUPPORTED for the >1 GPU categories,
+ * INVALID for bad ids/pointers/lengths, RESOURCE when the queue is full. */
+int epara_submit(epara_ctx*, int model_id, int category, const epara_inputs* in, uint64_t* ticket);
+
+/* Runs one step on `cuda_stream` (a cudaStream_t), asynchronously:
+ *  - drops requests whose deadline_ns < now_ns (Section 3.2, first handler rule);
+ *  - per model admits the oldest <= cap_ls latency-sensitive requests, then frequency-
+ *    sensitive ones up to cap_fs, by MF when mf_max > 0: floor(cap_fs / mf_max) streams
+ *    (Eq. 5), the same number of frames from each;
+ *  - runs all admitted groups of all models together, one grouped launch per kernel kind
+ *    per dependency wave.
+ * now_ns < 0 uses the host's monotonic clock.  info may be NULL. */
+int epara_step(epara_ctx*, void* cuda_stream, long long now_ns, epara_step_info* info);
+
+/* PENDING until the step that took the ticket has finished on the device (never blocks);
+ * then OK with out filled, TIMEOUT if the request was dropped, DEVICE on a device error.
+ * INVALID for an unknown (or already collected) ticket.  A ticket still queued is PENDING. */
+int epara_collect(epara_ctx*, uint64_t ticket, epara_output* out);
+
+/* With cfg.profile = 1: per kernel kind, total milliseconds and launch count of the most
+ * recent finished step (arrays of EPARA_K_COUNT).  Synchronises that step.  */
+int epara_step_profile(epara_ctx*, float* ms_per_kind, int* launches_per_kind);
+
+int epara_destroy(epara_ctx*);
+const char* epara_strerror(int status);
+
+/* Bytes of workspace epara_register_model will reserve for this model under cfg. */
+size_t epara_model_workspace_bytes(const epara_config* cfg, const epara_model_desc* m);
+
+/* ---- host policy, exposed for testing and for callers that plan ahead (pure host code) ---- */
+
+/* Eq. 4: DP group count = ceil(required frame rate / frame rate of one group). */
+int epara_dp_group_count(double required_fps, double group_fps);
+/* Eq. 5: inter-request count = floor(BS / max inter-frame count). */
+int epara_inter_request_count(int bs, int mf_max);
+/* Admission of one queue (the rule epara_step applies).  Arrays are host memory of n entries in
+ * arrival order; out_admitted/out_dropped need room for n entries.  Returns EPARA_OK. */
+int epara_admit_queue(int n, const uint64_t* tickets, const long long* deadline_ns, const int* streams,
+                      long long now_ns, int cap, int mf_max,
+                      uint64_t* out_admitted, int* n_admitted, uint64_t* out_dropped, int* n_dropped);
+
+/* ---- single-kernel entry points (the same kernels a step launches), for parity tests and
+ *      roofline measurement.  All pointers device unless named host. ---- */
+
+typedef struct {
+  const void* A;      /* bf16 [M, lda]  */
+  const void* W;      /* bf16 [N, ldw], K contiguous */
+  void* C;            /* bf16 [M, ldc] (or fp32 when EPARA_EPI_RESID_F32); SwiGLU: [M, N/2] */
+  const void* bias;   /* bf16 [N] or NULL */
+  int M, N, K;
+  int lda, ldw, ldc;  /* elements; multiples of 8 */
+  int epilogue;       /* EPARA_EPI_* flags */
+} epara_gemm_problem;
+
+enum { EPARA_EPI_BIAS = 1, EPARA_EPI_GELU = 2, EPARA_EPI_SWIGLU = 4, EPARA_EPI_RESID_F32 = 8 };
+
+/* C_g = epilogue(A_g W_g^T + bias_g) for every problem in one grouped launch.  RESID_F32:
+ * C is fp32 and is updated in place, C += A W^T + bias.  `problems` is host memory;
+ * `scratch` is device memory of at least epara_gemm_scratch_bytes(n) bytes. */
+int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm_problem* problems, int n,
+                       void* scratch, size_t scratch_bytes);
+size_t epara_gemm_scratch_bytes(int n_problems);
+
+/* Split-KV paged decode attention with GQA (one layer).  q: bf16 [B, q_stride] (head h at
+ * column h*hd); kv_layer: bf16 [pages][2][Hkv][16][hd]; kv_lens int32 [B] = tokens to attend
+ * (cached + appended); tables: int32 [B, table_stride]; out bf16 [B, Hq*hd];
+ * scratch: at least epara_decode_attention_scratch_bytes(B, Hq, hd, max_len) bytes. */
+int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
+                           const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out,
+                           int B, int Hq, int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes);
+size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EPARA_H */

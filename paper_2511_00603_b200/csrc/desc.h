@@ -1,0 +1,121 @@
+// Device-visible descriptors written by the host step planner and read by the kernels.
+// One step uploads one blob holding the request table and, per launch, an array of groups
+// (one group = one model's problem in that launch).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace epara {
+
+typedef __nv_bfloat16 bf16;
+
+enum : int { EPI_BIAS = 1, EPI_GELU = 2, EPI_SWIGLU = 4, EPI_RESID_F32 = 8 };
+
+// Per admitted request (model order, then batch order).
+struct ReqDesc {
+  const void* input;     // MLP row / ViT image
+  const int32_t* table;  // decoder block table
+  void* out_logits;
+  int32_t* out_argmax;
+  int token;
+  int kv_len;            // cached tokens before this step
+  int n_blocks;
+  int pad;
+};
+
+// C = epi(A W^T + bias).  tmA/tmW are the TMA maps of A [rows, K] and W [N, K] (K innermost,
+// 128-byte swizzle, box 64 x 128 rows for A and 64 x BN rows for W).
+struct alignas(64) GemmGroup {
+  CUtensorMap tmA;
+  CUtensorMap tmW;
+  const bf16* A;
+  const bf16* W;
+  void* C;
+  const bf16* bias;
+  int M, N, K;
+  int lda, ldw, ldc;
+  int epi;
+  int tile_start;  // first tile index of this group in the launch
+  int tiles_m, tiles_n;
+  int pad0, pad1;
+};
+
+struct GemmLaunch {      // header followed by groups
+  int n_groups;
+  int total_tiles;
+};
+
+enum : int { NORM_LN = 0, NORM_RMS = 1 };
+struct NormGroup {
+  const float* x;        // fp32 [M rows, row stride x_stride]
+  bf16* y;               // bf16 [M, d]
+  const bf16* gamma;
+  const bf16* beta;      // LN only
+  long long x_stride;
+  int M, d, kind;
+  float eps;
+};
+
+enum : int { GATHER_ROWS = 0, GATHER_EMB = 1, GATHER_PATCH = 2 };
+struct GatherGroup {
+  const ReqDesc* reqs;
+  void* out;             // ROWS: bf16 [B, ld]; EMB: fp32 [B, d]; PATCH: bf16 [B*np, 3*p*p]
+  const bf16* emb;       // EMB
+  int kind, B, width, ld;
+  int img, patch;
+  int blocks;            // blocks this group needs
+  int pad;
+};
+
+struct RopeGroup {
+  bf16* qkv;             // [B, (Hq+2Hkv)*hd], q rotated in place
+  bf16* kv_layer;        // [pages][2][Hkv][16][hd]
+  const ReqDesc* reqs;
+  const double* inv_freq;  // [hd/2]
+  int B, Hq, Hkv, hd;
+};
+
+struct AttnReq {
+  const int32_t* table;
+  int len;               // tokens to attend (cached + appended)
+  int pad;
+};
+
+struct AttnDecGroup {
+  const bf16* q;         // [B, q_stride], head h at column h*hd
+  const bf16* kv_layer;
+  const AttnReq* reqs;
+  bf16* out;             // [B, Hq*hd]
+  float* partial;        // [B][Hq][max_chunks][hd + 2]  (m, l, o[hd])
+  int q_stride;
+  int B, Hq, Hkv, hd;
+  int max_chunks;
+  int req_start;         // first grid.z index of this group
+  int pad;
+};
+
+struct AttnEncGroup {
+  const bf16* qkv;       // [B*T, 3d]: q | k | v, head h at column h*hd within each
+  bf16* out;             // [B*T, d]
+  int B, T, H, hd;
+  int blk_start;         // first block of this group
+  int q_blocks;          // query blocks per (image, head)
+  int pad0, pad1;
+};
+
+struct AssembleGroup {   // z[b, 0] = cls + pos[0]; z[b, 1+p] = E[b*np + p] + pos[1+p]
+  const bf16* E;
+  const bf16* cls;
+  const bf16* pos;
+  float* z;
+  int B, T, d, pad;
+};
+
+struct OutputGroup {     // copy logits rows to the requests' buffers and take the argmax
+  const bf16* logits;    // [B, ld]
+  const ReqDesc* reqs;
+  int B, N, ld, pad;
+};
+
+}  // namespace epara

@@ -1,0 +1,982 @@
+// C ABI, category table, admission and step planner (host code).
+//
+// epara_register_model turns a model into a static list of ops (gather, norm, GEMM, RoPE+append,
+// attention, ...) over buffers carved from the caller's workspace, with the TMA maps of every
+// GEMM operand built once.  epara_step admits requests per (model, category), then walks all
+// active models' op lists together: in each sweep over the kernel kinds, every model whose next
+// op is of that kind contributes one group to a single grouped launch (MT: different services in
+// one launch; BS: a group's M is its batch).  All descriptors of the step travel in one pinned
+// blob with one host-to-device copy.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <chrono>
+#include <cmath>
+#include <cstring>
+#include <deque>
+#include <new>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/epara.h"
+#include "desc.h"
+#include "kernels.h"
+
+using namespace epara;
+
+namespace {
+
+constexpr int N_SLOTS = 4;
+constexpr size_t BLOB_BYTES = 4u << 20;
+constexpr int MAX_PROFILE_LAUNCHES = 4096;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
+
+// ---- TMA map encoding through the runtime's driver entry point (no link against libcuda) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+// bf16 matrix [rows, cols] with leading dimension ld, cols innermost; box = 64 cols x box_rows,
+// 128-byte swizzle, out-of-range elements read as zero.
+bool make_tmap(CUtensorMap* tm, const void* ptr, long long rows, long long cols, long long ld, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Op {
+  int kind;           // EPARA_K_*
+  int rows_per_req;   // rows of this op = batch * rows_per_req
+  GemmGroup gemm;
+  NormGroup norm;
+  GatherGroup gather;
+  RopeGroup rope;
+  AttnDecGroup adec;
+  AttnEncGroup aenc;
+  AssembleGroup asmb;
+  OutputGroup outp;
+  double weight_bytes;
+};
+
+struct Request {
+  uint64_t ticket;
+  epara_inputs in;
+};
+
+enum { T_QUEUED = 0, T_INFLIGHT = 1, T_DROPPED = 2 };
+struct Ticket {
+  int state;
+  int model;
+  uint64_t step;
+  void* out_logits;
+  int32_t* out_argmax;
+};
+
+struct Model {
+  epara_model_desc d;
+  std::vector<const void*> tensors;
+  std::vector<int> dims;
+  int max_batch;
+  int n_out;
+  std::vector<Op> ops;
+  std::deque<Request> q[2];
+  int max_chunks;       // decoder
+  double kv_bytes_per_token;
+};
+
+struct Slot {
+  unsigned char* host;  // pinned blob
+  unsigned char* dev;   // device blob (in the workspace)
+  int* status_host;     // pinned
+  cudaEvent_t done;
+  uint64_t step_id;     // 0 = never used
+  bool busy;
+  std::vector<cudaEvent_t> prof;   // 2 per launch when profiling
+  std::vector<int> prof_kind;
+};
+
+struct Launch {
+  int kind;
+  size_t off;
+  int n_groups;
+  int p0, p1, p2, p3;
+};
+
+}  // namespace
+
+struct epara_ctx {
+  epara_config cfg;
+  int sm_count;
+  unsigned char* ws;
+  size_t ws_bytes, ws_used;
+  int* dev_status;
+  std::vector<Model*> models;
+  std::unordered_map<uint64_t, Ticket> tickets;
+  uint64_t next_ticket, next_step;
+  Slot slots[N_SLOTS];
+  uint64_t last_step_slot;
+};
+
+namespace {
+
+void* carve(epara_ctx* c, size_t bytes) {
+  const size_t off = align_up(c->ws_used, 256);
+  if (off + bytes > c->ws_bytes) return nullptr;
+  c->ws_used = off + bytes;
+  return c->ws + off;
+}
+
+size_t carve_size(size_t& used, size_t bytes) {
+  const size_t off = align_up(used, 256);
+  used = off + bytes;
+  return off;
+}
+
+struct Buf {
+  void* p;
+};
+
+// Builds the op list of a model.  With c == nullptr only counts workspace bytes (in *need).
+// Buffers are requested through `get`, which either carves or counts.
+struct Builder {
+  epara_ctx* c;
+  size_t need;
+  bool fail;
+  void* get(size_t bytes) {
+    if (!c) { carve_size(need, bytes); return reinterpret_cast<void*>(size_t(256)); }
+    void* p = carve(c, bytes);
+    if (!p) fail = true;
+    return p;
+  }
+};
+
+bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap, const void* W, int N, int K,
+              void* C, int ldc, const void* bias, int epi, int rows_per_req) {
+  Op op;
+  memset(&op, 0, sizeof(op));
+  op.kind = EPARA_K_GEMM;
+  op.rows_per_req = rows_per_req;
+  GemmGroup& g = op.gemm;
+  g.A = (const bf16*)A; g.W = (const bf16*)W; g.C = C; g.bias = (const bf16*)bias;
+  g.N = N; g.K = K; g.lda = lda; g.ldw = K; g.ldc = ldc; g.epi = epi | (bias ? EPI_BIAS : 0);
+  op.weight_bytes = 2.0 * N * K;
+  if (bl.c) {
+    if (!make_tmap(&g.tmA, A, rows_cap, K, lda, TC_BM)) return false;
+    if (!make_tmap(&g.tmW, W, N, K, K, TC_BN)) return false;
+  }
+  m->ops.push_back(op);
+  return true;
+}
+
+void add_norm(Model* m, const float* x, long long x_stride, bf16* y, const void* gamma, const void* beta, int d,
+              int kind, float eps, int rows_per_req) {
+  Op op;
+  memset(&op, 0, sizeof(op));
+  op.kind = EPARA_K_NORM;
+  op.rows_per_req = rows_per_req;
+  op.norm.x = x; op.norm.y = y; op.norm.gamma = (const bf16*)gamma; op.norm.beta = (const bf16*)beta;
+  op.norm.x_stride = x_stride; op.norm.d = d; op.norm.kind = kind; op.norm.eps = eps;
+  m->ops.push_back(op);
+}
+
+int validate_desc(const epara_model_desc* d) {
+  if (!d || !d->tensors) return EPARA_E_INVALID;
+  for (int i = 0; i < d->n_tensors; ++i)
+    if (!d->tensors[i] || (reinterpret_cast<uintptr_t>(d->tensors[i]) & 15)) return EPARA_E_INVALID;
+  if (d->n_layers <= 0) return EPARA_E_INVALID;
+  switch (d->kind) {
+    case EPARA_MODEL_MLP:
+      if (!d->mlp_dims || d->n_tensors != 2 * d->n_layers) return EPARA_E_INVALID;
+      for (int i = 0; i < d->n_layers; ++i)
+        if (d->mlp_dims[i] <= 0 || d->mlp_dims[i] % 8) return EPARA_E_INVALID;
+      if (d->mlp_dims[d->n_layers] <= 0) return EPARA_E_INVALID;
+      return EPARA_OK;
+    case EPARA_MODEL_VIT:
+      if (d->n_tensors != 4 + 12 * d->n_layers + 4) return EPARA_E_INVALID;
+      if (d->d <= 0 || d->d % 8 || d->d > 8192 || d->n_heads <= 0 || d->d != d->n_heads * d->head_dim)
+        return EPARA_E_INVALID;
+      if (d->head_dim != 64) return EPARA_E_UNSUPPORTED;
+      if (d->patch <= 0 || d->patch % 8 || d->img <= 0 || d->img % d->patch || d->img % 8) return EPARA_E_INVALID;
+      if (d->ffn <= 0 || d->ffn % 8 || d->vocab <= 0) return EPARA_E_INVALID;
+      return EPARA_OK;
+    case EPARA_MODEL_DECODER: {
+      if (d->n_tensors != 1 + 6 * d->n_layers + 2) return EPARA_E_INVALID;
+      if (d->d <= 0 || d->d % 8 || d->d > 8192 || d->ffn <= 0 || d->ffn % 8 || d->vocab <= 0) return EPARA_E_INVALID;
+      if (d->n_heads <= 0 || d->n_kv_heads <= 0 || d->n_heads % d->n_kv_heads) return EPARA_E_INVALID;
+      const int g = d->n_heads / d->n_kv_heads, hd = d->head_dim;
+      const bool hd_ok = hd == 16 || hd == 32 || hd == 64 || hd == 128;
+      const bool g_ok = g == 1 || g == 2 || g == 4 || (g == 8 && hd >= 64);
+      if (!hd_ok || !g_ok) return EPARA_E_UNSUPPORTED;
+      if (!d->kv_pool || (reinterpret_cast<uintptr_t>(d->kv_pool) & 15) || d->kv_pages <= 0 || d->max_kv_len < 0)
+        return EPARA_E_INVALID;
+      return EPARA_OK;
+    }
+    default:
+      return EPARA_E_INVALID;
+  }
+}
+
+int build_model(Builder& bl, Model* m, const epara_config& cfg) {
+  const epara_model_desc& d = m->d;
+  const int B = m->max_batch;
+  const long long Bcap = round_up(B, TC_BM);
+  const void* const* t = m->tensors.data();
+  if (d.kind == EPARA_MODEL_MLP) {
+    const int L = d.n_layers;
+    int maxw = 0;
+    for (int i = 1; i <= L; ++i) maxw = std::max(maxw, round_up(m->dims[i], 8));
+    bf16* x0 = (bf16*)bl.get((size_t)Bcap * m->dims[0] * 2);
+    bf16* pp[2] = {(bf16*)bl.get((size_t)Bcap * maxw * 2), (bf16*)bl.get((size_t)Bcap * maxw * 2)};
+    if (bl.fail) return EPARA_E_RESOURCE;
+    Op g;
+    memset(&g, 0, sizeof(g));
+    g.kind = EPARA_K_GATHER; g.rows_per_req = 1;
+    g.gather.kind = GATHER_ROWS; g.gather.out = x0; g.gather.width = m->dims[0]; g.gather.ld = m->dims[0];
+    m->ops.push_back(g);
+    const bf16* in = x0;
+    int ld_in = m->dims[0];
+    for (int l = 0; l < L; ++l) {
+      const int N = m->dims[l + 1], K = m->dims[l], ldc = round_up(N, 8);
+      bf16* out = pp[l & 1];
+      if (!add_gemm(bl, m, in, ld_in, Bcap, t[2 * l], N, K, out, ldc, t[2 * l + 1], (l + 1 < L) ? EPI_GELU : 0, 1))
+        return EPARA_E_CUDA;
+      in = out; ld_in = ldc;
+    }
+    Op o;
+    memset(&o, 0, sizeof(o));
+    o.kind = EPARA_K_OUTPUT; o.rows_per_req = 1;
+    o.outp.logits = in; o.outp.N = m->dims[L]; o.outp.ld = ld_in;
+    m->ops.push_back(o);
+    m->n_out = m->dims[L];
+    return EPARA_OK;
+  }
+  if (d.kind == EPARA_MODEL_VIT) {
+    const int dm = d.d, T = (d.img / d.patch) * (d.img / d.patch) + 1, np = T - 1;
+    const int pk = 3 * d.patch * d.patch;
+    const long long Mcap = round_up(B * T, TC_BM);
+    const int fw = std::max(d.ffn, pk);
+    float* z = (float*)bl.get((size_t)Mcap * dm * 4);
+    bf16* h = (bf16*)bl.get((size_t)Mcap * dm * 2);
+    bf16* qkv = (bf16*)bl.get((size_t)Mcap * 3 * dm * 2);
+    bf16* a = (bf16*)bl.get((size_t)Mcap * dm * 2);
+    bf16* f = (bf16*)bl.get((size_t)Mcap * fw * 2);
+    bf16* cvec = (bf16*)bl.get((size_t)Bcap * dm * 2);
+    const int ldl = round_up(d.vocab, 8);
+    bf16* logits = (bf16*)bl.get((size_t)Bcap * ldl * 2);
+    if (bl.fail) return EPARA_E_RESOURCE;
+    Op g;
+    memset(&g, 0, sizeof(g));
+    g.kind = EPARA_K_GATHER; g.rows_per_req = np;
+    g.gather.kind = GATHER_PATCH; g.gather.out = f; g.gather.width = pk; g.gather.ld = pk;
+    g.gather.img = d.img; g.gather.patch = d.patch;
+    m->ops.push_back(g);
+    if (!add_gemm(bl, m, f, pk, Mcap, t[0], dm, pk, a, dm, t[1], 0, np)) return EPARA_E_CUDA;
+    Op as;
+    memset(&as, 0, sizeof(as));
+    as.kind = EPARA_K_ASSEMBLE; as.rows_per_req = T;
+    as.asmb.E = a; as.asmb.cls = (const bf16*)t[2]; as.asmb.pos = (const bf16*)t[3]; as.asmb.z = z;
+    as.asmb.T = T; as.asmb.d = dm;
+    m->ops.push_back(as);
+    for (int l = 0; l < d.n_layers; ++l) {
+      const void* const* w = t + 4 + 12 * l;
+      add_norm(m, z, dm, h, w[0], w[1], dm, NORM_LN, 1e-6f, T);
+      if (!add_gemm(bl, m, h, dm, Mcap, w[2], 3 * dm, dm, qkv, 3 * dm, w[3], 0, T)) return EPARA_E_CUDA;
+      Op at;
+      memset(&at, 0, sizeof(at));
+      at.kind = EPARA_K_ATTN_ENC; at.rows_per_req = T;
+      at.aenc.qkv = qkv; at.aenc.out = a; at.aenc.T = T; at.aenc.H = d.n_heads; at.aenc.hd = d.head_dim;
+      m->ops.push_back(at);
+      if (!add_gemm(bl, m, a, dm, Mcap, w[4], dm, dm, z, dm, w[5], EPI_RESID_F32, T)) return EPARA_E_CUDA;
+      add_norm(m, z, dm, h, w[6], w[7], dm, NORM_LN, 1e-6f, T);
+      if (!add_gemm(bl, m, h, dm, Mcap, w[8], d.ffn, dm, f, d.ffn, w[9], EPI_GELU, T)) return EPARA_E_CUDA;
+      if (!add_gemm(bl, m, f, d.ffn, Mcap, w[10], dm, d.ffn, z, dm, w[11], EPI_RESID_F32, T)) return EPARA_E_CUDA;
+    }
+    const void* const* w = t + 4 + 12 * d.n_layers;
+    add_norm(m, z, (long long)T * dm, cvec, w[0], w[1], dm, NORM_LN, 1e-6f, 1);
+    if (!add_gemm(bl, m, cvec, dm, Bcap, w[2], d.vocab, dm, logits, ldl, w[3], 0, 1)) return EPARA_E_CUDA;
+    Op o;
+    memset(&o, 0, sizeof(o));
+    o.kind = EPARA_K_OUTPUT; o.rows_per_req = 1;
+    o.outp.logits = logits; o.outp.N = d.vocab; o.outp.ld = ldl;
+    m->ops.push_back(o);
+    m->n_out = d.vocab;
+    return EPARA_OK;
+  }
+  // decoder
+  const int dm = d.d, Hq = d.n_heads, Hkv = d.n_kv_heads, hd = d.head_dim, F = d.ffn;
+  const int nq = (Hq + 2 * Hkv) * hd;
+  m->max_chunks = (d.max_kv_len + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK;
+  m->kv_bytes_per_token = 2.0 * Hkv * hd * 2.0 * d.n_layers;
+  float* x = (float*)bl.get((size_t)Bcap * dm * 4);
+  bf16* h = (bf16*)bl.get((size_t)Bcap * dm * 2);
+  bf16* qkv = (bf16*)bl.get((size_t)Bcap * nq * 2);
+  bf16* a = (bf16*)bl.get((size_t)Bcap * Hq * hd * 2);
+  bf16* f = (bf16*)bl.get((size_t)Bcap * F * 2);
+  const int ldl = round_up(d.vocab, 8);
+  bf16* logits = (bf16*)bl.get((size_t)Bcap * ldl * 2);
+  float* partial = (float*)bl.get((size_t)B * Hq * m->max_chunks * (hd + 2) * 4);
+  double* inv_freq = (double*)bl.get((size_t)(hd / 2) * 8);
+  if (bl.fail) return EPARA_E_RESOURCE;
+  if (bl.c) {
+    std::vector<double> f64(hd / 2);
+    for (int j = 0; j < hd / 2; ++j) f64[j] = std::pow(10000.0, -2.0 * j / hd);
+    if (cudaMemcpy(inv_freq, f64.data(), f64.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess) return EPARA_E_CUDA;
+  }
+  Op g;
+  memset(&g, 0, sizeof(g));
+  g.kind = EPARA_K_GATHER; g.rows_per_req = 1;
+  g.gather.kind = GATHER_EMB; g.gather.out = x; g.gather.emb = (const bf16*)t[0]; g.gather.width = dm; g.gather.ld = dm;
+  m->ops.push_back(g);
+  const size_t layer_elems = (size_t)d.kv_pages * 2 * Hkv * 16 * hd;
+  for (int l = 0; l < d.n_layers; ++l) {
+    const void* const* w = t + 1 + 6 * l;
+    bf16* kv_layer = (bf16*)d.kv_pool + layer_elems * l;
+    add_norm(m, x, dm, h, w[0], nullptr, dm, NORM_RMS, 1e-5f, 1);
+    if (!add_gemm(bl, m, h, dm, Bcap, w[1], nq, dm, qkv, nq, nullptr, 0, 1)) return EPARA_E_CUDA;
+    Op r;
+    memset(&r, 0, sizeof(r));
+    r.kind = EPARA_K_ROPE; r.rows_per_req = 1;
+    r.rope.qkv = qkv; r.rope.kv_layer = kv_layer; r.rope.inv_freq = inv_freq;
+    r.rope.Hq = Hq; r.rope.Hkv = Hkv; r.rope.hd = hd;
+    m->ops.push_back(r);
+    Op at;
+    memset(&at, 0, sizeof(at));
+    at.kind = EPARA_K_ATTN_DEC; at.rows_per_req = 1;
+    at.adec.q = qkv; at.adec.q_stride = nq; at.adec.kv_layer = kv_layer; at.adec.out = a; at.adec.partial = partial;
+    at.adec.Hq = Hq; at.adec.Hkv = Hkv; at.adec.hd = hd; at.adec.max_chunks = m->max_chunks;
+    m->ops.push_back(at);
+    if (!add_gemm(bl, m, a, Hq * hd, Bcap, w[2], dm, Hq * hd, x, dm, nullptr, EPI_RESID_F32, 1)) return EPARA_E_CUDA;
+    add_norm(m, x, dm, h, w[3], nullptr, dm, NORM_RMS, 1e-5f, 1);
+    if (!add_gemm(bl, m, h, dm, Bcap, w[4], 2 * F, dm, f, F, nullptr, EPI_SWIGLU, 1)) return EPARA_E_CUDA;
+    if (!add_gemm(bl, m, f, F, Bcap, w[5], dm, F, x, dm, nullptr, EPI_RESID_F32, 1)) return EPARA_E_CUDA;
+  }
+  const void* const* w = t + 1 + 6 * d.n_layers;
+  add_norm(m, x, dm, h, w[0], nullptr, dm, NORM_RMS, 1e-5f, 1);
+  if (!add_gemm(bl, m, h, dm, Bcap, w[1], d.vocab, dm, logits, ldl, nullptr, 0, 1)) return EPARA_E_CUDA;
+  Op o;
+  memset(&o, 0, sizeof(o));
+  o.kind = EPARA_K_OUTPUT; o.rows_per_req = 1;
+  o.outp.logits = logits; o.outp.N = d.vocab; o.outp.ld = ldl;
+  m->ops.push_back(o);
+  m->n_out = d.vocab;
+  return EPARA_OK;
+}
+
+int effective_max_batch(const epara_config& cfg, const epara_model_desc& d) {
+  const int ls = cfg.cap_ls > 0 ? cfg.cap_ls : 4, fs = cfg.cap_fs > 0 ? cfg.cap_fs : 256;
+  return d.max_batch > 0 ? d.max_batch : ls + fs;
+}
+
+void admit_impl(int n, const uint64_t* tickets, const long long* deadline, const int* streams, long long now, int cap,
+                int mf_max, std::vector<int>& admitted, std::vector<int>& dropped) {
+  std::vector<int> live;
+  for (int i = 0; i < n; ++i) {
+    if (deadline[i] != 0 && deadline[i] < now) dropped.push_back(i); else live.push_back(i);
+  }
+  if (mf_max <= 0) {
+    for (int i = 0; i < (int)live.size() && i < cap; ++i) admitted.push_back(live[i]);
+    return;
+  }
+  const int n_streams = cap / mf_max;   // Eq. 5
+  std::vector<int> order;
+  for (int i : live)
+    if (std::find(order.begin(), order.end(), streams[i]) == order.end()) order.push_back(streams[i]);
+  if ((int)order.size() > n_streams) order.resize(n_streams);
+  if (order.empty()) return;
+  int f = mf_max;
+  for (int s : order) {
+    int cnt = 0;
+    for (int i : live) cnt += streams[i] == s;
+    f = std::min(f, cnt);
+  }
+  for (int s : order) {
+    int cnt = 0;
+    for (int i : live)
+      if (streams[i] == s && cnt < f) { admitted.push_back(i); ++cnt; }
+  }
+  (void)tickets;
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+extern "C" {
+
+const char* epara_strerror(int s) {
+  switch (s) {
+    case EPARA_OK: return "ok";
+    case EPARA_PENDING: return "pending";
+    case EPARA_E_INVALID: return "invalid argument";
+    case EPARA_E_UNSUPPORTED: return "unsupported (needs more than one GPU, or an unsupported shape)";
+    case EPARA_E_TIMEOUT: return "timeout";
+    case EPARA_E_RESOURCE: return "resource insufficiency";
+    case EPARA_E_DEVICE: return "device-side error";
+    case EPARA_E_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+int epara_dp_group_count(double required_fps, double group_fps) {
+  if (!(group_fps > 0) || !(required_fps >= 0)) return EPARA_E_INVALID;
+  return (int)std::ceil(required_fps / group_fps);
+}
+
+int epara_inter_request_count(int bs, int mf_max) {
+  if (bs < 0 || mf_max <= 0) return EPARA_E_INVALID;
+  return bs / mf_max;
+}
+
+int epara_admit_queue(int n, const uint64_t* tickets, const long long* deadline_ns, const int* streams,
+                      long long now_ns, int cap, int mf_max, uint64_t* out_admitted, int* n_admitted,
+                      uint64_t* out_dropped, int* n_dropped) {
+  if (n < 0 || (n > 0 && (!tickets || !deadline_ns || !streams)) || !n_admitted || !n_dropped || cap < 0)
+    return EPARA_E_INVALID;
+  std::vector<int> a, d;
+  admit_impl(n, tickets, deadline_ns, streams, now_ns, cap, mf_max, a, d);
+  for (size_t i = 0; i < a.size(); ++i) out_admitted[i] = tickets[a[i]];
+  for (size_t i = 0; i < d.size(); ++i) out_dropped[i] = tickets[d[i]];
+  *n_admitted = (int)a.size();
+  *n_dropped = (int)d.size();
+  return EPARA_OK;
+}
+
+size_t epara_model_workspace_bytes(const epara_config* cfg, const epara_model_desc* d) {
+  if (!cfg || validate_desc(d) != EPARA_OK) return 0;
+  Model m;
+  m.d = *d;
+  m.tensors.assign(d->tensors, d->tensors + d->n_tensors);
+  if (d->kind == EPARA_MODEL_MLP) m.dims.assign(d->mlp_dims, d->mlp_dims + d->n_layers + 1);
+  m.max_batch = effective_max_batch(*cfg, *d);
+  Builder bl{nullptr, 0, false};
+  build_model(bl, &m, *cfg);
+  return bl.need + 256;
+}
+
+int epara_init(const epara_config* cfg, epara_ctx** out) {
+  if (!cfg || !out) return EPARA_E_INVALID;
+  if (!cfg->workspace || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255)) return EPARA_E_INVALID;
+  const size_t fixed = N_SLOTS * BLOB_BYTES + 256;
+  if (cfg->workspace_bytes < fixed) return EPARA_E_RESOURCE;
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return EPARA_E_CUDA;
+  epara_ctx* c = new (std::nothrow) epara_ctx();
+  if (!c) return EPARA_E_RESOURCE;
+  c->cfg = *cfg;
+  if (c->cfg.cap_ls <= 0) c->cfg.cap_ls = 4;
+  if (c->cfg.cap_fs <= 0) c->cfg.cap_fs = 256;
+  if (c->cfg.max_queue <= 0) c->cfg.max_queue = 4096;
+  c->ws = (unsigned char*)cfg->workspace;
+  c->ws_bytes = cfg->workspace_bytes;
+  c->ws_used = 0;
+  c->next_ticket = 1;
+  c->next_step = 1;
+  c->last_step_slot = 0;
+  int sm = 0;
+  if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) { delete c; return EPARA_E_CUDA; }
+  c->sm_count = sm;
+  c->dev_status = (int*)carve(c, 256);
+  if (cudaMemset(c->dev_status, 0, 256) != cudaSuccess) { delete c; return EPARA_E_CUDA; }
+  for (int i = 0; i < N_SLOTS; ++i) {
+    Slot& s = c->slots[i];
+    s.dev = (unsigned char*)carve(c, BLOB_BYTES);
+    s.step_id = 0;
+    s.busy = false;
+    if (cudaMallocHost((void**)&s.host, BLOB_BYTES) != cudaSuccess ||
+        cudaMallocHost((void**)&s.status_host, 64) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) != cudaSuccess) {
+      return EPARA_E_CUDA;
+    }
+    *s.status_host = 0;
+  }
+  *out = c;
+  return EPARA_OK;
+}
+
+int epara_destroy(epara_ctx* c) {
+  if (!c) return EPARA_E_INVALID;
+  cudaSetDevice(c->cfg.device);
+  for (int i = 0; i < N_SLOTS; ++i) {
+    Slot& s = c->slots[i];
+    if (s.busy) cudaEventSynchronize(s.done);
+    for (cudaEvent_t e : s.prof) cudaEventDestroy(e);
+    cudaEventDestroy(s.done);
+    cudaFreeHost(s.host);
+    cudaFreeHost(s.status_host);
+  }
+  for (Model* m : c->models) delete m;
+  delete c;
+  return EPARA_OK;
+}
+
+int epara_register_model(epara_ctx* c, const epara_model_desc* d, int* model_id) {
+  if (!c || !model_id) return EPARA_E_INVALID;
+  int v = validate_desc(d);
+  if (v != EPARA_OK) return v;
+  if (cudaSetDevice(c->cfg.device) != cudaSuccess) return EPARA_E_CUDA;
+  Model* m = new (std::nothrow) Model();
+  if (!m) return EPARA_E_RESOURCE;
+  m->d = *d;
+  m->tensors.assign(d->tensors, d->tensors + d->n_tensors);
+  if (d->kind == EPARA_MODEL_MLP) m->dims.assign(d->mlp_dims, d->mlp_dims + d->n_layers + 1);
+  m->d.tensors = nullptr;
+  m->d.mlp_dims = nullptr;
+  m->max_batch = effective_max_batch(c->cfg, *d);
+  m->max_chunks = 0;
+  m->kv_bytes_per_token = 0;
+  const size_t mark = c->ws_used;
+  Builder bl{c, 0, false};
+  int r = build_model(bl, m, c->cfg);
+  if (r != EPARA_OK) {
+    c->ws_used = mark;
+    delete m;
+    return r;
+  }
+  c->models.push_back(m);
+  *model_id = (int)c->models.size() - 1;
+  return EPARA_OK;
+}
+
+int epara_submit(epara_ctx* c, int model_id, int category, const epara_inputs* in, uint64_t* ticket) {
+  if (!c || !in || !ticket) return EPARA_E_INVALID;
+  if (model_id < 0 || model_id >= (int)c->models.size()) return EPARA_E_INVALID;
+  if (category == EPARA_CAT_LS_GT1 || category == EPARA_CAT_FS_GT1) return EPARA_E_UNSUPPORTED;
+  if (category != EPARA_CAT_LS_LT1 && category != EPARA_CAT_FS_LT1) return EPARA_E_INVALID;
+  Model* m = c->models[model_id];
+  if (!in->out_logits && !in->out_argmax) return EPARA_E_INVALID;
+  if (reinterpret_cast<uintptr_t>(in->out_logits) & 1) return EPARA_E_INVALID;
+  if (m->d.kind == EPARA_MODEL_DECODER) {
+    if (!in->block_table || in->kv_len < 0 || in->kv_len > m->d.max_kv_len) return EPARA_E_INVALID;
+    if (in->n_blocks < in->kv_len / EPARA_KV_PAGE + 1) return EPARA_E_INVALID;
+    if (in->token < 0 || in->token >= m->d.vocab) return EPARA_E_INVALID;
+  } else {
+    if (!in->input || (reinterpret_cast<uintptr_t>(in->input) & 15)) return EPARA_E_INVALID;
+  }
+  if ((int)m->q[category].size() >= c->cfg.max_queue) return EPARA_E_RESOURCE;
+  Request r;
+  r.ticket = c->next_ticket++;
+  r.in = *in;
+  m->q[category].push_back(r);
+  Ticket t;
+  t.state = T_QUEUED; t.model = model_id; t.step = 0; t.out_logits = in->out_logits; t.out_argmax = in->out_argmax;
+  c->tickets[r.ticket] = t;
+  *ticket = r.ticket;
+  return EPARA_OK;
+}
+
+int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_info* info) {
+  if (!c) return EPARA_E_INVALID;
+  if (cudaSetDevice(c->cfg.device) != cudaSuccess) return EPARA_E_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (now_ns < 0)
+    now_ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now().time_since_epoch()).count();
+  epara_step_info inf;
+  memset(&inf, 0, sizeof(inf));
+  const uint64_t step_id = c->next_step++;
+  inf.step_id = step_id;
+
+  // ---- admission (A0) ----
+  struct Active { Model* m; int B; size_t req_off; size_t areq_off; size_t cursor; std::vector<Request> reqs; };
+  std::vector<Active> act;
+  for (size_t mi = 0; mi < c->models.size(); ++mi) {
+    Model* m = c->models[mi];
+    Active a;
+    a.m = m; a.B = 0; a.cursor = 0; a.req_off = 0; a.areq_off = 0;
+    for (int cat = 0; cat < 2; ++cat) {
+      std::deque<Request>& q = m->q[cat];
+      if (q.empty()) continue;
+      const int n = (int)q.size();
+      std::vector<uint64_t> tk(n);
+      std::vector<long long> dl(n);
+      std::vector<int> sid(n);
+      for (int i = 0; i < n; ++i) { tk[i] = q[i].ticket; dl[i] = q[i].in.deadline_ns; sid[i] = q[i].in.stream; }
+      int cap = (cat == EPARA_CAT_LS_LT1) ? c->cfg.cap_ls : c->cfg.cap_fs;
+      cap = std::min(cap, m->max_batch - a.B);
+      std::vector<int> adm, drp;
+      admit_impl(n, tk.data(), dl.data(), sid.data(), now_ns, cap, (cat == EPARA_CAT_FS_LT1) ? c->cfg.mf_max : 0, adm, drp);
+      std::vector<char> gone(n, 0);
+      for (int i : adm) { a.reqs.push_back(q[i]); gone[i] = 1; c->tickets[q[i].ticket].state = T_INFLIGHT; c->tickets[q[i].ticket].step = step_id; }
+      for (int i : drp) { gone[i] = 1; c->tickets[q[i].ticket].state = T_DROPPED; }
+      std::deque<Request> rest;
+      for (int i = 0; i < n; ++i) if (!gone[i]) rest.push_back(q[i]);
+      q.swap(rest);
+      inf.admitted[cat] += (int)adm.size();
+      inf.dropped[cat] += (int)drp.size();
+      a.B += (int)adm.size();
+    }
+    if (a.B > 0) act.push_back(std::move(a));
+  }
+  if (act.empty()) {
+    if (info) *info = inf;
+    return EPARA_OK;
+  }
+
+  // ---- blob slot ----
+  Slot& slot = c->slots[step_id % N_SLOTS];
+  if (slot.busy) {
+    if (cudaEventSynchronize(slot.done) != cudaSuccess) return EPARA_E_CUDA;
+    slot.busy = false;
+  }
+  size_t off = 0;
+  auto put = [&](const void* src, size_t bytes, size_t align) -> size_t {
+    off = align_up(off, align);
+    if (off + bytes > BLOB_BYTES) return (size_t)-1;
+    memcpy(slot.host + off, src, bytes);
+    const size_t at = off;
+    off += bytes;
+    return at;
+  };
+  bool overflow = false;
+  for (Active& a : act) {
+    std::vector<ReqDesc> rd(a.B);
+    std::vector<AttnReq> ar(a.B);
+    for (int b = 0; b < a.B; ++b) {
+      const epara_inputs& in = a.reqs[b].in;
+      rd[b].input = in.input; rd[b].table = in.block_table; rd[b].out_logits = in.out_logits;
+      rd[b].out_argmax = in.out_argmax; rd[b].token = in.token; rd[b].kv_len = in.kv_len;
+      rd[b].n_blocks = in.n_blocks; rd[b].pad = 0;
+      ar[b].table = in.block_table; ar[b].len = in.kv_len + 1; ar[b].pad = 0;
+      if (a.m->d.kind == EPARA_MODEL_DECODER) inf.kv_bytes += a.m->kv_bytes_per_token * in.kv_len;
+    }
+    a.req_off = put(rd.data(), rd.size() * sizeof(ReqDesc), 16);
+    if (a.m->d.kind == EPARA_MODEL_DECODER) a.areq_off = put(ar.data(), ar.size() * sizeof(AttnReq), 16);
+    if (a.req_off == (size_t)-1 || a.areq_off == (size_t)-1) overflow = true;
+  }
+
+  // ---- plan (A1): sweep the kernel kinds until every model's op list is exhausted ----
+  static const int sweep[] = {EPARA_K_GATHER, EPARA_K_ASSEMBLE, EPARA_K_NORM, EPARA_K_GEMM, EPARA_K_ROPE,
+                              EPARA_K_ATTN_DEC, EPARA_K_ATTN_ENC, EPARA_K_OUTPUT};
+  std::vector<Launch> launches;
+  const bool simt = c->cfg.gemm_impl == EPARA_GEMM_SIMT;
+  bool more = true;
+  while (more && !overflow) {
+    more = false;
+    for (int kind : sweep) {
+      std::vector<Active*> who;
+      for (Active& a : act)
+        if (a.cursor < a.m->ops.size() && a.m->ops[a.cursor].kind == kind) who.push_back(&a);
+      if (who.empty()) continue;
+      more = true;
+      Launch L;
+      memset(&L, 0, sizeof(L));
+      L.kind = kind;
+      L.n_groups = (int)who.size();
+      off = align_up(off, 64);
+      L.off = off;
+      if (kind == EPARA_K_ATTN_DEC) {
+        // decode attention is templated on (hd, G): one launch per distinct pair
+        std::vector<Active*> rest = who;
+        bool first = true;
+        while (!rest.empty()) {
+          const Op& o0 = rest[0]->m->ops[rest[0]->cursor];
+          const int hd = o0.adec.hd, G = o0.adec.Hq / o0.adec.Hkv;
+          std::vector<Active*> same, other;
+          for (Active* a : rest) {
+            const Op& o = a->m->ops[a->cursor];
+            ((o.adec.hd == hd && o.adec.Hq / o.adec.Hkv == G) ? same : other).push_back(a);
+          }
+          Launch LL;
+          memset(&LL, 0, sizeof(LL));
+          LL.kind = kind; LL.n_groups = (int)same.size();
+          off = align_up(off, 64);
+          LL.off = off;
+          int total_B = 0, max_hkv = 0, max_hq = 0, max_chunks = 0;
+          for (Active* a : same) {
+            AttnDecGroup g = a->m->ops[a->cursor].adec;
+            g.B = a->B; g.reqs = (const AttnReq*)(slot.dev + a->areq_off); g.req_start = total_B;
+            total_B += a->B;
+            max_hkv = std::max(max_hkv, g.Hkv); max_hq = std::max(max_hq, g.Hq);
+            for (int b = 0; b < a->B; ++b)
+              max_chunks = std::max(max_chunks, (a->reqs[b].in.kv_len + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK);
+            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+          }
+          LL.p0 = total_B; LL.p1 = max_hkv; LL.p2 = max_chunks; LL.p3 = (hd << 8) | G;
+          launches.push_back(LL);
+          Launch LC = LL;
+          LC.kind = EPARA_K_ATTN_COMBINE; LC.p1 = max_hq;
+          launches.push_back(LC);
+          rest.swap(other);
+          (void)first;
+        }
+        for (Active* a : who) a->cursor++;
+        continue;
+      }
+      int total = 0, mx = 0;
+      for (Active* a : who) {
+        const Op& op = a->m->ops[a->cursor];
+        const int rows = a->B * op.rows_per_req;
+        switch (kind) {
+          case EPARA_K_GATHER: {
+            GatherGroup g = op.gather;
+            g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B; g.blocks = rows;
+            mx = std::max(mx, rows);
+            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            break;
+          }
+          case EPARA_K_ASSEMBLE: {
+            AssembleGroup g = op.asmb;
+            g.B = a->B;
+            mx = std::max(mx, rows);
+            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            break;
+          }
+          case EPARA_K_NORM: {
+            NormGroup g = op.norm;
+            g.M = rows;
+            mx = std::max(mx, rows);
+            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            break;
+          }
+          case EPARA_K_GEMM: {
+            GemmGroup g = op.gemm;
+            g.M = rows;
+            const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : TC_BN;
+            g.tiles_m = (rows + tm - 1) / tm; g.tiles_n = (g.N + tn - 1) / tn;
+            g.tile_start = total;
+            total += g.tiles_m * g.tiles_n;
+            inf.gemm_groups++;
+            inf.gemm_flops += 2.0 * rows * g.N * g.K;
+            inf.weight_bytes += op.weight_bytes;
+            if (put(&g, sizeof(g), 64) == (size_t)-1) overflow = true;
+            break;
+          }
+          case EPARA_K_ROPE: {
+            RopeGroup g = op.rope;
+            g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
+            mx = std::max(mx, a->B);
+            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            break;
+          }
+          case EPARA_K_ATTN_ENC: {
+            AttnEncGroup g = op.aenc;
+            g.B = a->B; g.q_blocks = attn_encoder_q_blocks(g.T); g.blk_start = total;
+            total += a->B * g.H * g.q_blocks;
+            mx = std::max(mx, g.T);
+            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            break;
+          }
+          case EPARA_K_OUTPUT: {
+            OutputGroup g = op.outp;
+            g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
+            mx = std::max(mx, a->B);
+            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            break;
+          }
+        }
+        a->cursor++;
+      }
+      L.p0 = total; L.p1 = mx;
+      launches.push_back(L);
+    }
+  }
+  if (overflow) {
+    // nothing was launched: give the admitted requests a definite answer
+    for (Active& a : act)
+      for (Request& r : a.reqs) c->tickets[r.ticket].state = T_DROPPED;
+    if (info) *info = inf;
+    return EPARA_E_RESOURCE;
+  }
+
+  // ---- upload + launch ----
+  if (cudaMemcpyAsync(slot.dev, slot.host, off, cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
+  const bool prof = c->cfg.profile != 0;
+  if (prof) {
+    if (launches.size() > MAX_PROFILE_LAUNCHES) return EPARA_E_RESOURCE;
+    while (slot.prof.size() < 2 * launches.size()) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return EPARA_E_CUDA;
+      slot.prof.push_back(e);
+    }
+    slot.prof_kind.clear();
+  }
+  cudaError_t err = cudaSuccess;
+  int li = 0;
+  for (const Launch& L : launches) {
+    const unsigned char* gp = slot.dev + L.off;
+    if (prof) { cudaEventRecord(slot.prof[2 * li], st); slot.prof_kind.push_back(L.kind); }
+    switch (L.kind) {
+      case EPARA_K_GATHER: launch_gather((const GatherGroup*)gp, L.n_groups, L.p1, st); break;
+      case EPARA_K_ASSEMBLE: launch_assemble((const AssembleGroup*)gp, L.n_groups, L.p1, st); break;
+      case EPARA_K_NORM: launch_norm((const NormGroup*)gp, L.n_groups, L.p1, st); break;
+      case EPARA_K_GEMM:
+        if (simt) launch_gemm_simt((const GemmGroup*)gp, L.n_groups, L.p0, st);
+        else err = launch_gemm_tc((const GemmGroup*)gp, L.n_groups, L.p0, c->dev_status, c->sm_count, st);
+        break;
+      case EPARA_K_ROPE: launch_rope_append((const RopeGroup*)gp, L.n_groups, L.p1, st); break;
+      case EPARA_K_ATTN_DEC:
+        err = launch_attn_decode((const AttnDecGroup*)gp, L.n_groups, L.p0, L.p1, L.p2, L.p3 >> 8, L.p3 & 255, st);
+        break;
+      case EPARA_K_ATTN_COMBINE:
+        err = launch_attn_combine((const AttnDecGroup*)gp, L.n_groups, L.p0, L.p1, L.p3 >> 8, st);
+        break;
+      case EPARA_K_ATTN_ENC: err = launch_attn_encoder((const AttnEncGroup*)gp, L.n_groups, L.p0, L.p1, st); break;
+      case EPARA_K_OUTPUT: launch_output((const OutputGroup*)gp, L.n_groups, L.p1, st); break;
+    }
+    if (prof) cudaEventRecord(slot.prof[2 * li + 1], st);
+    ++li;
+    if (err != cudaSuccess) break;
+  }
+  if (err == cudaSuccess) err = cudaGetLastError();
+  cudaMemcpyAsync(slot.status_host, c->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  cudaEventRecord(slot.done, st);
+  slot.busy = true;
+  slot.step_id = step_id;
+  c->last_step_slot = step_id % N_SLOTS;
+  inf.launches = (int)launches.size();
+  if (info) *info = inf;
+  return err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
+}
+
+int epara_collect(epara_ctx* c, uint64_t ticket, epara_output* out) {
+  if (!c) return EPARA_E_INVALID;
+  auto it = c->tickets.find(ticket);
+  if (it == c->tickets.end()) return EPARA_E_INVALID;
+  Ticket& t = it->second;
+  if (t.state == T_QUEUED) return EPARA_PENDING;
+  int result = EPARA_OK;
+  if (t.state == T_DROPPED) {
+    result = EPARA_E_TIMEOUT;
+  } else {
+    Slot& s = c->slots[t.step % N_SLOTS];
+    if (s.step_id == t.step && s.busy) {
+      cudaError_t e = cudaEventQuery(s.done);
+      if (e == cudaErrorNotReady) return EPARA_PENDING;
+      if (e != cudaSuccess) return EPARA_E_CUDA;
+      s.busy = false;
+    }
+    if (s.step_id == t.step && *s.status_host != 0) result = EPARA_E_DEVICE;
+  }
+  if (out) {
+    out->status = result;
+    out->step_id = t.step;
+    out->logits = t.out_logits;
+    out->argmax = t.out_argmax;
+    out->n_out = c->models[t.model]->n_out;
+  }
+  c->tickets.erase(it);
+  return result;
+}
+
+int epara_step_profile(epara_ctx* c, float* ms_per_kind, int* launches_per_kind) {
+  if (!c || !ms_per_kind || !launches_per_kind) return EPARA_E_INVALID;
+  if (!c->cfg.profile) return EPARA_E_UNSUPPORTED;
+  Slot& s = c->slots[c->last_step_slot];
+  if (s.step_id == 0) return EPARA_E_INVALID;
+  if (cudaEventSynchronize(s.done) != cudaSuccess) return EPARA_E_CUDA;
+  for (int k = 0; k < EPARA_K_COUNT; ++k) { ms_per_kind[k] = 0.f; launches_per_kind[k] = 0; }
+  for (size_t i = 0; i < s.prof_kind.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, s.prof[2 * i], s.prof[2 * i + 1]) != cudaSuccess) return EPARA_E_CUDA;
+    ms_per_kind[s.prof_kind[i]] += ms;
+    launches_per_kind[s.prof_kind[i]]++;
+  }
+  return EPARA_OK;
+}
+
+// ---------------------------------------------------------------- single-kernel entry points
+size_t epara_gemm_scratch_bytes(int n) { return (size_t)(n > 0 ? n : 0) * sizeof(GemmGroup) + 256; }
+
+int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm_problem* p, int n, void* scratch,
+                       size_t scratch_bytes) {
+  if (n < 0 || (n > 0 && !p) || !scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return EPARA_E_INVALID;
+  if (scratch_bytes < epara_gemm_scratch_bytes(n)) return EPARA_E_RESOURCE;
+  if (n == 0) return EPARA_OK;
+  if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const bool simt = impl == EPARA_GEMM_SIMT;
+  std::vector<GemmGroup> gs(n);
+  int total = 0;
+  for (int i = 0; i < n; ++i) {
+    const epara_gemm_problem& q = p[i];
+    if (!q.A || !q.W || !q.C || q.M < 0 || q.N <= 0 || q.K <= 0) return EPARA_E_INVALID;
+    if ((q.lda % 8) || (q.ldw % 8) || q.lda < q.K || q.ldw < q.K) return EPARA_E_INVALID;
+    if ((reinterpret_cast<uintptr_t>(q.A) & 15) || (reinterpret_cast<uintptr_t>(q.W) & 15) ||
+        (reinterpret_cast<uintptr_t>(q.C) & 15))
+      return EPARA_E_INVALID;
+    if ((q.epilogue & EPARA_EPI_SWIGLU) && (q.N % 2 || (q.epilogue & EPARA_EPI_RESID_F32))) return EPARA_E_INVALID;
+    if ((q.epilogue & EPARA_EPI_BIAS) && !q.bias) return EPARA_E_INVALID;
+    GemmGroup& g = gs[i];
+    memset(&g, 0, sizeof(g));
+    g.A = (const bf16*)q.A; g.W = (const bf16*)q.W; g.C = q.C; g.bias = (const bf16*)q.bias;
+    g.M = q.M; g.N = q.N; g.K = q.K; g.lda = q.lda; g.ldw = q.ldw; g.ldc = q.ldc; g.epi = q.epilogue;
+    const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : TC_BN;
+    g.tiles_m = (q.M + tm - 1) / tm; g.tiles_n = (q.N + tn - 1) / tn;
+    g.tile_start = total;
+    total += g.tiles_m * g.tiles_n;
+    if (!simt && q.M > 0) {
+      if (!make_tmap(&g.tmA, q.A, q.M, q.K, q.lda, TC_BM)) return EPARA_E_CUDA;
+      if (!make_tmap(&g.tmW, q.W, q.N, q.K, q.ldw, TC_BN)) return EPARA_E_CUDA;
+    }
+  }
+  int* status = (int*)scratch;
+  GemmGroup* dev_groups = (GemmGroup*)((unsigned char*)scratch + 256);
+  if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) return EPARA_E_CUDA;
+  if (cudaMemcpyAsync(dev_groups, gs.data(), gs.size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return EPARA_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return EPARA_E_CUDA;   // gs is pageable host memory
+  cudaError_t err = cudaSuccess;
+  if (simt) {
+    launch_gemm_simt(dev_groups, n, total, st);
+    err = cudaGetLastError();
+  } else {
+    int sm = 0;
+    cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device);
+    err = launch_gemm_tc(dev_groups, n, total, status, sm, st);
+  }
+  return err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
+}
+
+size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len) {
+  const int chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK;
+  return 256 + align_up((size_t)B * sizeof(AttnReq), 256) + (size_t)B * Hq * chunks * (hd + 2) * 4;
+}
+
+int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
+                           const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out, int B, int Hq,
+                           int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes) {
+  if (!q || !kv_layer || !kv_lens || !tables || !out || !scratch || B < 0 || Hkv <= 0 || Hq % Hkv || max_len <= 0)
+    return EPARA_E_INVALID;
+  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(kv_layer) & 15) || (q_stride % 8) ||
+      (reinterpret_cast<uintptr_t>(scratch) & 255))
+    return EPARA_E_INVALID;
+  if (scratch_bytes < epara_decode_attention_scratch_bytes(B, Hq, hd, max_len)) return EPARA_E_RESOURCE;
+  if (B == 0) return EPARA_OK;
+  if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  unsigned char* s = (unsigned char*)scratch;
+  AttnDecGroup g;
+  memset(&g, 0, sizeof(g));
+  AttnReq* reqs = (AttnReq*)(s + 256);
+  g.q = (const bf16*)q; g.q_stride = q_stride; g.kv_layer = (const bf16*)kv_layer; g.reqs = reqs; g.out = (bf16*)out;
+  g.partial = (float*)(s + 256 + align_up((size_t)B * sizeof(AttnReq), 256));
+  g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK; g.req_start = 0;
+  if (cudaMemcpyAsync(s, &g, sizeof(g), cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return EPARA_E_CUDA;
+  launch_attn_fill_reqs(reqs, kv_lens, tables, table_stride, B, st);
+  cudaError_t e = launch_attn_decode((const AttnDecGroup*)s, 1, B, Hkv, g.max_chunks, hd, Hq / Hkv, st);
+  if (e == cudaErrorInvalidValue) return EPARA_E_UNSUPPORTED;
+  if (e != cudaSuccess) return EPARA_E_CUDA;
+  e = launch_attn_combine((const AttnDecGroup*)s, 1, B, Hq, hd, st);
+  return e == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
+}
+
+}  // extern "C"

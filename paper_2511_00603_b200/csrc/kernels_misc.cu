@@ -1,0 +1,232 @@
+// Bandwidth-trivial kernels of a step: input gather / embedding / patchify, LayerNorm and
+// RMSNorm, RoPE + KV append, ViT token assembly, logits scatter + argmax.
+// Every launch is grouped: blockIdx.y selects the group (one model), blockIdx.x a unit of work
+// inside it; blocks beyond a group's extent return at once.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace epara {
+
+// ------------------------------------------------------------------ gather
+__global__ void __launch_bounds__(128) gather_kernel(const GatherGroup* __restrict__ groups) {
+  const GatherGroup g = groups[blockIdx.y];
+  if ((int)blockIdx.x >= g.blocks) return;
+  if (g.kind == GATHER_ROWS) {
+    const int b = blockIdx.x;
+    const uint4* src = reinterpret_cast<const uint4*>(g.reqs[b].input);
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(g.out) + (size_t)b * g.ld);
+    for (int i = threadIdx.x; i < g.width / 8; i += blockDim.x) dst[i] = src[i];
+  } else if (g.kind == GATHER_EMB) {
+    const int b = blockIdx.x;
+    const int tok = g.reqs[b].token;
+    const uint4* src = reinterpret_cast<const uint4*>(g.emb + (size_t)tok * g.width);
+    float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(g.out) + (size_t)b * g.width);
+    for (int i = threadIdx.x; i < g.width / 8; i += blockDim.x) {
+      float f[8];
+      unpack8(src[i], f);
+      dst[2 * i] = make_float4(f[0], f[1], f[2], f[3]);
+      dst[2 * i + 1] = make_float4(f[4], f[5], f[6], f[7]);
+    }
+  } else {  // GATHER_PATCH: row (b*np + i*gw + j), column c*p*p + u*p + v  <-  img[b][c][p*i+u][p*j+v]
+    const int p = g.patch, gw = g.img / p, np = gw * gw;
+    const int b = blockIdx.x / np, pi = blockIdx.x % np;
+    const int i = pi / gw, j = pi % gw;
+    const bf16* img = reinterpret_cast<const bf16*>(g.reqs[b].input);
+    bf16* dst = reinterpret_cast<bf16*>(g.out) + (size_t)blockIdx.x * g.width;
+    const int vec_per_row = p / 8;
+    for (int e = threadIdx.x; e < g.width / 8; e += blockDim.x) {
+      const int cu = e / vec_per_row, v8 = e % vec_per_row;   // cu = c*p + u
+      const int c = cu / p, u = cu % p;
+      const bf16* s = img + ((size_t)c * g.img + (size_t)(p * i + u)) * g.img + p * j + v8 * 8;
+      reinterpret_cast<uint4*>(dst)[e] = *reinterpret_cast<const uint4*>(s);
+    }
+  }
+}
+
+void launch_gather(const GatherGroup* groups, int n_groups, int max_blocks, cudaStream_t st) {
+  if (n_groups == 0 || max_blocks == 0) return;
+  gather_kernel<<<dim3(max_blocks, n_groups), 128, 0, st>>>(groups);
+}
+
+// ------------------------------------------------------------------ norms
+// One block per row; the row is held in registers (d <= 128 threads * 16 float4 = 8192).
+__global__ void __launch_bounds__(128) norm_kernel(const NormGroup* __restrict__ groups) {
+  __shared__ float red[32];
+  const NormGroup g = groups[blockIdx.y];
+  const int row = blockIdx.x;
+  if (row >= g.M) return;
+  const int nvec = g.d >> 2;
+  const float4* x = reinterpret_cast<const float4*>(g.x + (size_t)row * g.x_stride);
+  float4 v[16];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int c = threadIdx.x + i * 128;
+    if (c < nvec) {
+      v[i] = x[c];
+      s += (g.kind == NORM_LN) ? (v[i].x + v[i].y) + (v[i].z + v[i].w)
+                               : (v[i].x * v[i].x + v[i].y * v[i].y) + (v[i].z * v[i].z + v[i].w * v[i].w);
+    }
+  }
+  s = block_sum(s, red);
+  float mean = 0.f, rstd;
+  const float inv_d = 1.0f / (float)g.d;
+  if (g.kind == NORM_LN) {
+    mean = s * inv_d;
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int c = threadIdx.x + i * 128;
+      if (c < nvec) {
+        const float a = v[i].x - mean, b = v[i].y - mean, cc = v[i].z - mean, dd = v[i].w - mean;
+        q += (a * a + b * b) + (cc * cc + dd * dd);
+      }
+    }
+    q = block_sum(q, red);
+    rstd = 1.0f / sqrtf(q * inv_d + g.eps);
+  } else {
+    rstd = 1.0f / sqrtf(s * inv_d + g.eps);
+  }
+  uint2* y = reinterpret_cast<uint2*>(g.y + (size_t)row * g.d);
+  const uint2* gm = reinterpret_cast<const uint2*>(g.gamma);
+  const uint2* bt = reinterpret_cast<const uint2*>(g.beta);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int c = threadIdx.x + i * 128;
+    if (c < nvec) {
+      const uint2 gg = gm[c];
+      float ga[4] = {__uint_as_float(gg.x << 16), __uint_as_float(gg.x & 0xffff0000u),
+                     __uint_as_float(gg.y << 16), __uint_as_float(gg.y & 0xffff0000u)};
+      float be[4] = {0.f, 0.f, 0.f, 0.f};
+      if (g.kind == NORM_LN) {
+        const uint2 bb = bt[c];
+        be[0] = __uint_as_float(bb.x << 16); be[1] = __uint_as_float(bb.x & 0xffff0000u);
+        be[2] = __uint_as_float(bb.y << 16); be[3] = __uint_as_float(bb.y & 0xffff0000u);
+      }
+      uint2 o;
+      o.x = pack2((v[i].x - mean) * rstd * ga[0] + be[0], (v[i].y - mean) * rstd * ga[1] + be[1]);
+      o.y = pack2((v[i].z - mean) * rstd * ga[2] + be[2], (v[i].w - mean) * rstd * ga[3] + be[3]);
+      y[c] = o;
+    }
+  }
+}
+
+void launch_norm(const NormGroup* groups, int n_groups, int max_rows, cudaStream_t st) {
+  if (n_groups == 0 || max_rows == 0) return;
+  norm_kernel<<<dim3(max_rows, n_groups), 128, 0, st>>>(groups);
+}
+
+// ------------------------------------------------------------------ RoPE + KV append
+// One block per request.  The new token sits at position kv_len: q and k are rotated there
+// (interleaved pairs, angle pos * inv_freq[j], fp64 angle), q in place, k and v written to the
+// cache page table[pos/16], slot pos%16.
+__global__ void __launch_bounds__(128) rope_append_kernel(const RopeGroup* __restrict__ groups) {
+  __shared__ float cs[128], sn[128];
+  const RopeGroup g = groups[blockIdx.y];
+  const int b = blockIdx.x;
+  if (b >= g.B) return;
+  const ReqDesc r = g.reqs[b];
+  const int pos = r.kv_len, hd = g.hd, half = hd >> 1;
+  for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    double s, c;
+    sincos((double)pos * g.inv_freq[j], &s, &c);
+    cs[j] = (float)c;
+    sn[j] = (float)s;
+  }
+  __syncthreads();
+  const int page = r.table[pos / 16], slot = pos % 16;
+  bf16* row = g.qkv + (size_t)b * (g.Hq + 2 * g.Hkv) * hd;
+  const int n_rot = (g.Hq + g.Hkv) * half;
+  for (int e = threadIdx.x; e < n_rot; e += blockDim.x) {
+    const int h = e / half, j = e % half;
+    __nv_bfloat162* p2 = reinterpret_cast<__nv_bfloat162*>(row + (size_t)h * hd) + j;
+    const float2 v = __bfloat1622float2(*p2);
+    const float x0 = v.x * cs[j] - v.y * sn[j], x1 = v.x * sn[j] + v.y * cs[j];
+    const __nv_bfloat162 o = __floats2bfloat162_rn(x0, x1);
+    if (h < g.Hq) {
+      *p2 = o;
+    } else {
+      const int kh = h - g.Hq;
+      bf16* dst = g.kv_layer + (((size_t)page * 2 + 0) * g.Hkv + kh) * 16 * hd + (size_t)slot * hd;
+      reinterpret_cast<__nv_bfloat162*>(dst)[j] = o;
+    }
+  }
+  const bf16* vsrc = row + (size_t)(g.Hq + g.Hkv) * hd;
+  for (int e = threadIdx.x; e < g.Hkv * half; e += blockDim.x) {
+    const int kh = e / half, j = e % half;
+    bf16* dst = g.kv_layer + (((size_t)page * 2 + 1) * g.Hkv + kh) * 16 * hd + (size_t)slot * hd;
+    reinterpret_cast<__nv_bfloat162*>(dst)[j] = reinterpret_cast<const __nv_bfloat162*>(vsrc + (size_t)kh * hd)[j];
+  }
+}
+
+void launch_rope_append(const RopeGroup* groups, int n_groups, int max_B, cudaStream_t st) {
+  if (n_groups == 0 || max_B == 0) return;
+  rope_append_kernel<<<dim3(max_B, n_groups), 128, 0, st>>>(groups);
+}
+
+// ------------------------------------------------------------------ ViT token assembly
+__global__ void __launch_bounds__(128) assemble_kernel(const AssembleGroup* __restrict__ groups) {
+  const AssembleGroup g = groups[blockIdx.y];
+  const int row = blockIdx.x;
+  if (row >= g.B * g.T) return;
+  const int b = row / g.T, t = row % g.T;
+  const bf16* src = (t == 0) ? g.cls : g.E + ((size_t)b * (g.T - 1) + (t - 1)) * g.d;
+  const bf16* pos = g.pos + (size_t)t * g.d;
+  float* z = g.z + (size_t)row * g.d;
+  for (int i = threadIdx.x; i < g.d / 8; i += blockDim.x) {
+    float a[8], p[8];
+    unpack8(reinterpret_cast<const uint4*>(src)[i], a);
+    unpack8(reinterpret_cast<const uint4*>(pos)[i], p);
+    reinterpret_cast<float4*>(z)[2 * i] = make_float4(a[0] + p[0], a[1] + p[1], a[2] + p[2], a[3] + p[3]);
+    reinterpret_cast<float4*>(z)[2 * i + 1] = make_float4(a[4] + p[4], a[5] + p[5], a[6] + p[6], a[7] + p[7]);
+  }
+}
+
+void launch_assemble(const AssembleGroup* groups, int n_groups, int max_rows, cudaStream_t st) {
+  if (n_groups == 0 || max_rows == 0) return;
+  assemble_kernel<<<dim3(max_rows, n_groups), 128, 0, st>>>(groups);
+}
+
+// ------------------------------------------------------------------ output scatter + argmax
+// One block per request: copies its logits row to the request's buffer and writes the index of
+// the maximum (lowest index on ties; NaNs never win).
+__global__ void __launch_bounds__(256) output_kernel(const OutputGroup* __restrict__ groups) {
+  __shared__ float sv[8];
+  __shared__ int si[8];
+  const OutputGroup g = groups[blockIdx.y];
+  const int b = blockIdx.x;
+  if (b >= g.B) return;
+  const ReqDesc r = g.reqs[b];
+  const bf16* src = g.logits + (size_t)b * g.ld;
+  bf16* dst = reinterpret_cast<bf16*>(r.out_logits);
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int i = threadIdx.x; i < g.N; i += blockDim.x) {
+    const bf16 v = src[i];
+    if (dst) dst[i] = v;
+    const float f = bf2f(v);
+    if (f > best || (f == best && i < bi)) { best = f; bi = i; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+  }
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) { sv[w] = best; si[w] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int k = 1; k < 8; ++k)
+      if (sv[k] > best || (sv[k] == best && si[k] < bi)) { best = sv[k]; bi = si[k]; }
+    if (bi == 0x7fffffff) bi = 0;
+    if (r.out_argmax) *r.out_argmax = bi;
+  }
+}
+
+void launch_output(const OutputGroup* groups, int n_groups, int max_B, cudaStream_t st) {
+  if (n_groups == 0 || max_B == 0) return;
+  output_kernel<<<dim3(max_B, n_groups), 256, 0, st>>>(groups);
+}
+
+}  // namespace epara

@@ -1,0 +1,47 @@
+"""Shared helpers of the GPU parity tests."""
+import math
+
+import numpy as np
+import torch
+
+REL_TOL = 2e-2   # max relative error per output element (bf16 storage, fp32 accumulate)
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def max_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+    """max |g - r| / max(|r|, rho), rho = RMS of the reference tensor: the per-element relative
+    error with elements near zero measured against the tensor's scale."""
+    ref = np.asarray(ref, dtype=np.float64)
+    rho = math.sqrt(float(np.mean(ref * ref))) if ref.size else 0.0
+    den = np.maximum(np.abs(ref), max(rho, 1e-30))
+    return float(np.max(np.abs(got - ref) / den)) if ref.size else 0.0
+
+
+def assert_close(got, ref, what="", tol=REL_TOL):
+    g = to_f64(got) if isinstance(got, torch.Tensor) else np.asarray(got, dtype=np.float64)
+    assert np.all(np.isfinite(g)), f"{what}: non-finite output"
+    e = max_rel_err(g.reshape(-1), np.asarray(ref).reshape(-1))
+    assert e <= tol, f"{what}: max relative error {e:.3e} > {tol}"
+    return e
+
+
+def check_argmax(gpu_argmax: int, gpu_logits: torch.Tensor, ref_logits: np.ndarray, tol=REL_TOL):
+    """(i) the device argmax equals the lowest-index argmax of the device's own logits, bit-exact;
+    (ii) it equals the reference argmax when the reference's top-2 gap exceeds twice the tolerance
+    band; (iii) otherwise it must be one of the reference entries inside that band.
+    Returns True when the case was decided by (ii)."""
+    own = to_f64(gpu_logits)
+    assert gpu_argmax == int(np.argmax(own)), "argmax kernel disagrees with its own logits"
+    ref = np.asarray(ref_logits, dtype=np.float64)
+    rho = math.sqrt(float(np.mean(ref * ref)))
+    order = np.argsort(-ref, kind="stable")
+    top1, top2 = ref[order[0]], ref[order[1]] if ref.size > 1 else -np.inf
+    band = 2 * tol * max(abs(top1), rho)
+    if top1 - top2 > band:
+        assert gpu_argmax == int(order[0]), "argmax differs from the oracle outside the tie band"
+        return True
+    assert ref[gpu_argmax] >= top1 - band, "argmax is not among the oracle's near-maximal entries"
+    return False

@@ -1,0 +1,147 @@
+"""GPU parity of the single kernels against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import epara_oracle as O
+from paper_2511_00603_b200 import synth
+from tests.parity import assert_close, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2511_00603_b200 import build
+    build.build()
+    from paper_2511_00603_b200 import epara
+    return epara
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+GEMM_CASES = [
+    # M, N, K, epilogue flags (names)
+    (8, 512, 512, ("bias", "gelu")),
+    (32, 1024, 256, ("bias",)),
+    (197, 2304, 768, ("bias",)),
+    (1, 3072, 2048, ()),
+    (130, 10, 512, ("bias",)),          # N below one tile, not a multiple of 8
+    (300, 1000, 768, ("bias",)),        # ragged M and N
+    (33, 512, 256, ("swiglu",)),
+    (77, 768, 3072, ("bias", "resid")),
+    (0, 64, 64, ()),                    # empty group
+    (257, 136, 64, ("gelu", "bias")),   # single k-block, N tail of 8
+]
+
+
+def _run_gemm(E, impl, cases, seed=0):
+    dev = torch.device("cuda")
+    g = torch.Generator(device=dev).manual_seed(seed)
+    probs, refs = [], []
+    for (M, N, K, fl) in cases:
+        A = torch.randn((max(M, 1), K), generator=g, device=dev).to(torch.bfloat16)
+        W = (torch.randn((N, K), generator=g, device=dev) * 0.05).to(torch.bfloat16)
+        bias = (torch.randn((N,), generator=g, device=dev) * 0.5).to(torch.bfloat16) if "bias" in fl else None
+        epi = (E.EPI_BIAS if "bias" in fl else 0) | (E.EPI_GELU if "gelu" in fl else 0) | \
+              (E.EPI_SWIGLU if "swiglu" in fl else 0) | (E.EPI_RESID_F32 if "resid" in fl else 0)
+        ldc = ((N // 2 if "swiglu" in fl else N) + 7) // 8 * 8
+        if "resid" in fl:
+            Cc = torch.randn((max(M, 1), ldc), generator=g, device=dev, dtype=torch.float32)
+        else:
+            Cc = torch.full((max(M, 1), ldc), float("nan"), device=dev, dtype=torch.bfloat16)
+        C0 = Cc.clone()
+        probs.append({"A": A, "W": W, "C": Cc, "bias": bias, "M": M, "N": N, "K": K, "epilogue": epi})
+        # oracle
+        y = O.linear(O.bf16_to_f64(synth.to_bits(A))[:M], O.bf16_to_f64(synth.to_bits(W)),
+                     O.bf16_to_f64(synth.to_bits(bias)) if bias is not None else None)
+        if "gelu" in fl:
+            y = O.gelu(y)
+        if "swiglu" in fl:
+            y = O.silu(y[:, 0::2]) * y[:, 1::2]
+        if "resid" in fl:
+            y = C0[:M, :N].double().cpu().numpy() + y
+        refs.append(y)
+    scratch = torch.empty(E.lib.epara_gemm_scratch_bytes(len(probs)), dtype=torch.uint8, device=dev)
+    E.epara_grouped_gemm(probs, _stream(), scratch, impl=impl)
+    torch.cuda.synchronize()
+    status = int(scratch[:4].view(torch.int32).item())
+    assert status == 0, f"device status {status}"
+    return probs, refs
+
+
+@pytest.mark.parametrize("impl", ["simt", "tcgen05"])
+def test_grouped_gemm_matches_oracle(E, impl):
+    probs, refs = _run_gemm(E, E.GEMM_SIMT if impl == "simt" else E.GEMM_TCGEN05, GEMM_CASES)
+    for p, ref, case in zip(probs, refs, GEMM_CASES):
+        M, ncols = ref.shape
+        if M == 0:
+            continue
+        assert_close(p["C"][:M, :ncols], ref, what=f"{impl} gemm {case}")
+        if p["C"].dtype == torch.bfloat16 and p["C"].shape[1] > ncols:
+            assert torch.isnan(p["C"][:M, ncols:].float()).all(), "wrote beyond N"
+
+
+def test_grouped_gemm_many_tiles_and_group_independence(E):
+    """More tiles than SMs, several k-blocks beyond the stage ring, and the same problem alone vs
+    among others gives bit-identical output (no dependence on co-resident groups)."""
+    big = [(1576, 768, 768, ("bias",)), (640, 3072, 768, ("bias", "gelu")), (1000, 768, 3072, ("bias", "resid"))]
+    probs, refs = _run_gemm(E, E.GEMM_TCGEN05, big, seed=3)
+    for p, ref, case in zip(probs, refs, big):
+        assert_close(p["C"][:ref.shape[0], :ref.shape[1]], ref, what=f"gemm {case}")
+    alone, _ = _run_gemm(E, E.GEMM_TCGEN05, big[:1], seed=3)
+    assert torch.equal(alone[0]["C"], probs[0]["C"])
+
+
+def test_grouped_gemm_rejects_bad_arguments(E):
+    dev = torch.device("cuda")
+    A = torch.zeros((8, 64), device=dev, dtype=torch.bfloat16)
+    W = torch.zeros((8, 64), device=dev, dtype=torch.bfloat16)
+    Cc = torch.zeros((8, 8), device=dev, dtype=torch.bfloat16)
+    scratch = torch.empty(4096, dtype=torch.uint8, device=dev)
+    bad = {"A": A[:, 1:], "W": W, "C": Cc, "M": 8, "N": 8, "K": 63, "epilogue": 0}
+    with pytest.raises(E.EparaError) as ei:
+        E.epara_grouped_gemm([bad], _stream(), scratch)
+    assert ei.value.status == E.E_INVALID
+    small = torch.empty(256, dtype=torch.uint8, device=dev)
+    ok = {"A": A, "W": W, "C": Cc, "M": 8, "N": 8, "K": 64, "epilogue": 0}
+    with pytest.raises(E.EparaError) as ei:
+        E.epara_grouped_gemm([ok], _stream(), small)
+    assert ei.value.status == E.E_RESOURCE
+
+
+@pytest.mark.parametrize("Hq,Hkv,hd", [(8, 2, 64), (8, 2, 128), (4, 4, 64), (4, 2, 16)])
+def test_decode_attention_matches_oracle(E, Hq, Hkv, hd):
+    dev = torch.device("cuda")
+    lens = np.array([1, 16, 17, 255, 256, 257, 700, 1023], dtype=np.int32)
+    B = len(lens)
+    need = [(int(L) + 15) // 16 for L in lens]
+    npages = sum(need) + 3
+    rng = np.random.default_rng(5)
+    perm = rng.permutation(npages).astype(np.int32)
+    stride = max(need)
+    tables = np.zeros((B, stride), dtype=np.int32)
+    o = 0
+    for b, n in enumerate(need):
+        tables[b, :n] = perm[o:o + n]
+        o += n
+    pool = synth.make_kv_pool(1, npages, Hkv, hd, seed=6, device=dev)[0]
+    # poison the slots past each request's length: they must never be read
+    pool_ref = synth.to_bits(pool)
+    for b, L in enumerate(lens):
+        if L % 16:
+            pool[int(tables[b, need[b] - 1]), :, :, L % 16:, :] = float("nan")
+    q = torch.randn((B, Hq * hd), generator=torch.Generator(device=dev).manual_seed(7), device=dev).to(torch.bfloat16)
+    out = torch.empty((B, Hq * hd), device=dev, dtype=torch.bfloat16)
+    max_len = int(lens.max())
+    scratch = torch.empty(E.lib.epara_decode_attention_scratch_bytes(B, Hq, hd, max_len), dtype=torch.uint8, device=dev)
+    E.epara_decode_attention(q, pool, torch.as_tensor(lens, device=dev), torch.as_tensor(tables, device=dev), out,
+                             Hq, Hkv, hd, max_len, scratch, _stream())
+    torch.cuda.synchronize()
+    qf = O.bf16_to_f64(synth.to_bits(q)).reshape(B, Hq, hd)
+    for b, L in enumerate(lens):
+        K, V = O.gather_kv(lambda l, pg: pool_ref[pg], 0, tables[b], int(L))
+        ref = np.stack([O.attention(qf[b, h], K[h // (Hq // Hkv)], V[h // (Hq // Hkv)]) for h in range(Hq)])
+        assert_close(out[b].reshape(Hq, hd), ref, what=f"decode attention b={b} L={L}")

@@ -1,0 +1,259 @@
+"""GPU parity of whole serving steps (epara_register_model / submit / step / collect) against the
+fp64 oracle, request by request, on the synthetic configurations."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import epara_oracle as O
+from paper_2511_00603_b200 import synth
+from tests.parity import assert_close, check_argmax, to_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module")
+def mods():
+    from paper_2511_00603_b200 import build
+    build.build()
+    from paper_2511_00603_b200 import epara, server
+    return epara, server
+
+
+def _finish(srv, E, tickets):
+    torch.cuda.synchronize()
+    res = []
+    for t in tickets:
+        s, logits, am = srv.collect(t)
+        assert s == E.OK, E.lib.epara_strerror(s)
+        res.append((logits, int(am.item())))
+    return res
+
+
+@pytest.mark.parametrize("impl", ["simt", "tcgen05"])
+def test_config1_two_mlps_one_step(mods, impl):
+    """MLP-A 512->512->512->512->10 batch 8 (latency-sensitive) and MLP-B 256->1024->256 batch 32
+    (frequency-sensitive) in ONE step, seed 0."""
+    E, server = mods
+    srv = server.Server(workspace_bytes=64 << 20, gemm_impl=E.GEMM_SIMT if impl == "simt" else E.GEMM_TCGEN05)
+    pa = synth.make_mlp([512, 512, 512, 512, 10], seed=0, device=DEV)
+    pb = synth.make_mlp([256, 1024, 256], seed=1, device=DEV)
+    xa = synth.make_mlp_inputs(8, 512, seed=2, device=DEV)
+    xb = synth.make_mlp_inputs(32, 256, seed=3, device=DEV)
+    ma, mb = srv.add_model(pa), srv.add_model(pb)
+    ta = [srv.submit(ma, E.CAT_LS, x=xa[i]) for i in range(4)]
+    ta += [srv.submit(ma, E.CAT_FS, x=xa[i]) for i in range(4, 8)]   # one group may mix both categories
+    tb = [srv.submit(mb, E.CAT_FS, x=xb[i]) for i in range(32)]
+    info = srv.step()
+    assert info.admitted[0] == 4 and info.admitted[1] == 36 and info.gemm_groups == 6
+    ra, rb = _finish(srv, E, ta), _finish(srv, E, tb)
+    va, vb = synth.bits_view(pa), synth.bits_view(pb)
+    for i, (logits, am) in enumerate(ra):
+        ref, ram = O.mlp_forward(synth.to_bits(xa[i]), va["W"], va["b"])
+        assert_close(logits, ref, what=f"MLP-A req {i}")
+        check_argmax(am, logits, ref)
+    for i, (logits, am) in enumerate(rb):
+        ref, ram = O.mlp_forward(synth.to_bits(xb[i]), vb["W"], vb["b"])
+        assert_close(logits, ref, what=f"MLP-B req {i}")
+        check_argmax(am, logits, ref)
+    srv.close()
+
+
+def test_mlp_with_biases_and_batch_invariance(mods):
+    E, server = mods
+    srv = server.Server(workspace_bytes=64 << 20)
+    p = synth.make_mlp([256, 384, 72], seed=4, device=DEV, perturb=0.3, std=0.1)
+    x = synth.make_mlp_inputs(9, 256, seed=5, device=DEV)
+    m = srv.add_model(p)
+    t_alone = [srv.submit(m, E.CAT_LS, x=x[3])]
+    srv.step()
+    alone = _finish(srv, E, t_alone)[0]
+    ts = [srv.submit(m, E.CAT_FS, x=x[i]) for i in range(9)]
+    srv.step()
+    res = _finish(srv, E, ts)
+    v = synth.bits_view(p)
+    for i, (logits, am) in enumerate(res):
+        ref, _ = O.mlp_forward(synth.to_bits(x[i]), v["W"], v["b"])
+        assert_close(logits, ref, what=f"req {i}")
+    assert torch.equal(alone[0], res[3][0]) and alone[1] == res[3][1]   # bit-identical alone vs in a batch
+    srv.close()
+
+
+def _vit_check(srv, E, p, imgs, mid, cat):
+    ts = [srv.submit(mid, cat, x=imgs[i]) for i in range(imgs.shape[0])]
+    srv.step()
+    res = _finish(srv, E, ts)
+    v = synth.bits_view(p)
+    errs = []
+    for i, (logits, am) in enumerate(res):
+        ref, ram, _ = O.vit_forward(synth.to_bits(imgs[i]), v)
+        errs.append(assert_close(logits, ref, what=f"ViT image {i}"))
+        check_argmax(am, logits, ref)
+    return res, errs
+
+
+@pytest.mark.parametrize("impl", ["simt", "tcgen05"])
+def test_small_vit_with_biases(mods, impl):
+    E, server = mods
+    srv = server.Server(workspace_bytes=256 << 20, gemm_impl=E.GEMM_SIMT if impl == "simt" else E.GEMM_TCGEN05)
+    p = synth.make_vit(d=128, n_layers=2, n_heads=2, mlp=256, n_cls=10, seed=6, device=DEV, img=64, std=0.1, perturb=0.2)
+    imgs = synth.make_images(3, seed=7, device=DEV, img=64)
+    m = srv.add_model(p, max_batch=8)
+    _vit_check(srv, E, p, imgs, m, E.CAT_FS)
+    srv.close()
+
+
+def test_config2_vit_b16_batch_2(mods):
+    """ViT-B/16 shape (197 tokens, d 768, 12 layers, 12 heads, MLP 3072, 1000 classes)."""
+    E, server = mods
+    srv = server.Server(workspace_bytes=1 << 30)
+    p = synth.make_vit(d=768, n_layers=12, n_heads=12, mlp=3072, n_cls=1000, seed=1, device=DEV)
+    imgs = synth.make_images(2, seed=11, device=DEV)
+    m = srv.add_model(p, max_batch=8)
+    res, _ = _vit_check(srv, E, p, imgs, m, E.CAT_FS)
+    # batch invariance: image 1 alone reproduces its in-batch bits
+    t = [srv.submit(m, E.CAT_LS, x=imgs[1])]
+    srv.step()
+    alone = _finish(srv, E, t)[0]
+    assert torch.equal(alone[0], res[1][0])
+    srv.close()
+
+
+def _decoder_case(E, server, p, B, lo, hi, seed, impl=None, n_check=None):
+    toks, lens, tables, npages = synth.make_decode_batch(B, lo, hi, p["vocab"], seed=seed)
+    pool = synth.make_kv_pool(p["n_layers"], npages, p["n_kv_heads"], p["head_dim"], seed=seed + 1, device=DEV)
+    pool_before = synth.to_bits(pool)
+    srv = server.Server(workspace_bytes=1 << 30, gemm_impl=impl if impl is not None else E.GEMM_TCGEN05)
+    m = srv.add_model(p, kv_pool=pool, max_kv_len=hi, max_batch=max(B, 4))
+    tabs = [torch.as_tensor(t, device=DEV) for t in tables]
+    ts = [srv.submit(m, E.CAT_FS, token=int(toks[i]), kv_len=int(lens[i]), table=tabs[i]) for i in range(B)]
+    info = srv.step()
+    res = _finish(srv, E, ts)
+    v = synth.bits_view({k: p[k] for k in p if k != "packed_layers"})
+    pool_after = synth.to_bits(pool)
+    touched = np.zeros(pool_before.shape[:2] + (pool_before.shape[4],), dtype=bool)   # [layer, page, slot]
+    decided = 0
+    for i in (range(B) if n_check is None else range(n_check)):
+        r = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], lambda l, pg: pool_before[l, pg], v)
+        assert_close(res[i][0], r["logits"], what=f"decoder req {i} (L={lens[i]})")
+        decided += check_argmax(res[i][1], res[i][0], r["logits"])
+        for l, ap in enumerate(r["appended"]):
+            # the new k, v land in exactly the (page, slot) the block table names
+            got_k = O.bf16_to_f64(pool_after[l, ap["page"], 0, :, ap["slot"], :])
+            got_v = O.bf16_to_f64(pool_after[l, ap["page"], 1, :, ap["slot"], :])
+            assert_close(got_k, ap["k"], what=f"appended k req {i} layer {l}")
+            assert_close(got_v, ap["v"], what=f"appended v req {i} layer {l}")
+    for i in range(B):
+        touched[:, int(tables[i][lens[i] // 16]), int(lens[i]) % 16] = True
+    same = (pool_before == pool_after).all(axis=(2, 3, 5))          # [layer, page, slot]
+    assert same[~touched].all(), "a cache slot other than the appended ones changed"
+    srv.close()
+    return info, decided
+
+
+@pytest.mark.parametrize("impl", ["simt", "tcgen05"])
+def test_small_decoder_step(mods, impl):
+    E, server = mods
+    p = synth.make_decoder(d=256, n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=512, vocab=1000, seed=8,
+                           device=DEV, std=0.05, perturb=0.2)
+    _decoder_case(E, server, p, B=6, lo=0, hi=600, seed=9, impl=E.GEMM_SIMT if impl == "simt" else E.GEMM_TCGEN05)
+
+
+def test_config3_decoder_1b_batch_4(mods):
+    """Llama-style decoder d 2048, 16 layers, 32/8 heads (hd 64), FFN 8192, vocab 32000, KV lengths
+    U[128, 4096], 16-token pages, permuted block tables."""
+    E, server = mods
+    p = synth.make_decoder(d=2048, n_layers=16, n_q_heads=32, n_kv_heads=8, head_dim=64, ffn=8192, vocab=32000,
+                           seed=2, device=DEV)
+    info, decided = _decoder_case(E, server, p, B=4, lo=128, hi=4096, seed=21, n_check=2)
+    assert info.weight_bytes == pytest.approx(2 * (16 * (3072 * 2048 + 2048 * 2048 + 16384 * 2048 + 2048 * 8192)
+                                                   + 32000 * 2048))
+
+
+def test_decoder_batch_invariance_and_mixed_models(mods):
+    """One step holding an MLP, a ViT and a decoder: every request equals the oracle, and the decoder
+    request's bits do not depend on the co-resident models (MT)."""
+    E, server = mods
+    pd = synth.make_decoder(d=256, n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=512, vocab=500, seed=30,
+                            device=DEV, std=0.05)
+    pm = synth.make_mlp([128, 256, 16], seed=31, device=DEV, std=0.1)
+    pv = synth.make_vit(d=128, n_layers=1, n_heads=2, mlp=256, n_cls=10, seed=32, device=DEV, img=32, std=0.1)
+    toks, lens, tables, npages = synth.make_decode_batch(3, 10, 300, 500, seed=33)
+    pool = synth.make_kv_pool(2, npages, 2, 64, seed=34, device=DEV)
+    pool0 = pool.clone()
+    srv = server.Server(workspace_bytes=512 << 20)
+    md = srv.add_model(pd, kv_pool=pool, max_kv_len=300, max_batch=8)
+    mm = srv.add_model(pm, max_batch=8)
+    mv = srv.add_model(pv, max_batch=4)
+    tabs = [torch.as_tensor(t, device=DEV) for t in tables]
+    xs = synth.make_mlp_inputs(2, 128, seed=35, device=DEV)
+    imgs = synth.make_images(2, seed=36, device=DEV, img=32)
+    t_d = [srv.submit(md, E.CAT_FS, token=int(toks[i]), kv_len=int(lens[i]), table=tabs[i]) for i in range(3)]
+    t_m = [srv.submit(mm, E.CAT_LS, x=xs[i]) for i in range(2)]
+    t_v = [srv.submit(mv, E.CAT_FS, x=imgs[i]) for i in range(2)]
+    srv.step()
+    r_d, r_m, r_v = _finish(srv, E, t_d), _finish(srv, E, t_m), _finish(srv, E, t_v)
+    pb = synth.to_bits(pool0)
+    vd = synth.bits_view({k: pd[k] for k in pd if k != "packed_layers"})
+    for i in range(3):
+        r = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], lambda l, pg: pb[l, pg], vd)
+        assert_close(r_d[i][0], r["logits"], what=f"decoder {i}")
+    vm, vv = synth.bits_view(pm), synth.bits_view(pv)
+    for i in range(2):
+        assert_close(r_m[i][0], O.mlp_forward(synth.to_bits(xs[i]), vm["W"], vm["b"])[0], what=f"mlp {i}")
+        assert_close(r_v[i][0], O.vit_forward(synth.to_bits(imgs[i]), vv)[0], what=f"vit {i}")
+    # request 1 of the decoder alone, on a fresh copy of the cache
+    pool.copy_(pool0)
+    t = [srv.submit(md, E.CAT_LS, token=int(toks[1]), kv_len=int(lens[1]), table=tabs[1])]
+    srv.step()
+    alone = _finish(srv, E, t)[0]
+    assert torch.equal(alone[0], r_d[1][0]) and alone[1] == r_d[1][1]
+    srv.close()
+
+
+def test_request_handler_answers(mods):
+    """Timeout of an expired request, rejection of the >1 GPU categories, caps, pending tickets."""
+    E, server = mods
+    srv = server.Server(workspace_bytes=64 << 20, cap_ls=2, cap_fs=3)
+    p = synth.make_mlp([64, 64, 8], seed=40, device=DEV, std=0.1)
+    x = synth.make_mlp_inputs(8, 64, seed=41, device=DEV)
+    m = srv.add_model(p)
+    inp = E.Inputs()
+    inp.input = x[0].data_ptr()
+    out = torch.empty(8, dtype=torch.bfloat16, device=DEV)
+    inp.out_logits = out.data_ptr()
+    assert srv.ctx.epara_submit(m, E.CAT_LS_GT1, inp, raise_on_error=False)[0] == E.E_UNSUPPORTED
+    assert srv.ctx.epara_submit(m, E.CAT_FS_GT1, inp, raise_on_error=False)[0] == E.E_UNSUPPORTED
+    assert srv.ctx.epara_submit(m + 5, E.CAT_LS, inp, raise_on_error=False)[0] == E.E_INVALID
+    assert srv.ctx.epara_submit(m, 7, inp, raise_on_error=False)[0] == E.E_INVALID
+    late = srv.submit(m, E.CAT_LS, x=x[0], deadline_ns=1000)
+    live = [srv.submit(m, E.CAT_LS, x=x[i], deadline_ns=5000) for i in range(1, 4)]
+    fs = [srv.submit(m, E.CAT_FS, x=x[i]) for i in range(4, 8)]
+    assert srv.collect(live[0])[0] == E.PENDING            # still queued
+    info = srv.step(now_ns=2000)
+    assert list(info.dropped) == [1, 0] and list(info.admitted) == [2, 3]
+    torch.cuda.synchronize()
+    assert srv.collect(late)[0] == E.E_TIMEOUT
+    assert srv.collect(live[0])[0] == E.OK and srv.collect(live[1])[0] == E.OK
+    assert srv.collect(live[2])[0] == E.PENDING            # beyond the LS cap: waits for the next step
+    assert srv.collect(fs[3])[0] == E.PENDING
+    info = srv.step(now_ns=6000)                           # live[2] expired meanwhile
+    assert list(info.dropped) == [1, 0] and list(info.admitted) == [0, 1]
+    torch.cuda.synchronize()
+    assert srv.collect(live[2])[0] == E.E_TIMEOUT
+    s, logits, am = srv.collect(fs[3])
+    assert s == E.OK
+    v = synth.bits_view(p)
+    assert_close(logits, O.mlp_forward(synth.to_bits(x[7]), v["W"], v["b"])[0], what="late FS request")
+    assert srv.ctx.epara_collect(fs[3])[0] == E.E_INVALID  # already collected
+    srv.close()
+
+
+def test_workspace_too_small_is_resource_insufficiency(mods):
+    E, server = mods
+    srv = server.Server(workspace_bytes=20 << 20)
+    p = synth.make_vit(d=768, n_layers=1, n_heads=12, mlp=3072, n_cls=10, seed=50, device=DEV)
+    with pytest.raises(E.EparaError) as ei:
+        srv.add_model(p, max_batch=64)
+    assert ei.value.status == E.E_RESOURCE
+    srv.close()
