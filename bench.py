@@ -1,0 +1,430 @@
+"""Benchmark of the categorized serving step.
+
+  python bench.py --gpus N --steps K --warmup W            this library on N GPUs (N > 1: under torchrun)
+  python bench.py --impl reference ...                      the CPU oracle on the host cores
+
+A step is one epara_step over one full batch of every co-resident instance of the mixed
+workload (3 MLP-A, 3 ViT-S/16, 2 1B decoders; per family one latency-sensitive instance with
+batch 4 and frequency-sensitive ones with batch 256): every kernel kind of the path runs in
+every step.  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mixed-category requests/s"
+UNIT = "requests/s"
+WORKLOAD = ("mixed co-resident step (configs[3], saturated): 3x MLP-A, 3x ViT-S/16, 2x 1B decoder; per family "
+            "instance 0 latency-sensitive batch 4, others frequency-sensitive batch 256; decoder KV ~U[128,4096]")
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------ CPU oracle leg
+class OracleSampler:
+    """Times the oracle, as it stands, on a bounded sample of the mixed workload: 8 MLP-A requests,
+    1 ViT-S image, 1 decoder request (1B shape, KV length 2112 = the mean of U[128,4096]).  The models
+    are generated once; every sample() draws fresh inputs and returns seconds per request per family."""
+
+    def __init__(self, seed: int = 3):
+        from paper_2511_00603_b200 import synth, workloads as W
+        self.synth, self.seed = synth, seed
+        self.cores = os.cpu_count() or 1
+        self.mlp = synth.bits_view(synth.make_mlp(W.MLP_A, seed=seed))
+        self.vit = synth.bits_view(synth.make_vit(seed=seed + 2, **W.VIT_S))
+        self.dec = synth.bits_view(synth.make_decoder(seed=seed + 4, **W.DEC_1B))
+        self.n = 0
+
+    def sample(self):
+        from oracle import epara_oracle as O
+        synth, s = self.synth, self.seed + 100 * self.n
+        self.n += 1
+        t = {}
+        x = synth.make_mlp_inputs(8, 512, seed=s + 1)
+        t0 = time.perf_counter()
+        for i in range(8):
+            O.mlp_forward(synth.to_bits(x[i]), self.mlp["W"], self.mlp["b"])
+        t["mlp"] = (time.perf_counter() - t0) / 8
+        img = synth.to_bits(synth.make_images(1, seed=s + 3)[0])
+        t0 = time.perf_counter()
+        O.vit_forward(img, self.vit)
+        t["vit"] = time.perf_counter() - t0
+        toks, lens, tables, npages = synth.make_decode_batch(1, 2112, 2112, 32000, seed=s + 5)
+        pool = synth.to_bits(synth.make_kv_pool(16, npages, 8, 64, seed=s + 6))
+        t0 = time.perf_counter()
+        O.decoder_step(int(toks[0]), int(lens[0]), tables[0], lambda l, pg: pool[l, pg], self.dec)
+        t["decoder"] = time.perf_counter() - t0
+        return t
+
+
+def mixed_counts(ls=4, fs=256):
+    return {"mlp": ls + 2 * fs, "vit": ls + 2 * fs, "decoder": ls + fs}
+
+
+def oracle_rps(t, counts):
+    step_s = sum(counts[k] * t[k] for k in counts)
+    return sum(counts.values()) / step_s, step_s
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    counts = mixed_counts()
+    vals = []
+    smp = OracleSampler()
+    cores = smp.cores
+    for i in range(args.warmup + args.steps):
+        t = smp.sample()
+        if i >= args.warmup:
+            vals.append(oracle_rps(t, counts))
+    rps = sum(v[0] for v in vals) / len(vals)
+    step_s = sum(v[1] for v in vals) / len(vals)
+    sample = ("per step: 8 MLP-A + 1 ViT-S image + 1 decoder request (1B, KV 2112) timed, step time extrapolated "
+              "to the 1292-request mixed step by per-family counts")
+    line = {"impl": "reference", "metric": METRIC, "value": rps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD},
+            "cpu_baseline": {"value": rps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": rps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------ GPU leg
+def poisson_phase(srv, insts, E, W, torch, horizon_s=1.0, warm_s=0.1, seed=3):
+    """Closed-loop replay of seeded Poisson arrivals (virtual clock advanced by measured step time)."""
+    import ctypes as C
+    import numpy as np
+    from paper_2511_00603_b200 import synth
+    fam_idx = {"mlp": 0, "vit": 0, "decoder": 0}
+    arr = []
+    for k, inst in enumerate(insts):
+        rate = W.MIXED_RATES[inst.kind][fam_idx[inst.kind]]
+        fam_idx[inst.kind] += 1
+        arr.append((rate, synth.poisson_arrivals(rate, horizon_s + warm_s, seed * 10 + k)))
+    ptr = [0] * len(insts)
+    nsub = [0] * len(insts)
+    live = {}          # ticket -> (inst index, arrival, deadline)
+    ls_step_ms, ls_lat_ms, done_ls, done_fs, late_ls, dropped = [], [], 0, [0] * len(insts), 0, 0
+    now = 0
+    horizon_ns = int((horizon_s + warm_s) * 1e9)
+    warm_ns = int(warm_s * 1e9)
+    stream = torch.cuda.current_stream(srv.device)
+    inp = E.Inputs()
+    steps = 0
+    while now < horizon_ns:
+        any_q = bool(live)
+        for k, inst in enumerate(insts):
+            a = arr[k][1]
+            while ptr[k] < len(a) and a[ptr[k]] <= now:
+                t_arr = int(a[ptr[k]])
+                dl = t_arr + W.LS_DEADLINE_NS if inst.category == E.CAT_LS else 0
+                inst.fill(inp, nsub[k] % inst.n_req, nsub[k] % inst.n_req, deadline_ns=dl, arrival_ns=t_arr, stream=k)
+                tk = srv.ctx.epara_submit(inst.mid, inst.category, inp)
+                live[tk] = (k, t_arr, dl)
+                ptr[k] += 1
+                nsub[k] += 1
+                any_q = True
+        if not any_q:
+            nxt = min((arr[k][1][ptr[k]] for k in range(len(insts)) if ptr[k] < len(arr[k][1])), default=horizon_ns)
+            now = max(now + 1, int(nxt))
+            continue
+        t0 = time.perf_counter()
+        info = srv.ctx.epara_step(stream.cuda_stream, now)
+        stream.synchronize()
+        dt_ns = int((time.perf_counter() - t0) * 1e9)
+        steps += 1
+        end = now + dt_ns
+        had_ls = info.admitted[0] > 0
+        for tk in list(live.keys()):
+            s, _ = srv.ctx.epara_collect(tk)
+            if s == E.PENDING:
+                continue
+            k, t_arr, dl = live.pop(tk)
+            if t_arr < warm_ns:
+                continue
+            if s == E.E_TIMEOUT:
+                dropped += 1
+            elif insts[k].category == E.CAT_LS:
+                ls_lat_ms.append((end - t_arr) / 1e6)
+                if end <= dl:
+                    done_ls += 1
+                else:
+                    late_ls += 1
+            else:
+                done_fs[k] += 1
+        if had_ls and now >= warm_ns:
+            ls_step_ms.append(dt_ns / 1e6)
+        now = end
+    span = horizon_s
+    fs_credit = 0.0
+    for k, inst in enumerate(insts):
+        if inst.category == E.CAT_FS:
+            achieved = done_fs[k] / span
+            fs_credit += done_fs[k] * min(1.0, achieved / arr[k][0])     # frames x achieved / required rate
+    q = lambda v, p: (sorted(v)[min(len(v) - 1, int(p * len(v)))] if v else None)
+    return {"horizon_s": horizon_s, "steps": steps, "goodput_rps": (done_ls + fs_credit) / span,
+            "ls_in_deadline": done_ls, "ls_late": late_ls, "dropped": dropped,
+            "ls_step_ms_p50": q(ls_step_ms, 0.5), "ls_step_ms_p99": q(ls_step_ms, 0.99),
+            "ls_latency_ms_p50": q(ls_lat_ms, 0.5), "ls_latency_ms_p99": q(ls_lat_ms, 0.99)}
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2511_00603_b200 import build
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2511_00603_b200 import epara as E, server, workloads as W
+    peaks = read_peaks()
+    dev = torch.device("cuda", local)
+    srv = server.Server(device=local, workspace_bytes=3 << 30)
+    insts = W.build_mixed(srv, seed=3)
+    n_req = sum(i.n_req for i in insts)
+    stream = torch.cuda.current_stream(dev)
+
+    outstanding = []
+
+    def one_step():
+        for i in insts:
+            i.submit_all(srv.ctx)
+            outstanding.append(list(i.tickets))
+        return srv.ctx.epara_step(stream.cuda_stream, 0)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def drain():
+        for tks in outstanding:
+            for t in tks:
+                st, _ = srv.ctx.epara_collect(t)
+                if st != E.OK:
+                    raise RuntimeError(f"request {t}: {E.lib.epara_strerror(st).decode()}")
+        outstanding.clear()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+        torch.cuda.synchronize()
+        drain()
+
+    # ---- timed region: K steps, device-timed, per-launch events on (profile) ----
+    srv.ctx.epara_set_profile(True)
+    kinds = {k: [0.0, 0] for k in E.K_NAMES}
+    launches = 0
+    flops = wbytes = kvbytes = 0.0
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    infos = []
+    for _ in range(args.steps):
+        infos.append(one_step())
+    ev1.record(stream)
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    drain()
+    for info in infos:
+        launches += info.launches
+        flops += info.gemm_flops
+        wbytes += info.weight_bytes
+        kvbytes += info.kv_bytes
+    # per-kind device time of the last timed step (every step launches the same kernels)
+    prof = srv.ctx.epara_step_profile()
+    srv.ctx.epara_set_profile(False)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * n_req * args.steps / (ms_total / 1e3)
+
+    # ---- unprofiled repeat (shows what the event bracketing costs) ----
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        one_step()
+    ev1.record(stream)
+    barrier()
+    ms_plain = ev0.elapsed_time(ev1) / args.steps
+    drain()
+
+    # ---- end to end: pinned host inputs -> device, step, results -> pinned host, every step ----
+    h_in = [(i, i.x.cpu().pin_memory()) for i in insts if i.x is not None]
+    h_out = [(i, torch.empty_like(i.logits, device="cpu").pin_memory(), torch.empty_like(i.argmax, device="cpu").pin_memory())
+             for i in insts]
+    h2d = sum(x.numel() * x.element_size() for _, x in h_in)
+    d2h = sum(l.numel() * 2 + a.numel() * 4 for _, l, a in h_out)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        for i, hx in h_in:
+            i.x.copy_(hx, non_blocking=True)
+        one_step()
+        for i, hl, ha in h_out:
+            hl.copy_(i.logits, non_blocking=True)
+            ha.copy_(i.argmax, non_blocking=True)
+        stream.synchronize()
+    e2e_s = time.perf_counter() - t0
+    drain()
+    if world > 1:
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * n_req * args.steps / e2e_s
+
+    if rank != 0:
+        srv.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel ----
+    dom = max(prof, key=lambda k: prof[k][0])
+    per_step = lambda v: v / args.steps
+    if dom == "gemm":
+        ach = per_step(flops) / (prof["gemm"][0] / 1e3) / 1e12
+        roof = {"kernel": "gemm_tc_kernel (all GEMM launches of a step)", "bound": "tensor", "achieved": ach,
+                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
+                "traffic": None, "peak_source": peaks["source"] + " (sustained)"}
+    elif dom == "attn_dec":
+        ach = per_step(kvbytes) / (prof["attn_dec"][0] / 1e3) / 1e9
+        roof = {"kernel": "attn_decode_kernel (all launches of a step)", "bound": "hbm", "achieved": ach,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                "peak_source": peaks["source"]}
+    else:
+        roof = {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": None, "traffic": None, "peak_source": peaks["source"]}
+    kernels = {k: {"ms_per_step": prof[k][0], "launches_per_step": prof[k][1]} for k in prof if prof[k][1]}
+    if prof["gemm"][1]:
+        kernels["gemm"]["tflops"] = per_step(flops) / (prof["gemm"][0] / 1e3) / 1e12
+        kernels["gemm"]["weight_gbs"] = per_step(wbytes) / (prof["gemm"][0] / 1e3) / 1e9
+    if prof["attn_dec"][1]:
+        kernels["attn_dec"]["kv_gbs"] = per_step(kvbytes) / (prof["attn_dec"][0] / 1e3) / 1e9
+
+    poisson = None
+    if not args.no_poisson:
+        poisson = poisson_phase(srv, insts, E, W, torch)
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        smp = OracleSampler()
+        t, cores = smp.sample(), smp.cores
+        rps, step_s = oracle_rps(t, mixed_counts())
+        cpu = {"value": rps, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "8 MLP-A + 1 ViT-S image + 1 decoder request (1B, KV 2112) timed once each; step time "
+                         "extrapolated to the 1292-request mixed step by per-family counts",
+               "seconds_per_request": t}
+    srv.close()
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "requests_per_step": n_req, "l2": "inputs larger than L2 (17 GB of KV and 4.6 GB of weights per step)",
+                       "parallelism": f"replicas x{world}, no collective"},
+            "clocks": clocks, "gpu_launches": launches,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "ms_per_step_unprofiled": ms_plain,
+            "ls_latency": poisson}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="epara", choices=["epara", "reference"])
+    ap.add_argument("--no-poisson", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -158,6 +158,12 @@ int epara_register_model(epara_ctx*, const epara_model_desc* m, int* model_id);
  * INVALID for bad ids/pointers/lengths, RESOURCE when the queue is full. */
 int epara_submit(epara_ctx*, int model_id, int category, const epara_inputs* in, uint64_t* ticket);
 
+/* n requests of one (model, category) in one call, in order; same checks as epara_submit.  Stops at
+ * the first rejected request: *n_accepted (may be NULL) counts those queued, tickets[i] is filled
+ * for each of them, and the status of the rejected one is returned. */
+int epara_submit_many(epara_ctx*, int model_id, int category, const epara_inputs* in, int n, uint64_t* tickets,
+                      int* n_accepted);
+
 /* Runs one step on `cuda_stream` (a cudaStream_t), asynchronously:
  *  - drops requests whose deadline_ns < now_ns (Section 3.2, first handler rule);
  *  - per model admits the oldest <= cap_ls latency-sensitive requests, then frequency-
@@ -176,6 +182,9 @@ int epara_collect(epara_ctx*, uint64_t ticket, epara_output* out);
 /* With cfg.profile = 1: per kernel kind, total milliseconds and launch count of the most
  * recent finished step (arrays of EPARA_K_COUNT).  Synchronises that step.  */
 int epara_step_profile(epara_ctx*, float* ms_per_kind, int* launches_per_kind);
+
+/* Switches the per-launch event bracketing of epara_config.profile on (1) or off (0). */
+int epara_set_profile(epara_ctx*, int on);
 
 int epara_destroy(epara_ctx*);
 const char* epara_strerror(int status);

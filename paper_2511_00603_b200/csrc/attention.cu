@@ -104,6 +104,10 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __
     for (int i = 0; i < NL; ++i) {
       float vf[8];
       unpack8(vr[i], vf);
+      if ((pg * 16 + i * TPW + ts) >= t_end) {   // slots past the length may hold anything, NaN included
+#pragma unroll
+        for (int e = 0; e < 8; ++e) vf[e] = 0.f;
+      }
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         l[h] += s[i][h];
@@ -302,12 +306,8 @@ cudaError_t launch_attn_encoder(const AttnEncGroup* groups, int n_groups, int to
   if (n_groups == 0 || total_blocks == 0) return cudaSuccess;
   const size_t smem = (size_t)max_T * 64 * 2 * sizeof(bf16);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attn_encoder_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  cudaError_t e = cudaFuncSetAttribute(attn_encoder_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
   attn_encoder_kernel<64><<<total_blocks, ENC_QB, smem, st>>>(groups, n_groups);
   return cudaGetLastError();
 }

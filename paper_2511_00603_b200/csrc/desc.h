@@ -119,3 +119,12 @@ struct OutputGroup {     // copy logits rows to the requests' buffers and take t
 };
 
 }  // namespace epara
+
+// Group arrays are packed back to back in the step blob: sizes must keep 8-byte alignment.
+namespace epara {
+static_assert(sizeof(GemmGroup) % 64 == 0, "GemmGroup holds 64-byte aligned TMA maps");
+static_assert(sizeof(NormGroup) % 8 == 0 && sizeof(GatherGroup) % 8 == 0 && sizeof(RopeGroup) % 8 == 0 &&
+              sizeof(AttnDecGroup) % 8 == 0 && sizeof(AttnEncGroup) % 8 == 0 && sizeof(AssembleGroup) % 8 == 0 &&
+              sizeof(OutputGroup) % 8 == 0 && sizeof(ReqDesc) % 16 == 0 && sizeof(AttnReq) % 16 == 0,
+              "descriptor sizes");
+}  // namespace epara

@@ -112,6 +112,7 @@ struct Slot {
   cudaEvent_t done;
   uint64_t step_id;     // 0 = never used
   bool busy;
+  bool profiled;        // the step in this slot was bracketed with events
   std::vector<cudaEvent_t> prof;   // 2 per launch when profiling
   std::vector<int> prof_kind;
 };
@@ -501,6 +502,7 @@ int epara_init(const epara_config* cfg, epara_ctx** out) {
     s.dev = (unsigned char*)carve(c, BLOB_BYTES);
     s.step_id = 0;
     s.busy = false;
+    s.profiled = false;
     if (cudaMallocHost((void**)&s.host, BLOB_BYTES) != cudaSuccess ||
         cudaMallocHost((void**)&s.status_host, 64) != cudaSuccess ||
         cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) != cudaSuccess) {
@@ -580,6 +582,18 @@ int epara_submit(epara_ctx* c, int model_id, int category, const epara_inputs* i
   t.state = T_QUEUED; t.model = model_id; t.step = 0; t.out_logits = in->out_logits; t.out_argmax = in->out_argmax;
   c->tickets[r.ticket] = t;
   *ticket = r.ticket;
+  return EPARA_OK;
+}
+
+int epara_submit_many(epara_ctx* c, int model_id, int category, const epara_inputs* in, int n, uint64_t* tickets,
+                      int* n_accepted) {
+  if (n_accepted) *n_accepted = 0;
+  if (!c || n < 0 || (n > 0 && (!in || !tickets))) return EPARA_E_INVALID;
+  for (int i = 0; i < n; ++i) {
+    const int r = epara_submit(c, model_id, category, in + i, tickets + i);
+    if (r != EPARA_OK) return r;
+    if (n_accepted) *n_accepted = i + 1;
+  }
   return EPARA_OK;
 }
 
@@ -685,7 +699,6 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       if (kind == EPARA_K_ATTN_DEC) {
         // decode attention is templated on (hd, G): one launch per distinct pair
         std::vector<Active*> rest = who;
-        bool first = true;
         while (!rest.empty()) {
           const Op& o0 = rest[0]->m->ops[rest[0]->cursor];
           const int hd = o0.adec.hd, G = o0.adec.Hq / o0.adec.Hkv;
@@ -707,7 +720,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
             max_hkv = std::max(max_hkv, g.Hkv); max_hq = std::max(max_hq, g.Hq);
             for (int b = 0; b < a->B; ++b)
               max_chunks = std::max(max_chunks, (a->reqs[b].in.kv_len + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK);
-            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
           }
           LL.p0 = total_B; LL.p1 = max_hkv; LL.p2 = max_chunks; LL.p3 = (hd << 8) | G;
           launches.push_back(LL);
@@ -715,7 +728,6 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           LC.kind = EPARA_K_ATTN_COMBINE; LC.p1 = max_hq;
           launches.push_back(LC);
           rest.swap(other);
-          (void)first;
         }
         for (Active* a : who) a->cursor++;
         continue;
@@ -729,21 +741,21 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
             GatherGroup g = op.gather;
             g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B; g.blocks = rows;
             mx = std::max(mx, rows);
-            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_ASSEMBLE: {
             AssembleGroup g = op.asmb;
             g.B = a->B;
             mx = std::max(mx, rows);
-            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_NORM: {
             NormGroup g = op.norm;
             g.M = rows;
             mx = std::max(mx, rows);
-            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_GEMM: {
@@ -763,7 +775,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
             RopeGroup g = op.rope;
             g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
             mx = std::max(mx, a->B);
-            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_ATTN_ENC: {
@@ -771,14 +783,14 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
             g.B = a->B; g.q_blocks = attn_encoder_q_blocks(g.T); g.blk_start = total;
             total += a->B * g.H * g.q_blocks;
             mx = std::max(mx, g.T);
-            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_OUTPUT: {
             OutputGroup g = op.outp;
             g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
             mx = std::max(mx, a->B);
-            if (put(&g, sizeof(g), 16) == (size_t)-1) overflow = true;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
         }
@@ -799,6 +811,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
   // ---- upload + launch ----
   if (cudaMemcpyAsync(slot.dev, slot.host, off, cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
   const bool prof = c->cfg.profile != 0;
+  slot.profiled = prof;
   if (prof) {
     if (launches.size() > MAX_PROFILE_LAUNCHES) return EPARA_E_RESOURCE;
     while (slot.prof.size() < 2 * launches.size()) {
@@ -876,11 +889,16 @@ int epara_collect(epara_ctx* c, uint64_t ticket, epara_output* out) {
   return result;
 }
 
+int epara_set_profile(epara_ctx* c, int on) {
+  if (!c) return EPARA_E_INVALID;
+  c->cfg.profile = on ? 1 : 0;
+  return EPARA_OK;
+}
+
 int epara_step_profile(epara_ctx* c, float* ms_per_kind, int* launches_per_kind) {
   if (!c || !ms_per_kind || !launches_per_kind) return EPARA_E_INVALID;
-  if (!c->cfg.profile) return EPARA_E_UNSUPPORTED;
   Slot& s = c->slots[c->last_step_slot];
-  if (s.step_id == 0) return EPARA_E_INVALID;
+  if (s.step_id == 0 || !s.profiled) return EPARA_E_UNSUPPORTED;
   if (cudaEventSynchronize(s.done) != cudaSuccess) return EPARA_E_CUDA;
   for (int k = 0; k < EPARA_K_COUNT; ++k) { ms_per_kind[k] = 0.f; launches_per_kind[k] = 0; }
   for (size_t i = 0; i < s.prof_kind.size(); ++i) {

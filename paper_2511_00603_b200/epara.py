@@ -64,17 +64,20 @@ class GemmProblem(C.Structure):
                 ("ldc", C.c_int), ("epilogue", C.c_int)]
 
 
-EXPORTS = ["epara_init", "epara_register_model", "epara_submit", "epara_step", "epara_collect",
-           "epara_step_profile", "epara_destroy", "epara_strerror", "epara_model_workspace_bytes",
+EXPORTS = ["epara_init", "epara_register_model", "epara_submit", "epara_submit_many", "epara_step", "epara_collect",
+           "epara_step_profile", "epara_set_profile", "epara_destroy", "epara_strerror", "epara_model_workspace_bytes",
            "epara_dp_group_count", "epara_inter_request_count", "epara_admit_queue", "epara_grouped_gemm",
            "epara_gemm_scratch_bytes", "epara_decode_attention", "epara_decode_attention_scratch_bytes"]
 
 lib.epara_init.argtypes = [C.POINTER(Config), C.POINTER(C.c_void_p)]
 lib.epara_register_model.argtypes = [C.c_void_p, C.POINTER(ModelDesc), C.POINTER(C.c_int)]
 lib.epara_submit.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(Inputs), C.POINTER(C.c_uint64)]
+lib.epara_submit_many.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(Inputs), C.c_int, C.POINTER(C.c_uint64),
+                                  C.POINTER(C.c_int)]
 lib.epara_step.argtypes = [C.c_void_p, C.c_void_p, C.c_longlong, C.POINTER(StepInfo)]
 lib.epara_collect.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Output)]
 lib.epara_step_profile.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+lib.epara_set_profile.argtypes = [C.c_void_p, C.c_int]
 lib.epara_destroy.argtypes = [C.c_void_p]
 lib.epara_strerror.argtypes = [C.c_int]
 lib.epara_strerror.restype = C.c_char_p
@@ -208,6 +211,13 @@ class Context:
             return t.value
         return s, t.value
 
+    def epara_submit_many(self, model_id: int, category: int, inputs, n: int, tickets=None):
+        """inputs: a ctypes array of Inputs; returns the ctypes array of tickets."""
+        tk = tickets if tickets is not None else (C.c_uint64 * max(n, 1))()
+        acc = C.c_int(0)
+        _check(lib.epara_submit_many(self.h, model_id, category, inputs, n, tk, C.byref(acc)), "epara_submit_many")
+        return tk
+
     def epara_step(self, stream_ptr: int, now_ns: int = -1) -> StepInfo:
         info = StepInfo()
         _check(lib.epara_step(self.h, C.c_void_p(stream_ptr), now_ns, C.byref(info)), "epara_step")
@@ -217,6 +227,9 @@ class Context:
         out = Output()
         s = lib.epara_collect(self.h, ticket, C.byref(out))
         return s, out
+
+    def epara_set_profile(self, on: bool):
+        _check(lib.epara_set_profile(self.h, int(on)), "epara_set_profile")
 
     def epara_step_profile(self):
         ms = (C.c_float * K_COUNT)()

@@ -1,0 +1,114 @@
+"""The synthetic serving workloads: which models are co-resident, their categories, batches and
+inputs.  Only placement and argument marshalling happen here; every forward pass runs in the
+library's kernels.
+
+mixed step (the co-resident configuration): 8 instances -- 3x MLP-A (512->512->512->512->10),
+3x ViT-S/16 (d 384, 6 heads, 12 layers, MLP 1536, 1000 classes), 2x Llama-style 1B decoder
+(d 2048, 16 layers, 32/8 heads, hd 64, FFN 8192, vocab 32000).  Per family the first instance
+is latency-sensitive (batch <= 4, 20 ms deadline), the others frequency-sensitive (batch <= 256).
+Decoder requests have KV lengths ~U[128, 4096] in a paged cache filled N(0,1) with permuted
+block tables.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import Dict, List
+
+import numpy as np
+import torch
+
+from . import epara as E
+from . import synth
+
+MLP_A = [512, 512, 512, 512, 10]
+VIT_S = dict(d=384, n_layers=12, n_heads=6, mlp=1536, n_cls=1000)
+VIT_B = dict(d=768, n_layers=12, n_heads=12, mlp=3072, n_cls=1000)
+DEC_1B = dict(d=2048, n_layers=16, n_q_heads=32, n_kv_heads=8, head_dim=64, ffn=8192, vocab=32000)
+DEC_8B = dict(d=4096, n_layers=32, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=14336, vocab=32000)
+
+# arrival rates (requests/s) of the 8 instances, fixed table
+MIXED_RATES = {"mlp": [2000.0, 1500.0, 1000.0], "vit": [500.0, 300.0, 200.0], "decoder": [100.0, 50.0]}
+LS_DEADLINE_NS = 20_000_000
+
+
+class Instance:
+    """One placed model with a pool of ready-made requests (inputs, outputs, ctypes descriptors)."""
+
+    def __init__(self, srv, p: Dict, category: int, n_req: int, seed: int, kv_lo: int = 128, kv_hi: int = 4096,
+                 max_batch: int = 0):
+        dev = srv.device
+        self.p, self.category, self.n_req, self.kind = p, category, n_req, p["kind"]
+        self.kv_pool = None
+        self.tokens = self.lens = self.tables = None
+        if self.kind == "mlp":
+            self.x = synth.make_mlp_inputs(n_req, p["dims"][0], seed, device=dev)
+            self.n_out = p["dims"][-1]
+        elif self.kind == "vit":
+            self.x = synth.make_images(n_req, seed, device=dev, img=p["img"])
+            self.n_out = p["n_cls"]
+        else:
+            self.x = None
+            self.n_out = p["vocab"]
+            self.tokens, self.lens, self.tables, npages = synth.make_decode_batch(n_req, kv_lo, kv_hi, p["vocab"], seed)
+            self.kv_pool = synth.make_kv_pool(p["n_layers"], npages, p["n_kv_heads"], p["head_dim"], seed + 1, device=dev)
+            flat = np.concatenate(self.tables)
+            self.tables_dev = torch.as_tensor(flat, device=dev)
+            self.table_off = np.concatenate([[0], np.cumsum([len(t) for t in self.tables])])
+        self.mid = srv.add_model(p, kv_pool=self.kv_pool, max_kv_len=kv_hi, max_batch=max_batch or n_req)
+        self.logits = torch.zeros((n_req, self.n_out), dtype=torch.bfloat16, device=dev)
+        self.argmax = torch.full((n_req,), -1, dtype=torch.int32, device=dev)
+        self.inputs = (E.Inputs * n_req)()
+        self.tickets = (C.c_uint64 * n_req)()
+        for i in range(n_req):
+            self.fill(self.inputs[i], i, i)
+
+    def fill(self, inp: "E.Inputs", req: int, out_slot: int, deadline_ns: int = 0, arrival_ns: int = 0, stream: int = 0):
+        """Request `req` of the pool, writing its result to output row `out_slot`."""
+        if self.kind == "decoder":
+            inp.input = None
+            inp.token, inp.kv_len = int(self.tokens[req]), int(self.lens[req])
+            inp.block_table = self.tables_dev.data_ptr() + 4 * int(self.table_off[req])
+            inp.n_blocks = int(self.table_off[req + 1] - self.table_off[req])
+        else:
+            inp.input = self.x[req].data_ptr()
+        inp.deadline_ns, inp.arrival_ns, inp.stream = deadline_ns, arrival_ns, stream
+        inp.out_logits = self.logits[out_slot].data_ptr()
+        inp.out_argmax = self.argmax.data_ptr() + 4 * out_slot
+
+    def submit_all(self, ctx: "E.Context"):
+        ctx.epara_submit_many(self.mid, self.category, self.inputs, self.n_req, self.tickets)
+
+    def input_bytes(self) -> int:
+        return 0 if self.x is None else self.x.numel() * self.x.element_size()
+
+    def output_bytes(self) -> int:
+        return self.logits.numel() * 2 + self.argmax.numel() * 4
+
+
+def workspace_bytes_mixed(ls_batch: int, fs_batch: int) -> int:
+    # ViT-S activations dominate: ~8.5 KB per token, 197 tokens per image
+    vit = lambda b: (b * 197 + 128) * 10 * 1024
+    dec = lambda b: (b + 128) * (2048 * 6 + 3072 * 2 + 2048 * 2 + 8192 * 2 + 32000 * 2) + b * 32 * 17 * 66 * 4
+    return int(64 << 20) + vit(ls_batch) + 2 * vit(fs_batch) + dec(ls_batch) + dec(fs_batch) + (64 << 20)
+
+
+def build_mixed(srv, seed: int = 3, ls_batch: int = 4, fs_batch: int = 256, kv_lo: int = 128, kv_hi: int = 4096
+                ) -> List[Instance]:
+    """The 8 co-resident instances with one full batch of requests each."""
+    dev = srv.device
+    out: List[Instance] = []
+    k = 0
+    for i in range(3):
+        cat, n = (E.CAT_LS, ls_batch) if i == 0 else (E.CAT_FS, fs_batch)
+        out.append(Instance(srv, synth.make_mlp(MLP_A, seed=seed * 100 + k, device=dev), cat, n, seed * 1000 + k))
+        k += 1
+    for i in range(3):
+        cat, n = (E.CAT_LS, ls_batch) if i == 0 else (E.CAT_FS, fs_batch)
+        out.append(Instance(srv, synth.make_vit(seed=seed * 100 + k, device=dev, **VIT_S), cat, n, seed * 1000 + k))
+        k += 1
+    for i in range(2):
+        cat, n = (E.CAT_LS, ls_batch) if i == 0 else (E.CAT_FS, fs_batch)
+        out.append(Instance(srv, synth.make_decoder(seed=seed * 100 + k, device=dev, **DEC_1B), cat, n,
+                            seed * 1000 + k, kv_lo=kv_lo, kv_hi=kv_hi))
+        k += 1
+    return out
