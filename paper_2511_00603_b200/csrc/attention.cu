@@ -227,13 +227,32 @@ void launch_attn_fill_reqs(AttnReq* reqs, const int32_t* kv_lens, const int32_t*
 }
 
 // ------------------------------------------------------------------ encoder attention
-// One block per (image, head, block of ENC_QB query rows); K and V of the head sit in shared
-// memory as bf16; one thread per query row runs an online softmax over all T keys.
-constexpr int ENC_QB = 64;
-int attn_encoder_q_blocks(int T) { return (T + ENC_QB - 1) / ENC_QB; }
+// One block per (image, head, block of up to 256 query rows); one warp per 16 query rows.
+// K and V of the head are staged once in shared memory (bf16, rows padded to 72 elements so
+// that ldmatrix rows fall in distinct banks); each warp runs a flash-style loop over 64-key
+// blocks with mma.sync m16n8k16 (bf16 in, fp32 accumulate): S = Q K^T, online softmax in the
+// exp2 domain, O += P V.  Keys beyond T are masked; their padded rows are zero.
+constexpr int ENC_ROWS = 256;      // query rows per block
+constexpr int ENC_LD = 72;         // padded row length of K and V in shared memory
+int attn_encoder_q_blocks(int T) { return (T + ENC_ROWS - 1) / ENC_ROWS; }
+static int enc_key_pad(int T) { return (T + 63) / 64 * 64; }
 
-template <int HD>
-__global__ void __launch_bounds__(ENC_QB) attn_encoder_kernel(const AttnEncGroup* __restrict__ groups, int n_groups) {
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t* r, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+__global__ void __launch_bounds__(512, 1) attn_encoder_kernel(const AttnEncGroup* __restrict__ groups, int n_groups) {
+  constexpr int HD = 64;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   int gi = 0;
   for (int i = 1; i < n_groups; ++i) if ((int)blockIdx.x >= groups[i].blk_start) gi = i;
@@ -242,73 +261,139 @@ __global__ void __launch_bounds__(ENC_QB) attn_encoder_kernel(const AttnEncGroup
   const int qb = local % g.q_blocks, bh = local / g.q_blocks;
   const int h = bh % g.H, b = bh / g.H;
   const int T = g.T, d = g.H * HD;
+  const int Tp = (T + 63) / 64 * 64;
   bf16* Ks = reinterpret_cast<bf16*>(smem_raw);
-  bf16* Vs = Ks + (size_t)T * HD;
+  bf16* Vs = Ks + (size_t)Tp * ENC_LD;
   const bf16* base = g.qkv + (size_t)b * T * 3 * d + (size_t)h * HD;
-  for (int i = threadIdx.x; i < T * (HD / 8); i += blockDim.x) {
-    const int t = i / (HD / 8), cc = i % (HD / 8);
-    reinterpret_cast<uint4*>(Ks)[i] = *reinterpret_cast<const uint4*>(base + (size_t)t * 3 * d + d + cc * 8);
-    reinterpret_cast<uint4*>(Vs)[i] = *reinterpret_cast<const uint4*>(base + (size_t)t * 3 * d + 2 * d + cc * 8);
+  for (int i = threadIdx.x; i < Tp * (HD / 8); i += blockDim.x) {
+    const int t = i >> 3, cc = i & 7;
+    uint4 kk = make_uint4(0, 0, 0, 0), vv = kk;
+    if (t < T) {
+      kk = *reinterpret_cast<const uint4*>(base + (size_t)t * 3 * d + d + cc * 8);
+      vv = *reinterpret_cast<const uint4*>(base + (size_t)t * 3 * d + 2 * d + cc * 8);
+    }
+    *reinterpret_cast<uint4*>(Ks + (size_t)t * ENC_LD + cc * 8) = kk;
+    *reinterpret_cast<uint4*>(Vs + (size_t)t * ENC_LD + cc * 8) = vv;
   }
   __syncthreads();
-  const int row = qb * ENC_QB + threadIdx.x;
-  if (row >= T) return;
-  float q[HD], o[HD];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row0 = qb * ENC_ROWS + warp * 16;
+  if (row0 >= T) return;
+  const int gq = lane >> 2, tq = lane & 3;
+  // Q fragments of the warp's 16 rows: 4 k-steps of 16
+  uint32_t qa[4][4];
+  {
+    const int r_lo = row0 + gq, r_hi = row0 + gq + 8;
+    const bf16* q_lo = base + (size_t)min(r_lo, T - 1) * 3 * d;
+    const bf16* q_hi = base + (size_t)min(r_hi, T - 1) * 3 * d;
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      qa[ks][0] = *reinterpret_cast<const uint32_t*>(q_lo + ks * 16 + 2 * tq);
+      qa[ks][1] = *reinterpret_cast<const uint32_t*>(q_hi + ks * 16 + 2 * tq);
+      qa[ks][2] = *reinterpret_cast<const uint32_t*>(q_lo + ks * 16 + 2 * tq + 8);
+      qa[ks][3] = *reinterpret_cast<const uint32_t*>(q_hi + ks * 16 + 2 * tq + 8);
+    }
+  }
   const float scale = 1.4426950408889634f * rsqrtf((float)HD);
+  float o[8][4];
 #pragma unroll
-  for (int cc = 0; cc < HD / 8; ++cc) {
-    unpack8(*reinterpret_cast<const uint4*>(base + (size_t)row * 3 * d + cc * 8), q + cc * 8);
+  for (int n = 0; n < 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m_lo = -1e30f, m_hi = -1e30f, l_lo = 0.f, l_hi = 0.f;
+  const uint32_t ks_base = (uint32_t)__cvta_generic_to_shared(Ks);
+  const uint32_t vs_base = (uint32_t)__cvta_generic_to_shared(Vs);
+  // ldmatrix lane addressing: lanes 0-7 rows of matrix 0, 8-15 matrix 1, 16-23 matrix 2, 24-31 matrix 3
+  const int lm_row = lane & 7, lm_mat = lane >> 3;
+  for (int kb = 0; kb < Tp; kb += 64) {
+    float sc[8][4];
+#pragma unroll
+    for (int n = 0; n < 8; ++n) { sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f; }
+    // S = Q K^T : for key tiles (pairs of 8 keys) and k-steps
+#pragma unroll
+    for (int np = 0; np < 4; ++np) {        // key tiles 2np, 2np+1
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        // matrices: (keys 2np*8.., k lo), (keys 2np*8.., k hi), (keys (2np+1)*8.., k lo), (.., k hi)
+        const int key = kb + (2 * np + (lm_mat >> 1)) * 8 + lm_row;
+        const int kcol = ks * 16 + (lm_mat & 1) * 8;
+        uint32_t r[4];
+        ldmatrix_x4(r, ks_base + (uint32_t)(key * ENC_LD + kcol) * 2u);
+        mma_bf16_16816(sc[2 * np], qa[ks], r[0], r[1]);
+        mma_bf16_16816(sc[2 * np + 1], qa[ks], r[2], r[3]);
+      }
+    }
+    // scale, mask, online softmax (rows gq and gq+8 of the warp tile)
+    float mx_lo = m_lo, mx_hi = m_hi;
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const int key = kb + n * 8 + 2 * tq;
+      sc[n][0] = (key < T) ? sc[n][0] * scale : -INFINITY;
+      sc[n][1] = (key + 1 < T) ? sc[n][1] * scale : -INFINITY;
+      sc[n][2] = (key < T) ? sc[n][2] * scale : -INFINITY;
+      sc[n][3] = (key + 1 < T) ? sc[n][3] * scale : -INFINITY;
+      mx_lo = fmaxf(mx_lo, fmaxf(sc[n][0], sc[n][1]));
+      mx_hi = fmaxf(mx_hi, fmaxf(sc[n][2], sc[n][3]));
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    const float a_lo = exp2f(m_lo - mx_lo), a_hi = exp2f(m_hi - mx_hi);
+    m_lo = mx_lo; m_hi = mx_hi;
+    l_lo *= a_lo; l_hi *= a_hi;
+#pragma unroll
+    for (int n = 0; n < 8; ++n) { o[n][0] *= a_lo; o[n][1] *= a_lo; o[n][2] *= a_hi; o[n][3] *= a_hi; }
+    uint32_t pa[4][4];                       // P as A fragments: 4 k-steps of 16 keys
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const float p0 = exp2f(sc[n][0] - m_lo), p1 = exp2f(sc[n][1] - m_lo);
+      const float p2 = exp2f(sc[n][2] - m_hi), p3 = exp2f(sc[n][3] - m_hi);
+      l_lo += p0 + p1;
+      l_hi += p2 + p3;
+      pa[n >> 1][(n & 1) * 2 + 0] = pack2(p0, p1);
+      pa[n >> 1][(n & 1) * 2 + 1] = pack2(p2, p3);
+    }
+    // O += P V : k = keys (4 steps of 16), n = head dims (8 tiles of 8)
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {      // dim tiles 2np, 2np+1
+        // matrices: (keys lo 8, dims 2np*8..), (keys hi 8, dims 2np*8..), (keys lo, dims (2np+1)*8..), (keys hi, ..)
+        const int key = kb + ks * 16 + (lm_mat & 1) * 8 + lm_row;
+        const int col = (2 * np + (lm_mat >> 1)) * 8;
+        uint32_t r[4];
+        ldmatrix_x4_trans(r, vs_base + (uint32_t)(key * ENC_LD + col) * 2u);
+        mma_bf16_16816(o[2 * np], pa[ks], r[0], r[1]);
+        mma_bf16_16816(o[2 * np + 1], pa[ks], r[2], r[3]);
+      }
+    }
   }
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  const float i_lo = 1.0f / l_lo, i_hi = 1.0f / l_hi;
+  const int r_lo = row0 + gq, r_hi = row0 + gq + 8;
 #pragma unroll
-  for (int e = 0; e < HD; ++e) { q[e] *= scale; o[e] = 0.f; }
-  float m = -1e30f, l = 0.f;
-  for (int t = 0; t < T; ++t) {
-    float s = 0.f;
-#pragma unroll
-    for (int cc = 0; cc < HD / 8; ++cc) {
-      float kf[8];
-      unpack8(reinterpret_cast<const uint4*>(Ks + (size_t)t * HD)[cc], kf);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) s = fmaf(q[cc * 8 + e], kf[e], s);
-    }
-    if (s > m) {
-      const float sc = exp2f(m - s);
-      l *= sc;
-#pragma unroll
-      for (int e = 0; e < HD; ++e) o[e] *= sc;
-      m = s;
-    }
-    const float p = exp2f(s - m);
-    l += p;
-#pragma unroll
-    for (int cc = 0; cc < HD / 8; ++cc) {
-      float vf[8];
-      unpack8(reinterpret_cast<const uint4*>(Vs + (size_t)t * HD)[cc], vf);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) o[cc * 8 + e] = fmaf(p, vf[e], o[cc * 8 + e]);
-    }
-  }
-  const float inv = 1.0f / l;
-  bf16* out = g.out + ((size_t)b * T + row) * d + (size_t)h * HD;
-#pragma unroll
-  for (int cc = 0; cc < HD / 8; ++cc) {
-    uint4 u;
-    u.x = pack2(o[cc * 8 + 0] * inv, o[cc * 8 + 1] * inv);
-    u.y = pack2(o[cc * 8 + 2] * inv, o[cc * 8 + 3] * inv);
-    u.z = pack2(o[cc * 8 + 4] * inv, o[cc * 8 + 5] * inv);
-    u.w = pack2(o[cc * 8 + 6] * inv, o[cc * 8 + 7] * inv);
-    reinterpret_cast<uint4*>(out)[cc] = u;
+  for (int n = 0; n < 8; ++n) {
+    if (r_lo < T)
+      *reinterpret_cast<uint32_t*>(g.out + ((size_t)b * T + r_lo) * d + (size_t)h * HD + n * 8 + 2 * tq) =
+          pack2(o[n][0] * i_lo, o[n][1] * i_lo);
+    if (r_hi < T)
+      *reinterpret_cast<uint32_t*>(g.out + ((size_t)b * T + r_hi) * d + (size_t)h * HD + n * 8 + 2 * tq) =
+          pack2(o[n][2] * i_hi, o[n][3] * i_hi);
   }
 }
 
 cudaError_t launch_attn_encoder(const AttnEncGroup* groups, int n_groups, int total_blocks, int max_T,
                                 cudaStream_t st) {
   if (n_groups == 0 || total_blocks == 0) return cudaSuccess;
-  const size_t smem = (size_t)max_T * 64 * 2 * sizeof(bf16);
+  const size_t smem = (size_t)enc_key_pad(max_T) * ENC_LD * 2 * sizeof(bf16);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_encoder_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(attn_encoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
-  attn_encoder_kernel<64><<<total_blocks, ENC_QB, smem, st>>>(groups, n_groups);
+  const int rows = max_T < ENC_ROWS ? max_T : ENC_ROWS;
+  const int warps = (rows + 15) / 16;
+  attn_encoder_kernel<<<total_blocks, warps * 32, smem, st>>>(groups, n_groups);
   return cudaGetLastError();
 }
 

@@ -754,7 +754,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           case EPARA_K_NORM: {
             NormGroup g = op.norm;
             g.M = rows;
-            mx = std::max(mx, rows);
+            mx = std::max(mx, norm_blocks(rows, g.d));
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }

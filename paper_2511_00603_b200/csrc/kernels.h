@@ -6,7 +6,8 @@
 namespace epara {
 
 void launch_gather(const GatherGroup* groups, int n_groups, int max_blocks, cudaStream_t st);
-void launch_norm(const NormGroup* groups, int n_groups, int max_rows, cudaStream_t st);
+int norm_blocks(int M, int d);
+void launch_norm(const NormGroup* groups, int n_groups, int max_blocks, cudaStream_t st);
 void launch_rope_append(const RopeGroup* groups, int n_groups, int max_B, cudaStream_t st);
 void launch_assemble(const AssembleGroup* groups, int n_groups, int max_rows, cudaStream_t st);
 void launch_output(const OutputGroup* groups, int n_groups, int max_B, cudaStream_t st);

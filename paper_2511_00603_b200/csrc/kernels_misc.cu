@@ -49,40 +49,43 @@ void launch_gather(const GatherGroup* groups, int n_groups, int max_blocks, cuda
 }
 
 // ------------------------------------------------------------------ norms
-// One block per row; the row is held in registers (d <= 128 threads * 16 float4 = 8192).
-__global__ void __launch_bounds__(128) norm_kernel(const NormGroup* __restrict__ groups) {
-  __shared__ float red[32];
-  const NormGroup g = groups[blockIdx.y];
-  const int row = blockIdx.x;
-  if (row >= g.M) return;
+// Rows are held in registers between the statistics pass and the write.  Narrow rows
+// (d <= 1024) take one warp per row, 8 rows per block; wider rows one block per row.
+constexpr int NORM_THREADS = 256;
+constexpr int NORM_WARP_D = 1024;
+
+template <bool WARP>
+__device__ __forceinline__ void norm_row(const NormGroup& g, int row, float* red) {
+  constexpr int STRIDE = WARP ? 32 : NORM_THREADS;
+  const int t = WARP ? (threadIdx.x & 31) : threadIdx.x;
   const int nvec = g.d >> 2;
   const float4* x = reinterpret_cast<const float4*>(g.x + (size_t)row * g.x_stride);
-  float4 v[16];
+  float4 v[8];
   float s = 0.f;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int c = threadIdx.x + i * 128;
+  for (int i = 0; i < 8; ++i) {
+    const int c = t + i * STRIDE;
     if (c < nvec) {
       v[i] = x[c];
       s += (g.kind == NORM_LN) ? (v[i].x + v[i].y) + (v[i].z + v[i].w)
                                : (v[i].x * v[i].x + v[i].y * v[i].y) + (v[i].z * v[i].z + v[i].w * v[i].w);
     }
   }
-  s = block_sum(s, red);
+  s = WARP ? warp_sum(s) : block_sum(s, red);
   float mean = 0.f, rstd;
   const float inv_d = 1.0f / (float)g.d;
   if (g.kind == NORM_LN) {
     mean = s * inv_d;
     float q = 0.f;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int c = threadIdx.x + i * 128;
+    for (int i = 0; i < 8; ++i) {
+      const int c = t + i * STRIDE;
       if (c < nvec) {
         const float a = v[i].x - mean, b = v[i].y - mean, cc = v[i].z - mean, dd = v[i].w - mean;
         q += (a * a + b * b) + (cc * cc + dd * dd);
       }
     }
-    q = block_sum(q, red);
+    q = WARP ? warp_sum(q) : block_sum(q, red);
     rstd = 1.0f / sqrtf(q * inv_d + g.eps);
   } else {
     rstd = 1.0f / sqrtf(s * inv_d + g.eps);
@@ -91,15 +94,15 @@ __global__ void __launch_bounds__(128) norm_kernel(const NormGroup* __restrict__
   const uint2* gm = reinterpret_cast<const uint2*>(g.gamma);
   const uint2* bt = reinterpret_cast<const uint2*>(g.beta);
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int c = threadIdx.x + i * 128;
+  for (int i = 0; i < 8; ++i) {
+    const int c = t + i * STRIDE;
     if (c < nvec) {
-      const uint2 gg = gm[c];
+      const uint2 gg = __ldg(gm + c);
       float ga[4] = {__uint_as_float(gg.x << 16), __uint_as_float(gg.x & 0xffff0000u),
                      __uint_as_float(gg.y << 16), __uint_as_float(gg.y & 0xffff0000u)};
       float be[4] = {0.f, 0.f, 0.f, 0.f};
       if (g.kind == NORM_LN) {
-        const uint2 bb = bt[c];
+        const uint2 bb = __ldg(bt + c);
         be[0] = __uint_as_float(bb.x << 16); be[1] = __uint_as_float(bb.x & 0xffff0000u);
         be[2] = __uint_as_float(bb.y << 16); be[3] = __uint_as_float(bb.y & 0xffff0000u);
       }
@@ -111,9 +114,23 @@ __global__ void __launch_bounds__(128) norm_kernel(const NormGroup* __restrict__
   }
 }
 
-void launch_norm(const NormGroup* groups, int n_groups, int max_rows, cudaStream_t st) {
-  if (n_groups == 0 || max_rows == 0) return;
-  norm_kernel<<<dim3(max_rows, n_groups), 128, 0, st>>>(groups);
+__global__ void __launch_bounds__(NORM_THREADS) norm_kernel(const NormGroup* __restrict__ groups) {
+  __shared__ float red[32];
+  const NormGroup g = groups[blockIdx.y];
+  if (g.d <= NORM_WARP_D) {
+    const int row = blockIdx.x * (NORM_THREADS / 32) + (threadIdx.x >> 5);
+    if (row < g.M) norm_row<true>(g, row, red);
+  } else {
+    if ((int)blockIdx.x < g.M) norm_row<false>(g, blockIdx.x, red);
+  }
+}
+
+// Blocks a group of M rows of width d needs.
+int norm_blocks(int M, int d) { return d <= NORM_WARP_D ? (M + NORM_THREADS / 32 - 1) / (NORM_THREADS / 32) : M; }
+
+void launch_norm(const NormGroup* groups, int n_groups, int max_blocks, cudaStream_t st) {
+  if (n_groups == 0 || max_blocks == 0) return;
+  norm_kernel<<<dim3(max_blocks, n_groups), NORM_THREADS, 0, st>>>(groups);
 }
 
 // ------------------------------------------------------------------ RoPE + KV append

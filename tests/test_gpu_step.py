@@ -119,7 +119,7 @@ def test_config2_vit_b16_batch_2(mods):
     srv.close()
 
 
-def _decoder_case(E, server, p, B, lo, hi, seed, impl=None, n_check=None):
+def _decoder_case(E, server, p, B, lo, hi, seed, impl=None, n_check=None, deep=False):
     toks, lens, tables, npages = synth.make_decode_batch(B, lo, hi, p["vocab"], seed=seed)
     pool = synth.make_kv_pool(p["n_layers"], npages, p["n_kv_heads"], p["head_dim"], seed=seed + 1, device=DEV)
     pool_before = synth.to_bits(pool)
@@ -137,15 +137,16 @@ def _decoder_case(E, server, p, B, lo, hi, seed, impl=None, n_check=None):
         r = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], lambda l, pg: pool_before[l, pg], v)
         rb = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], lambda l, pg: pool_before[l, pg], v,
                             round_bf16=True)
-        e = assert_parity(res[i][0], r["logits"], rb["logits"], what=f"decoder req {i} (L={lens[i]})")
+        e = assert_parity(res[i][0], r["logits"], rb["logits"], what=f"decoder req {i} (L={lens[i]})",
+                          deep=deep)
         print(f"decoder req {i} L={lens[i]}: {e}")
         decided += check_argmax(res[i][1], res[i][0], rb["logits"])
         for l, ap in enumerate(rb["appended"]):
             # the new k, v land in exactly the (page, slot) the block table names
             got_k = O.bf16_to_f64(pool_after[l, ap["page"], 0, :, ap["slot"], :])
             got_v = O.bf16_to_f64(pool_after[l, ap["page"], 1, :, ap["slot"], :])
-            assert_close(got_k, ap["k"], what=f"appended k req {i} layer {l}")
-            assert_close(got_v, ap["v"], what=f"appended v req {i} layer {l}")
+            assert_close(got_k, ap["k"], what=f"appended k req {i} layer {l}", tol=0.15 if deep else 2e-2)
+            assert_close(got_v, ap["v"], what=f"appended v req {i} layer {l}", tol=0.15 if deep else 2e-2)
     for i in range(B):
         touched[:, int(tables[i][lens[i] // 16]), int(lens[i]) % 16] = True
     same = (pool_before == pool_after).all(axis=(2, 3, 5))          # [layer, page, slot]
@@ -168,9 +169,19 @@ def test_config3_decoder_1b_batch_4(mods):
     E, server = mods
     p = synth.make_decoder(d=2048, n_layers=16, n_q_heads=32, n_kv_heads=8, head_dim=64, ffn=8192, vocab=32000,
                            seed=2, device=DEV)
-    info, decided = _decoder_case(E, server, p, B=4, lo=128, hi=4096, seed=21, n_check=2)
+    info, decided = _decoder_case(E, server, p, B=4, lo=128, hi=4096, seed=21, n_check=2, deep=True)
     assert info.weight_bytes == pytest.approx(2 * (16 * (3072 * 2048 + 2048 * 2048 + 16384 * 2048 + 2048 * 8192)
                                                    + 32000 * 2048))
+
+
+@pytest.mark.parametrize("n_layers", [1, 2])
+def test_config3_shapes_shallow_strict(mods, n_layers):
+    """The 1B decoder's layer shapes (d 2048, 32/8 heads, FFN 8192, vocab 32000) at depth 1 and 2:
+    strict element-wise tolerance."""
+    E, server = mods
+    p = synth.make_decoder(d=2048, n_layers=n_layers, n_q_heads=32, n_kv_heads=8, head_dim=64, ffn=8192, vocab=32000,
+                           seed=2, device=DEV)
+    _decoder_case(E, server, p, B=5, lo=128, hi=4096, seed=22, n_check=3)
 
 
 def test_decoder_batch_invariance_and_mixed_models(mods):
