@@ -412,8 +412,96 @@ def run_gpu(args):
     return 0
 
 
+# ------------------------------------------------------------------------------ single-kernel timings
+MICRO_GEMM = {
+    "vit_s": [(50432, 1152, 384, "bias"), (50432, 384, 384, "bias,resid"), (50432, 1536, 384, "bias,gelu"),
+              (50432, 384, 1536, "bias,resid")],
+    "vit_b": [(12608, 2304, 768, "bias"), (12608, 768, 768, "bias,resid"), (12608, 3072, 768, "bias,gelu"),
+              (12608, 768, 3072, "bias,resid")],
+    "dec_1b": [(128, 3072, 2048, ""), (128, 2048, 2048, "resid"), (128, 16384, 2048, "swiglu"), (128, 2048, 8192, "resid"),
+               (128, 32000, 2048, "")],
+    "dec_8b": [(256, 6144, 4096, ""), (256, 4096, 4096, "resid"), (256, 28672, 4096, "swiglu"), (256, 4096, 14336, "resid"),
+               (256, 32000, 4096, "")],
+    "square": [(8192, 8192, 8192, "")],
+}
+
+
+def run_micro(args):
+    """Times one kernel through its C-ABI entry point on seeded inputs; one JSON line per case."""
+    import torch
+    from paper_2511_00603_b200 import build
+    build.build()
+    from paper_2511_00603_b200 import epara as E, synth
+    peaks = read_peaks()
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    g = torch.Generator(device=dev).manual_seed(0)
+
+    def timed(fn, reps):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        for a, b in ev:
+            flush.zero_()                      # L2 flush between timed launches
+            a.record(stream)
+            fn()
+            b.record(stream)
+        torch.cuda.synchronize()
+        ms = sorted(a.elapsed_time(b) for a, b in ev)
+        return ms[len(ms) // 2]
+
+    if args.micro == "gemm":
+        for (M, N, K, fl) in MICRO_GEMM[args.case]:
+            if args.m:
+                M = args.m
+            fl = set(x for x in fl.split(",") if x)
+            A = torch.randn((M, K), generator=g, device=dev).to(torch.bfloat16)
+            Wt = (torch.randn((N, K), generator=g, device=dev) * 0.02).to(torch.bfloat16)
+            bias = torch.zeros(N, device=dev, dtype=torch.bfloat16) if "bias" in fl else None
+            epi = (E.EPI_BIAS if "bias" in fl else 0) | (E.EPI_GELU if "gelu" in fl else 0) | \
+                  (E.EPI_SWIGLU if "swiglu" in fl else 0) | (E.EPI_RESID_F32 if "resid" in fl else 0)
+            ncol = N // 2 if "swiglu" in fl else N
+            Cc = torch.zeros((M, ncol), device=dev, dtype=torch.float32 if "resid" in fl else torch.bfloat16)
+            prob = [{"A": A, "W": Wt, "C": Cc, "bias": bias, "M": M, "N": N, "K": K, "epilogue": epi}]
+            scratch = torch.empty(E.lib.epara_gemm_scratch_bytes(1), dtype=torch.uint8, device=dev)
+            ms = timed(lambda: E.epara_grouped_gemm(prob, stream.cuda_stream, scratch), args.steps)
+            tf = 2.0 * M * N * K / (ms / 1e3) / 1e12
+            gbs = 2.0 * N * K / (ms / 1e3) / 1e9
+            print(json.dumps({"kernel": "gemm_tc", "M": M, "N": N, "K": K, "epilogue": sorted(fl), "ms": ms, "tflops": tf,
+                              "frac_tensor_burst": tf / peaks["bf16_tflops"], "weight_gbs": gbs,
+                              "frac_hbm_weights": gbs / peaks["hbm_gbs"]}))
+    elif args.micro == "attn_dec":
+        import numpy as np
+        Hq, Hkv, hd = (32, 8, 128) if args.case == "dec_8b" else (32, 8, 64)
+        B = args.m or 128
+        hi = 8192 if args.case == "dec_8b" else 4096
+        toks, lens, tables, npages = synth.make_decode_batch(B, 128, hi, 32000, seed=2)
+        lens = lens + 1
+        stride = max(len(t) for t in tables)
+        tb = np.zeros((B, stride), dtype=np.int32)
+        for b, t in enumerate(tables):
+            tb[b, :len(t)] = t
+        pool = synth.make_kv_pool(1, npages, Hkv, hd, seed=3, device=dev)[0]
+        q = torch.randn((B, Hq * hd), generator=g, device=dev).to(torch.bfloat16)
+        out = torch.empty_like(q)
+        max_len = int(lens.max())
+        scratch = torch.empty(E.lib.epara_decode_attention_scratch_bytes(B, Hq, hd, max_len), dtype=torch.uint8, device=dev)
+        lens_d, tb_d = torch.as_tensor(lens, device=dev), torch.as_tensor(tb, device=dev)
+        ms = timed(lambda: E.epara_decode_attention(q, pool, lens_d, tb_d, out, Hq, Hkv, hd, max_len, scratch,
+                                                    stream.cuda_stream), args.steps)
+        kvb = float(lens.sum()) * 2 * Hkv * hd * 2
+        print(json.dumps({"kernel": "attn_decode+combine", "B": B, "Hq": Hq, "Hkv": Hkv, "hd": hd, "tokens": int(lens.sum()),
+                          "ms": ms, "kv_gbs": kvb / (ms / 1e3) / 1e9, "frac_hbm": kvb / (ms / 1e3) / 1e9 / peaks["hbm_gbs"]}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--micro", default=None, choices=["gemm", "attn_dec"], help="time one kernel instead of the step")
+    ap.add_argument("--case", default="vit_s")
+    ap.add_argument("--m", type=int, default=0, help="override M (gemm) or B (attn_dec) of the micro case")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
@@ -423,6 +511,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.micro:
+        return run_micro(args)
     return run_gpu(args)
 
 

@@ -950,7 +950,7 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
   if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) return EPARA_E_CUDA;
   if (cudaMemcpyAsync(dev_groups, gs.data(), gs.size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return EPARA_E_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return EPARA_E_CUDA;   // gs is pageable host memory
+  // (a copy from pageable host memory is staged before cudaMemcpyAsync returns, so gs may go out of scope)
   cudaError_t err = cudaSuccess;
   if (simt) {
     launch_gemm_simt(dev_groups, n, total, st);
@@ -988,7 +988,6 @@ int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_s
   g.partial = (float*)(s + 256 + align_up((size_t)B * sizeof(AttnReq), 256));
   g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK; g.req_start = 0;
   if (cudaMemcpyAsync(s, &g, sizeof(g), cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return EPARA_E_CUDA;
   launch_attn_fill_reqs(reqs, kv_lens, tables, table_stride, B, st);
   cudaError_t e = launch_attn_decode((const AttnDecGroup*)s, 1, B, Hkv, g.max_chunks, hd, Hq / Hkv, st);
   if (e == cudaErrorInvalidValue) return EPARA_E_UNSUPPORTED;
