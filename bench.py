@@ -465,7 +465,7 @@ def run_micro(args):
             ncol = N // 2 if "swiglu" in fl else N
             Cc = torch.zeros((M, ncol), device=dev, dtype=torch.float32 if "resid" in fl else torch.bfloat16)
             prob = [{"A": A, "W": Wt, "C": Cc, "bias": bias, "M": M, "N": N, "K": K, "epilogue": epi}]
-            scratch = torch.empty(E.lib.epara_gemm_scratch_bytes(1), dtype=torch.uint8, device=dev)
+            scratch = torch.empty(E.epara_gemm_scratch_bytes_for(prob), dtype=torch.uint8, device=dev)
             ms = timed(lambda: E.epara_grouped_gemm(prob, stream.cuda_stream, scratch), args.steps)
             tf = 2.0 * M * N * K / (ms / 1e3) / 1e12
             gbs = 2.0 * N * K / (ms / 1e3) / 1e9

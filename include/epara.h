@@ -221,10 +221,13 @@ enum { EPARA_EPI_BIAS = 1, EPARA_EPI_GELU = 2, EPARA_EPI_SWIGLU = 4, EPARA_EPI_R
 
 /* C_g = epilogue(A_g W_g^T + bias_g) for every problem in one grouped launch.  RESID_F32:
  * C is fp32 and is updated in place, C += A W^T + bias.  `problems` is host memory;
- * `scratch` is device memory of at least epara_gemm_scratch_bytes(n) bytes. */
+ * `scratch` is device memory, 256-byte aligned, of at least epara_gemm_scratch_bytes_for(problems, n)
+ * bytes (descriptors, plus fp32 partials for small-M problems that are split along K);
+ * epara_gemm_scratch_bytes(n) suffices for EPARA_GEMM_SIMT. */
 int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm_problem* problems, int n,
                        void* scratch, size_t scratch_bytes);
 size_t epara_gemm_scratch_bytes(int n_problems);
+size_t epara_gemm_scratch_bytes_for(const epara_gemm_problem* problems, int n);
 
 /* Split-KV paged decode attention with GQA (one layer).  q: bf16 [B, q_stride] (head h at
  * column h*hd); kv_layer: bf16 [pages][2][Hkv][16][hd]; kv_lens int32 [B] = tokens to attend

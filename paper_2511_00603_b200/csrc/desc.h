@@ -25,7 +25,10 @@ struct ReqDesc {
 };
 
 // C = epi(A W^T + bias).  tmA/tmW are the TMA maps of A [rows, K] and W [N, K] (K innermost,
-// 128-byte swizzle, box 64 x 128 rows for A and 64 x BN rows for W).
+// 128-byte swizzle, box 64 x 128 rows for A and 64 x bn rows for W).  The tensor-core kernel cuts
+// the group into tiles_m x tiles_n tiles of 128 x bn and every tile into ksplit ranges of
+// k-blocks; with ksplit > 1 each range leaves an fp32 partial in `partial` and the range that
+// arrives last (counted in `counters`) adds them in range order and runs the epilogue.
 struct alignas(64) GemmGroup {
   CUtensorMap tmA;
   CUtensorMap tmW;
@@ -36,9 +39,11 @@ struct alignas(64) GemmGroup {
   int M, N, K;
   int lda, ldw, ldc;
   int epi;
-  int tile_start;  // first tile index of this group in the launch
+  int tile_start;  // first work item of this group in the launch
   int tiles_m, tiles_n;
-  int pad0, pad1;
+  int bn, ksplit;  // tensor-core kernel only: tile width (128 or 256), k ranges per tile
+  float* partial;  // [ksplit][tiles_m * 128][tiles_n * bn] fp32, ksplit > 1 only
+  int* counters;   // [tiles_m * tiles_n], zero between launches
 };
 
 struct GemmLaunch {      // header followed by groups

@@ -103,6 +103,7 @@ struct Model {
   std::deque<Request> q[2];
   int max_chunks;       // decoder
   double kv_bytes_per_token;
+  size_t splitk_bytes = 0, splitk_tiles = 0;   // largest split-k partial buffer / tile count of its GEMMs
 };
 
 struct Slot {
@@ -164,6 +165,7 @@ struct Builder {
   epara_ctx* c;
   size_t need;
   bool fail;
+  int sm_count;
   void* get(size_t bytes) {
     if (!c) { carve_size(need, bytes); return reinterpret_cast<void*>(size_t(256)); }
     void* p = carve(c, bytes);
@@ -174,6 +176,7 @@ struct Builder {
 
 bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap, const void* W, int N, int K,
               void* C, int ldc, const void* bias, int epi, int rows_per_req) {
+  const int sm_count = bl.sm_count;
   Op op;
   memset(&op, 0, sizeof(op));
   op.kind = EPARA_K_GEMM;
@@ -182,9 +185,15 @@ bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap,
   g.A = (const bf16*)A; g.W = (const bf16*)W; g.C = C; g.bias = (const bf16*)bias;
   g.N = N; g.K = K; g.lda = lda; g.ldw = K; g.ldc = ldc; g.epi = epi | (bias ? EPI_BIAS : 0);
   op.weight_bytes = 2.0 * N * K;
+  gemm_tc_config(rows_cap, N, K, g.epi, sm_count, &g.bn, &g.ksplit);
+  if (g.ksplit > 1) {
+    const size_t tiles_m = (size_t)((rows_cap + TC_BM - 1) / TC_BM), tiles_n = (size_t)((N + g.bn - 1) / g.bn);
+    m->splitk_bytes = std::max(m->splitk_bytes, (size_t)g.ksplit * tiles_m * TC_BM * tiles_n * g.bn * 4);
+    m->splitk_tiles = std::max(m->splitk_tiles, tiles_m * tiles_n);
+  }
   if (bl.c) {
     if (!make_tmap(&g.tmA, A, rows_cap, K, lda, TC_BM)) return false;
-    if (!make_tmap(&g.tmW, W, N, K, K, TC_BN)) return false;
+    if (!make_tmap(&g.tmW, W, N, K, K, g.bn)) return false;
   }
   m->ops.push_back(op);
   return true;
@@ -384,6 +393,21 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
   return EPARA_OK;
 }
 
+// Split-k scratch shared by the model's GEMMs (they run one after the other): fp32 partials and
+// per-tile arrival counters (zero between launches).
+int finish_model(Builder& bl, Model* m) {
+  if (m->splitk_bytes == 0) return EPARA_OK;
+  float* partial = (float*)bl.get(m->splitk_bytes);
+  int* counters = (int*)bl.get(m->splitk_tiles * sizeof(int));
+  if (bl.fail) return EPARA_E_RESOURCE;
+  if (bl.c) {
+    if (cudaMemset(counters, 0, m->splitk_tiles * sizeof(int)) != cudaSuccess) return EPARA_E_CUDA;
+    for (Op& op : m->ops)
+      if (op.kind == EPARA_K_GEMM && op.gemm.ksplit > 1) { op.gemm.partial = partial; op.gemm.counters = counters; }
+  }
+  return EPARA_OK;
+}
+
 int effective_max_batch(const epara_config& cfg, const epara_model_desc& d) {
   const int ls = cfg.cap_ls > 0 ? cfg.cap_ls : 4, fs = cfg.cap_fs > 0 ? cfg.cap_fs : 256;
   return d.max_batch > 0 ? d.max_batch : ls + fs;
@@ -469,8 +493,9 @@ size_t epara_model_workspace_bytes(const epara_config* cfg, const epara_model_de
   m.tensors.assign(d->tensors, d->tensors + d->n_tensors);
   if (d->kind == EPARA_MODEL_MLP) m.dims.assign(d->mlp_dims, d->mlp_dims + d->n_layers + 1);
   m.max_batch = effective_max_batch(*cfg, *d);
-  Builder bl{nullptr, 0, false};
+  Builder bl{nullptr, 0, false, 148};
   build_model(bl, &m, *cfg);
+  finish_model(bl, &m);
   return bl.need + 256;
 }
 
@@ -546,8 +571,9 @@ int epara_register_model(epara_ctx* c, const epara_model_desc* d, int* model_id)
   m->max_chunks = 0;
   m->kv_bytes_per_token = 0;
   const size_t mark = c->ws_used;
-  Builder bl{c, 0, false};
+  Builder bl{c, 0, false, c->sm_count};
   int r = build_model(bl, m, c->cfg);
+  if (r == EPARA_OK) r = finish_model(bl, m);
   if (r != EPARA_OK) {
     c->ws_used = mark;
     delete m;
@@ -761,10 +787,10 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           case EPARA_K_GEMM: {
             GemmGroup g = op.gemm;
             g.M = rows;
-            const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : TC_BN;
+            const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : g.bn;
             g.tiles_m = (rows + tm - 1) / tm; g.tiles_n = (g.N + tn - 1) / tn;
             g.tile_start = total;
-            total += g.tiles_m * g.tiles_n;
+            total += g.tiles_m * g.tiles_n * (simt ? 1 : g.ksplit);
             inf.gemm_groups++;
             inf.gemm_flops += 2.0 * rows * g.N * g.K;
             inf.weight_bytes += op.weight_bytes;
@@ -913,16 +939,32 @@ int epara_step_profile(epara_ctx* c, float* ms_per_kind, int* launches_per_kind)
 // ---------------------------------------------------------------- single-kernel entry points
 size_t epara_gemm_scratch_bytes(int n) { return (size_t)(n > 0 ? n : 0) * sizeof(GemmGroup) + 256; }
 
+size_t epara_gemm_scratch_bytes_for(const epara_gemm_problem* p, int n) {
+  size_t bytes = epara_gemm_scratch_bytes(n);
+  for (int i = 0; i < n && p; ++i) {
+    int bn = 128, ks = 1;
+    gemm_tc_config(p[i].M, p[i].N, p[i].K, p[i].epilogue, 148, &bn, &ks);
+    if (ks > 1) {
+      const size_t tiles_m = (size_t)(p[i].M + TC_BM - 1) / TC_BM, tiles_n = (size_t)(p[i].N + bn - 1) / bn;
+      bytes = align_up(bytes, 256) + (size_t)ks * tiles_m * TC_BM * tiles_n * bn * 4;
+      bytes = align_up(bytes, 256) + tiles_m * tiles_n * sizeof(int);
+    }
+  }
+  return bytes;
+}
+
 int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm_problem* p, int n, void* scratch,
                        size_t scratch_bytes) {
   if (n < 0 || (n > 0 && !p) || !scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return EPARA_E_INVALID;
-  if (scratch_bytes < epara_gemm_scratch_bytes(n)) return EPARA_E_RESOURCE;
+  if (scratch_bytes < (impl == EPARA_GEMM_SIMT ? epara_gemm_scratch_bytes(n) : epara_gemm_scratch_bytes_for(p, n)))
+    return EPARA_E_RESOURCE;
   if (n == 0) return EPARA_OK;
   if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool simt = impl == EPARA_GEMM_SIMT;
   std::vector<GemmGroup> gs(n);
   int total = 0;
+  size_t soff = epara_gemm_scratch_bytes(n);
   for (int i = 0; i < n; ++i) {
     const epara_gemm_problem& q = p[i];
     if (!q.A || !q.W || !q.C || q.M < 0 || q.N <= 0 || q.K <= 0) return EPARA_E_INVALID;
@@ -936,13 +978,24 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
     memset(&g, 0, sizeof(g));
     g.A = (const bf16*)q.A; g.W = (const bf16*)q.W; g.C = q.C; g.bias = (const bf16*)q.bias;
     g.M = q.M; g.N = q.N; g.K = q.K; g.lda = q.lda; g.ldw = q.ldw; g.ldc = q.ldc; g.epi = q.epilogue;
-    const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : TC_BN;
+    g.bn = 128; g.ksplit = 1;
+    if (!simt) gemm_tc_config(q.M, q.N, q.K, q.epilogue, 148, &g.bn, &g.ksplit);
+    const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : g.bn;
     g.tiles_m = (q.M + tm - 1) / tm; g.tiles_n = (q.N + tn - 1) / tn;
     g.tile_start = total;
-    total += g.tiles_m * g.tiles_n;
+    total += g.tiles_m * g.tiles_n * g.ksplit;
     if (!simt && q.M > 0) {
       if (!make_tmap(&g.tmA, q.A, q.M, q.K, q.lda, TC_BM)) return EPARA_E_CUDA;
-      if (!make_tmap(&g.tmW, q.W, q.N, q.K, q.ldw, TC_BN)) return EPARA_E_CUDA;
+      if (!make_tmap(&g.tmW, q.W, q.N, q.K, q.ldw, g.bn)) return EPARA_E_CUDA;
+    }
+    if (g.ksplit > 1) {
+      soff = align_up(soff, 256);
+      g.partial = (float*)((unsigned char*)scratch + soff);
+      soff += (size_t)g.ksplit * g.tiles_m * TC_BM * g.tiles_n * g.bn * 4;
+      soff = align_up(soff, 256);
+      g.counters = (int*)((unsigned char*)scratch + soff);
+      if (cudaMemsetAsync(g.counters, 0, (size_t)g.tiles_m * g.tiles_n * sizeof(int), st) != cudaSuccess) return EPARA_E_CUDA;
+      soff += (size_t)g.tiles_m * g.tiles_n * sizeof(int);
     }
   }
   int* status = (int*)scratch;

@@ -1,18 +1,22 @@
 // Grouped bf16 GEMM on the sm_100a tensor cores: C_g = epi(A_g W_g^T + bias_g).
 //
 // One persistent launch covers every group (one group = one model's GEMM in this wave, with its
-// own M, N, K).  Tiles of 128 x TC_BN are numbered group after group; CTA i takes tiles
-// i, i + grid, ...  Inside a CTA three roles run concurrently:
+// own M, N, K, tile width bn in {128, 256} and k-split count).  Work items -- (tile, k range) --
+// are numbered group after group; CTA i takes items i, i + grid, ...  Inside a CTA three roles
+// run concurrently:
 //   warp 0 (one lane)  TMA producer: for each 64-wide k-block loads the A tile (128 x 64) and the
-//                      W tile (TC_BN x 64) into a ring of shared-memory stages (plain, non-multicast
+//                      W tile (bn x 64) into a ring of shared-memory stages (plain, non-multicast
 //                      cp.async.bulk.tensor; out-of-range rows/columns arrive as zeros);
-//   warp 1 (one lane)  MMA issuer: tcgen05.mma (M 128, N TC_BN, K 16) from shared memory into one
-//                      of two TMEM accumulators, releasing stages with tcgen05.commit;
-//   warps 2..5         epilogue: tcgen05.ld of the finished accumulator, bias / GELU / SwiGLU /
-//                      fp32 residual update, bf16 store -- while the MMA warp already fills the
-//                      other accumulator.
-// The K reduction of an output element is always the same sequence of k-blocks, whatever else is
-// in the launch, so results do not depend on co-resident groups.
+//   warp 1 (one lane)  MMA issuer: tcgen05.mma (M 128, N bn, K 16) from shared memory into one
+//                      of two TMEM accumulators (256 columns each), releasing stages with
+//                      tcgen05.commit;
+//   warps 2..9         epilogue: tcgen05.ld of the finished accumulator (two warps per TMEM lane
+//                      quarter, alternating 32-column chunks), bias / GELU / SwiGLU / fp32 residual
+//                      update, bf16 store -- while the MMA warp already fills the other accumulator.
+// Split-k (weight-streaming groups with few tiles): every k range of a tile writes its fp32
+// partial; the range that finishes last (an atomic counter per tile, no waiting) adds the partials
+// in range order and runs the epilogue, so the result does not depend on arrival order.
+// The K reduction of an output element is the same sequence whatever else is in the launch.
 // Every mbarrier wait is bounded: when a wait runs out the kernel records a code in *status, all
 // roles leave their loops, TMEM is freed and the kernel returns.
 #include "common.cuh"
@@ -22,13 +26,16 @@ namespace epara {
 
 namespace {
 
-constexpr int STAGES = 6;
+constexpr int STAGES = 4;
 constexpr int A_BYTES = TC_BM * TC_BK * 2;          // 16 KB
-constexpr int B_BYTES = TC_BN * TC_BK * 2;          // 16 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int TMEM_COLS = 2 * TC_BN;                // two accumulators
-constexpr int N_THREADS = 192;
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + 256;
+constexpr int B_BYTES_MAX = TC_BN_MAX * TC_BK * 2;  // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES_MAX;
+constexpr int ACC_COLS = TC_BN_MAX;                 // TMEM columns per accumulator
+constexpr int TMEM_COLS = 2 * ACC_COLS;             // 512: the whole TMEM of the SM
+constexpr int EPI_WARPS = 8;
+constexpr int N_THREADS = 64 + EPI_WARPS * 32;
+constexpr int STAGE_OUT_BYTES = 128 * 256;          // epilogue staging: 128 rows x 256 bytes
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + STAGE_OUT_BYTES + 256;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -54,11 +61,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
-    if ((it & 63u) == 63u) {
+    if ((it & 1023u) == 1023u) {
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer();
       if (t0 == 0) t0 = now;
@@ -87,15 +94,17 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
   d |= (uint64_t)2 << 61;                           // SWIZZLE_128B
   return d;
 }
-// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = TC_BN.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = bn.
+__device__ __forceinline__ uint32_t make_idesc(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
 
-__device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+__device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -111,105 +120,199 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// Two 32-column loads in flight, one wait: the read latency is paid once per 64 columns.
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(EPI_WARPS * 32) : "memory"); }
 
-__device__ __forceinline__ int find_group_tc(const GemmGroup* groups, int n, int tile) {
+__device__ __forceinline__ int find_group_tc(const GemmGroup* groups, int n, int item) {
   int lo = 0, hi = n - 1;
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
-    if (groups[mid].tile_start <= tile) lo = mid; else hi = mid - 1;
+    if (groups[mid].tile_start <= item) lo = mid; else hi = mid - 1;
   }
   return lo;
 }
 
-// Epilogue of 32 consecutive columns [n, n+32) of one row.
-__device__ __forceinline__ void epilogue_row(const GemmGroup& g, int m, int n, const uint32_t* r) {
+// Register copy of a group's scalar fields for the epilogue threads.  The descriptors live in
+// global memory and the epilogue is full of asm statements that clobber memory, so reading
+// fields through the descriptor pointer would reload them (at L2 latency) again and again.
+struct GView {
+  const bf16* bias;
+  void* C;
+  float* partial;
+  int* counters;
+  int M, N, K, ldc, epi, tile_start, tiles_m, tiles_n, bn, ksplit;
+};
+__device__ __forceinline__ GView load_view(const GemmGroup* g) {
+  GView v;
+  v.bias = g->bias; v.C = g->C; v.partial = g->partial; v.counters = g->counters;
+  v.M = g->M; v.N = g->N; v.K = g->K; v.ldc = g->ldc; v.epi = g->epi; v.tile_start = g->tile_start;
+  v.tiles_m = g->tiles_m; v.tiles_n = g->tiles_n; v.bn = g->bn; v.ksplit = g->ksplit;
+  return v;
+}
+
+// A work item of a group: tile (tm, tn) and k-block range [kb0, kb1).
+struct Item {
+  int m0, n0, tile, split, kb0, kb1;
+};
+template <class G>
+__device__ __forceinline__ Item decode_item(const G& g, int local) {
+  Item it;
+  it.split = local % g.ksplit;
+  it.tile = local / g.ksplit;
+  it.m0 = (it.tile / g.tiles_n) * TC_BM;
+  it.n0 = (it.tile % g.tiles_n) * g.bn;
+  const int kblocks = (g.K + TC_BK - 1) / TC_BK;
+  const int per = (kblocks + g.ksplit - 1) / g.ksplit;
+  it.kb0 = it.split * per;
+  it.kb1 = min(kblocks, it.kb0 + per);
+  return it;
+}
+
+// Per-thread copy of the fields the single-thread roles need, refreshed only when the item leaves
+// the current group (descriptor reads from global memory are latency the MMA issuer cannot hide).
+struct GroupCache {
+  const GemmGroup* g;
+  int start, end, tiles_n, ksplit, bn, kblocks;
+};
+__device__ __forceinline__ void group_cache(GroupCache& c, const GemmGroup* groups, int n_groups, int item) {
+  if (c.g != nullptr && item >= c.start && item < c.end) return;
+  const GemmGroup* g = groups + find_group_tc(groups, n_groups, item);
+  c.g = g;
+  c.start = g->tile_start;
+  c.tiles_n = g->tiles_n;
+  c.ksplit = g->ksplit;
+  c.bn = g->bn;
+  c.end = c.start + g->tiles_m * g->tiles_n * g->ksplit;
+  c.kblocks = (g->K + TC_BK - 1) / TC_BK;
+}
+__device__ __forceinline__ Item decode_item(const GroupCache& c, int item) {
+  const int local = item - c.start;
+  Item it;
+  it.split = local % c.ksplit;
+  it.tile = local / c.ksplit;
+  it.m0 = (it.tile / c.tiles_n) * TC_BM;
+  it.n0 = (it.tile % c.tiles_n) * c.bn;
+  const int per = (c.kblocks + c.ksplit - 1) / c.ksplit;
+  it.kb0 = it.split * per;
+  it.kb1 = min(c.kblocks, it.kb0 + per);
+  return it;
+}
+
+// Epilogue of 4 consecutive columns [n, n+4) of one row (split-k reduction path).
+__device__ __forceinline__ void epilogue4(const GView& g, int m, int n, float4 a) {
   const int N = g.N;
-  float v[32];
-#pragma unroll
-  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-  const bool full = (n + 32 <= N);
+  float v[4] = {a.x, a.y, a.z, a.w};
+  const bool full = (n + 4 <= N);
   if (g.epi & EPI_BIAS) {
-    if (full) {
 #pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        float b[8];
-        unpack8(__ldg(reinterpret_cast<const uint4*>(g.bias + n + j)), b);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) v[j + e] += b[e];
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) if (n + j < N) v[j] += bf2f(g.bias[n + j]);
-    }
+    for (int j = 0; j < 4; ++j) if (n + j < N) v[j] += bf2f(g.bias[n + j]);
   }
   if (g.epi & EPI_GELU) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+    for (int j = 0; j < 4; ++j) v[j] = gelu_erf(v[j]);
   }
   if (g.epi & EPI_RESID_F32) {
     float* C = reinterpret_cast<float*>(g.C) + (size_t)m * g.ldc + n;
     if (full) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 4) {
-        float4 c = *reinterpret_cast<float4*>(C + j);
-        c.x += v[j]; c.y += v[j + 1]; c.z += v[j + 2]; c.w += v[j + 3];
-        *reinterpret_cast<float4*>(C + j) = c;
-      }
+      float4 c = *reinterpret_cast<float4*>(C);
+      c.x += v[0]; c.y += v[1]; c.z += v[2]; c.w += v[3];
+      *reinterpret_cast<float4*>(C) = c;
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (n + j < N) C[j] += v[j];
+      for (int j = 0; j < 4; ++j) if (n + j < N) C[j] += v[j];
     }
   } else if (g.epi & EPI_SWIGLU) {
     bf16* C = reinterpret_cast<bf16*>(g.C) + (size_t)m * g.ldc + (n >> 1);
     if (full) {
-      uint32_t o[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        o[j] = pack2(silu_f(v[4 * j]) * v[4 * j + 1], silu_f(v[4 * j + 2]) * v[4 * j + 3]);
-      reinterpret_cast<uint4*>(C)[0] = make_uint4(o[0], o[1], o[2], o[3]);
-      reinterpret_cast<uint4*>(C)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+      *reinterpret_cast<uint32_t*>(C) = pack2(silu_f(v[0]) * v[1], silu_f(v[2]) * v[3]);
     } else {
-#pragma unroll
-      for (int j = 0; j < 32; j += 2) if (n + j + 1 < N) C[j >> 1] = f2bf(silu_f(v[j]) * v[j + 1]);
+      if (n + 1 < N) C[0] = f2bf(silu_f(v[0]) * v[1]);
     }
   } else {
     bf16* C = reinterpret_cast<bf16*>(g.C) + (size_t)m * g.ldc + n;
     if (full) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        uint4 o;
-        o.x = pack2(v[j], v[j + 1]); o.y = pack2(v[j + 2], v[j + 3]);
-        o.z = pack2(v[j + 4], v[j + 5]); o.w = pack2(v[j + 6], v[j + 7]);
-        *reinterpret_cast<uint4*>(C + j) = o;
-      }
+      *reinterpret_cast<uint2*>(C) = make_uint2(pack2(v[0], v[1]), pack2(v[2], v[3]));
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (n + j < N) C[j] = f2bf(v[j]);
+      for (int j = 0; j < 4; ++j) if (n + j < N) C[j] = f2bf(v[j]);
+    }
+  }
+}
+
+// Split-k reduction of one tile by the 256 epilogue threads: positions (row, 4 columns) are swept
+// coalesced along the row, U positions x up to KSMAX ranges of loads in flight per thread; the
+// ranges of a position are added in range order.
+template <int U, int KSMAX>
+__device__ __forceinline__ void splitk_reduce(const GView& g, const Item& it, int et, size_t pld) {
+  const int rows = min(TC_BM, g.M - it.m0);
+  const int cols4 = (min(g.bn, g.N - it.n0) + 3) >> 2;
+  const int npos = rows * cols4;
+  const size_t sstride = (size_t)g.tiles_m * TC_BM * pld;
+  const float* p0 = g.partial + (size_t)it.m0 * pld + it.n0;
+  const int ks = g.ksplit;
+  constexpr int STEP = EPI_WARPS * 32;
+  for (int base_pos = et; base_pos < npos; base_pos += STEP * U) {
+    float4 pv[U][KSMAX];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int pos = base_pos + u * STEP;
+      const int r = pos / cols4, c4 = pos - r * cols4;
+#pragma unroll
+      for (int s2 = 0; s2 < KSMAX; ++s2)
+        if (s2 < ks && pos < npos)
+          pv[u][s2] = __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)r * pld + c4 * 4 + s2 * sstride));
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int pos = base_pos + u * STEP;
+      if (pos < npos) {
+        float4 a4 = pv[u][0];
+#pragma unroll
+        for (int s2 = 1; s2 < KSMAX; ++s2)
+          if (s2 < ks) { a4.x += pv[u][s2].x; a4.y += pv[u][s2].y; a4.z += pv[u][s2].z; a4.w += pv[u][s2].w; }
+        const int r = pos / cols4, c4 = pos - r * cols4;
+        epilogue4(g, it.m0 + r, it.n0 + c4 * 4, a4);
+      }
     }
   }
 }
 
 __global__ void __launch_bounds__(N_THREADS, 1)
-gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_tiles, int* __restrict__ status) {
+gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status) {
   extern __shared__ unsigned char smem_dyn[];
   // 1024-byte aligned tile area (128-byte swizzle atoms are 1024 bytes)
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
-  const uint32_t bars = base + STAGES * STAGE_BYTES;
+  unsigned char* stage_out = base_ptr + STAGES * STAGE_BYTES;
+  const uint32_t bars = base + STAGES * STAGE_BYTES + STAGE_OUT_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * STAGE_BYTES + STAGE_OUT_BYTES + 8 * (2 * STAGES + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  volatile int* votes = reinterpret_cast<volatile int*>(tmem_slot + 4);   // one per epilogue warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), EPI_WARPS); }
     *abort_flag = 0;
+    *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -222,25 +325,48 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_til
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
+    if (lane != 0) {
+      // ---------------------------------------------------------- L2 prefetch of residual tiles
+      // The fp32 residual epilogue reads C before it adds to it; these lanes ask L2 for the C tiles of
+      // this CTA's items ahead of time so that those reads do not wait on HBM.
+      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        const GemmGroup& g = groups[find_group_tc(groups, n_groups, item)];
+        if (!(g.epi & EPI_RESID_F32)) continue;
+        const Item it = decode_item(g, item - g.tile_start);
+        if (it.split != g.ksplit - 1) continue;        // once per tile
+        const int ncols = min(g.bn, g.N - it.n0);
+        for (int r = lane - 1; r < TC_BM && it.m0 + r < g.M; r += 31) {
+          const float* rowp = reinterpret_cast<const float*>(g.C) + (size_t)(it.m0 + r) * g.ldc + it.n0;
+          for (int c = 0; c < ncols; c += 32)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + c));
+        }
+      }
+    }
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       uint32_t issued_mask = 0, last_parity = 0;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const GemmGroup* g = groups + find_group_tc(groups, n_groups, tile);
-        const int local = tile - g->tile_start;
-        const int m0 = (local / g->tiles_n) * TC_BM, n0 = (local % g->tiles_n) * TC_BN;
-        tensormap_acquire(&g->tmA);
-        tensormap_acquire(&g->tmW);
-        const int kblocks = (g->K + TC_BK - 1) / TC_BK;
-        for (int kb = 0; kb < kblocks; ++kb) {
+      const GemmGroup* g_prev = nullptr;
+      GroupCache gc;
+      gc.g = nullptr;
+      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+        group_cache(gc, groups, n_groups, item);
+        const GemmGroup* g = gc.g;
+        const Item it = decode_item(gc, item);
+        if (g != g_prev) {                     // the maps were written by a host copy: acquire once per group
+          tensormap_acquire(&g->tmA);
+          tensormap_acquire(&g->tmW);
+          g_prev = g;
+        }
+        const uint32_t bytes = A_BYTES + (uint32_t)gc.bn * TC_BK * 2;
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 1); break; }
-          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          mbar_expect_tx(full_bar(stage), bytes);
           const uint32_t sa = base + stage * STAGE_BYTES;
-          tma_load_2d(sa, &g->tmA, kb * TC_BK, m0, full_bar(stage));
-          tma_load_2d(sa + A_BYTES, &g->tmW, kb * TC_BK, n0, full_bar(stage));
+          tma_load_2d(sa, &g->tmA, kb * TC_BK, it.m0, full_bar(stage));
+          tma_load_2d(sa + A_BYTES, &g->tmW, kb * TC_BK, it.n0, full_bar(stage));
           issued_mask |= 1u << stage;
           last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -262,20 +388,23 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_til
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const GemmGroup* g = groups + find_group_tc(groups, n_groups, tile);
-        const int kblocks = (g->K + TC_BK - 1) / TC_BK;
+      GroupCache gc;
+      gc.g = nullptr;
+      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+        group_cache(gc, groups, n_groups, item);
+        const Item it = decode_item(gc, item);
+        const uint32_t idesc = make_idesc(gc.bn);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 2); break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TC_BN);
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; atomicExch(status, 3); break; }
           tc_fence_after();
           const uint32_t sa = base + stage * STAGE_BYTES;
           const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + A_BYTES);
 #pragma unroll
           for (int k = 0; k < TC_BK / 16; ++k)
-            mma_f16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), (kb > 0 || k > 0) ? 1u : 0u);
+            mma_f16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
           mma_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -286,29 +415,202 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_til
       if (!ok) *abort_flag = 1;
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..9)
+    const int ew = warp - 2;
+    const int et = threadIdx.x - 64;          // 0..255 among the epilogue threads
     const int quarter = warp & 3;             // TMEM lanes 32*quarter .. +31 belong to this warp
+    const int half = ew >> 2;                 // which of the two warps of the quarter: 32-column chunks half, half+2, ...
+    const int row = quarter * 32 + lane;      // row of the tile this thread reads from TMEM
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const GemmGroup& g = groups[find_group_tc(groups, n_groups, tile)];
-      const int local = tile - g.tile_start;
-      const int m0 = (local / g.tiles_n) * TC_BM, n0 = (local % g.tiles_n) * TC_BN;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 4); break; }
-      tc_fence_after();
-      const int m = m0 + quarter * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * TC_BN);
-#pragma unroll 1
-      for (int c = 0; c < TC_BN; c += 32) {
-        if (n0 + c >= g.N) break;              // uniform across the warp
-        uint32_t r[32];
-        tmem_ld32(taddr + (uint32_t)c, r);
-        if (m < g.M) epilogue_row(g, m, n0 + c, r);
+    GView g;
+    int g_end = -1;
+    g.tile_start = 0;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      if (item >= g_end || item < g.tile_start) {
+        g = load_view(groups + find_group_tc(groups, n_groups, item));
+        g_end = g.tile_start + g.tiles_m * g.tiles_n * g.ksplit;
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      const Item it = decode_item(g, item - g.tile_start);
+      bool got = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
+      if (g.ksplit > 1) {
+        // the split path uses block-level barriers among the epilogue warps: leave together
+        if (lane == 0) votes[ew] = got ? 1 : 0;
+        epi_barrier();
+        for (int w = 0; w < EPI_WARPS; ++w) got = got && (votes[w] != 0);
+        epi_barrier();
+      }
+      if (!got) { ok = false; if (lane == 0) atomicExch(status, 4); break; }
+      tc_fence_after();
+      const int m = it.m0 + row;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * ACC_COLS);
+      const bool split = g.ksplit > 1;
+      const size_t pld = (size_t)g.tiles_n * g.bn;                                   // partial row length
+      if (split) {
+        float* part = g.partial + ((size_t)it.split * g.tiles_m * TC_BM + m) * pld + it.n0;
+#pragma unroll 1
+        for (int c = half * 32; c < g.bn; c += 64) {
+          if (it.n0 + c >= g.N) break;           // uniform across the warp
+          uint32_t r[32];
+          tmem_ld32(taddr + (uint32_t)c, r);
+          if (m < g.M) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              __stcg(reinterpret_cast<float4*>(part + c + j),
+                     make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                 __uint_as_float(r[j + 3])));
+          }
+        }
+        // the accumulator is drained: hand it back to the MMA warp
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        // count this k range; the one that arrives last reduces all ranges in order
+        __threadfence();
+        epi_barrier();
+        if (et == 0) {
+          const int old = atomicAdd(g.counters + it.tile, 1);
+          const int last = (old == g.ksplit - 1);
+          if (last) atomicExch(g.counters + it.tile, 0);
+          *last_flag = last;
+        }
+        epi_barrier();
+        const bool last = *last_flag != 0;
+        if (last) {
+          __threadfence();
+          if (g.ksplit <= 2) splitk_reduce<4, 2>(g, it, et, pld);
+          else if (g.ksplit <= 4) splitk_reduce<2, 4>(g, it, et, pld);
+          else splitk_reduce<1, 8>(g, it, et, pld);
+        }
+        epi_barrier();                         // last_flag may be rewritten only after everyone read it
+      } else {
+        // direct epilogue, warp by warp with no block-level barrier.  Warp (quarter, half) owns rows
+        // quarter*32..+31 and the half-th half of the tile's columns, in sub-passes of 64 accumulator
+        // columns (32 for an fp32 residual).  Phase 1: each lane turns its row's chunk into output
+        // values and parks them in the warp's 4 KB staging area (16-byte pieces XOR-swizzled by row);
+        // phase 2: the warp writes the 32 rows out with 128-byte row segments.
+        const bool f32 = (g.epi & EPI_RESID_F32) != 0, swi = (g.epi & EPI_SWIGLU) != 0;
+        const int rows = min(32, g.M - it.m0 - quarter * 32);  // valid rows of this warp (may be <= 0)
+        unsigned char* wst = stage_out + ew * 4096;
+        unsigned char* srow = wst + lane * 128;
+        const int c_end = min((half + 1) * (g.bn >> 1), g.N - it.n0);
+        for (int g0 = half * (g.bn >> 1); g0 < c_end; g0 += 64) {
+#pragma unroll
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int c = g0 + 32 * h2;
+            if (c >= c_end) break;
+            const int n = it.n0 + c;
+            const int acc_valid = min(32, g.N - n);              // valid accumulator columns of this chunk
+            float4 cpre[8];
+            if (f32) {                                           // residual values of this chunk, requested early
+              const float* Cr = reinterpret_cast<const float*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + n;
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const int idx = lane + k * 32, r2 = idx >> 3, col = (idx & 7) << 2;
+                cpre[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r2 < rows && col + 4 <= acc_valid) cpre[k] = *reinterpret_cast<const float4*>(Cr + (size_t)r2 * g.ldc + col);
+              }
+            }
+            uint32_t r32[32];
+            tmem_ld32(taddr + (uint32_t)c, r32);
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r32[j]);
+            if (g.epi & EPI_BIAS) {
+              if (n + 32 <= g.N) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  float bb[8];
+                  unpack8(__ldg(reinterpret_cast<const uint4*>(g.bias + n) + j), bb);
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) v[8 * j + e] += bb[e];
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) if (n + j < g.N) v[j] += bf2f(g.bias[n + j]);
+              }
+            }
+            if (g.epi & EPI_GELU) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+            }
+            if (f32) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k)
+                *reinterpret_cast<float4*>(srow + ((k ^ (lane & 7)) << 4)) =
+                    make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+              __syncwarp();
+              float* C = reinterpret_cast<float*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + n;
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const int idx = lane + k * 32, r2 = idx >> 3, pp = idx & 7, col = pp << 2;
+                if (r2 >= rows || col >= acc_valid) continue;
+                const float4 a = *reinterpret_cast<const float4*>(wst + r2 * 128 + ((pp ^ (r2 & 7)) << 4));
+                float* cp = C + (size_t)r2 * g.ldc + col;
+                if (col + 4 <= acc_valid) {
+                  float4 cv = cpre[k];
+                  cv.x += a.x; cv.y += a.y; cv.z += a.z; cv.w += a.w;
+                  *reinterpret_cast<float4*>(cp) = cv;
+                } else {
+                  const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) if (col + j < acc_valid) cp[j] += av[j];
+                }
+              }
+              __syncwarp();                      // the staging area is reused by the next chunk
+            } else if (swi) {
+#pragma unroll
+              for (int k = 0; k < 2; ++k) {                      // 32 columns -> 16 outputs -> 2 pieces
+                uint4 o;
+                o.x = pack2(silu_f(v[16 * k]) * v[16 * k + 1], silu_f(v[16 * k + 2]) * v[16 * k + 3]);
+                o.y = pack2(silu_f(v[16 * k + 4]) * v[16 * k + 5], silu_f(v[16 * k + 6]) * v[16 * k + 7]);
+                o.z = pack2(silu_f(v[16 * k + 8]) * v[16 * k + 9], silu_f(v[16 * k + 10]) * v[16 * k + 11]);
+                o.w = pack2(silu_f(v[16 * k + 12]) * v[16 * k + 13], silu_f(v[16 * k + 14]) * v[16 * k + 15]);
+                *reinterpret_cast<uint4*>(srow + (((2 * h2 + k) ^ (lane & 7)) << 4)) = o;
+              }
+            } else {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {                      // 32 columns -> 4 pieces
+                uint4 o;
+                o.x = pack2(v[8 * k], v[8 * k + 1]); o.y = pack2(v[8 * k + 2], v[8 * k + 3]);
+                o.z = pack2(v[8 * k + 4], v[8 * k + 5]); o.w = pack2(v[8 * k + 6], v[8 * k + 7]);
+                *reinterpret_cast<uint4*>(srow + (((4 * h2 + k) ^ (lane & 7)) << 4)) = o;
+              }
+            }
+          }
+          if (!f32) {
+            __syncwarp();
+            // write the 32 rows x 64 accumulator columns out with 128-byte (SwiGLU: 64-byte) row segments
+            const int acc_valid = min(64, g.N - it.n0 - g0);
+            const int out_valid = swi ? (acc_valid >> 1) : acc_valid;
+            const int ppr = swi ? 4 : 8;                         // 8-element pieces per staged row
+            bf16* C = reinterpret_cast<bf16*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc +
+                      (swi ? ((it.n0 + g0) >> 1) : (it.n0 + g0));
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const int idx = lane + k * 32;
+              const int r2 = swi ? (idx >> 2) : (idx >> 3), pp = swi ? (idx & 3) : (idx & 7), col = pp << 3;
+              if (idx >= 32 * ppr || r2 >= rows || col >= out_valid) continue;
+              const uint4 a = *reinterpret_cast<const uint4*>(wst + r2 * 128 + ((pp ^ (r2 & 7)) << 4));
+              bf16* cp = C + (size_t)r2 * g.ldc + col;
+              if (col + 8 <= out_valid) {
+                *reinterpret_cast<uint4*>(cp) = a;
+              } else {
+                const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                  if (col + j < out_valid) cp[j] = __ushort_as_bfloat16((unsigned short)(aw[j >> 1] >> ((j & 1) * 16)));
+              }
+            }
+            __syncwarp();                        // the staging area is reused by the next 64 columns
+          }
+        }
+        // the accumulator is drained by this warp: hand it back to the MMA warp
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+      }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
     if (!ok) *abort_flag = 1;
@@ -323,13 +625,42 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_til
 
 }  // namespace
 
-cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_tiles, int* status, int sm_count,
+// Tile width and k-split of a GEMM whose row capacity is rows_cap (fixed when the model is placed,
+// so a request's reduction order never depends on the batch it happens to share).
+void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int* bn, int* ksplit) {
+  auto padded = [&](int b) { return (N + b - 1) / b * b; };
+  const int kblocks = (K + TC_BK - 1) / TC_BK;
+  if (rows_cap <= 0) { *bn = 128; *ksplit = 1; return; }
+  if (rows_cap > 256) {                       // dense: tensor-bound; a 128 x 256 MMA runs at about twice the
+    *bn = (N > 128) ? 256 : 128;              // efficiency of a 128 x 128 one, which outweighs padded columns
+    // ... except for the fp32 residual update, which is bound by its read-modify-write of C: there
+    // padded columns cost more than narrow MMAs
+    if ((epi & EPI_RESID_F32) && padded(128) < padded(256)) *bn = 128;
+    *ksplit = 1;
+    return;
+  }
+  // weight streaming: the widest tile (most W bytes in flight per stage).  Splitting K pays only when
+  // a handful of tiles would each stream a very long K: measured on B200, the fixed cost of a split
+  // item (partials, counter, reduction) exceeds the gain for K < 4096.
+  const int tiles_m = (int)((rows_cap + TC_BM - 1) / TC_BM);
+  *bn = (N > 128) ? 256 : 128;
+  const int tiles = tiles_m * (padded(*bn) / *bn);
+  int ks = 1;
+  if (kblocks >= 64 && tiles * 8 <= sm_count) {
+    ks = kblocks / 16;
+    if (ks > 8) ks = 8;
+    while (ks > 1 && (ks - 1) * ((kblocks + ks - 1) / ks) >= kblocks) --ks;   // no empty range
+  }
+  *ksplit = ks;
+}
+
+cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
                            cudaStream_t st) {
-  if (n_groups == 0 || total_tiles == 0) return cudaSuccess;
+  if (n_groups == 0 || total_items == 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-  gemm_tc_kernel<<<grid, N_THREADS, SMEM_BYTES, st>>>(groups, n_groups, total_tiles, status);
+  const int grid = total_items < sm_count ? total_items : sm_count;
+  gemm_tc_kernel<<<grid, N_THREADS, SMEM_BYTES, st>>>(groups, n_groups, total_items, status);
   return cudaGetLastError();
 }
 

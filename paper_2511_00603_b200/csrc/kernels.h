@@ -16,12 +16,14 @@ void launch_output(const OutputGroup* groups, int n_groups, int max_B, cudaStrea
 constexpr int SIMT_TILE = 64;
 void launch_gemm_simt(const GemmGroup* groups, int n_groups, int total_tiles, cudaStream_t st);
 
-// tcgen05 grouped GEMM, 128 x TC_BN tiles, persistent.  `status` is a device int the kernel
-// sets non-zero if a bounded wait ran out.  Returns the cudaError of the launch configuration.
+// tcgen05 grouped GEMM, 128 x bn tiles (bn = 128 or 256 per group), persistent.  `status` is a
+// device int the kernel sets non-zero if a bounded wait ran out.  total_items = sum over groups of
+// tiles_m * tiles_n * ksplit.  Returns the cudaError of the launch configuration.
 constexpr int TC_BM = 128;
-constexpr int TC_BN = 128;
+constexpr int TC_BN_MAX = 256;
 constexpr int TC_BK = 64;
-cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_tiles, int* status, int sm_count,
+void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int* bn, int* ksplit);
+cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
                            cudaStream_t st);
 
 // Decode attention (split-KV over 256-token chunks) and the combine of the chunk partials.

@@ -67,7 +67,7 @@ class GemmProblem(C.Structure):
 EXPORTS = ["epara_init", "epara_register_model", "epara_submit", "epara_submit_many", "epara_step", "epara_collect",
            "epara_step_profile", "epara_set_profile", "epara_destroy", "epara_strerror", "epara_model_workspace_bytes",
            "epara_dp_group_count", "epara_inter_request_count", "epara_admit_queue", "epara_grouped_gemm",
-           "epara_gemm_scratch_bytes", "epara_decode_attention", "epara_decode_attention_scratch_bytes"]
+           "epara_gemm_scratch_bytes", "epara_gemm_scratch_bytes_for", "epara_decode_attention", "epara_decode_attention_scratch_bytes"]
 
 lib.epara_init.argtypes = [C.POINTER(Config), C.POINTER(C.c_void_p)]
 lib.epara_register_model.argtypes = [C.c_void_p, C.POINTER(ModelDesc), C.POINTER(C.c_int)]
@@ -92,6 +92,8 @@ lib.epara_grouped_gemm.argtypes = [C.c_int, C.c_void_p, C.c_int, C.POINTER(GemmP
                                    C.c_size_t]
 lib.epara_gemm_scratch_bytes.argtypes = [C.c_int]
 lib.epara_gemm_scratch_bytes.restype = C.c_size_t
+lib.epara_gemm_scratch_bytes_for.argtypes = [C.POINTER(GemmProblem), C.c_int]
+lib.epara_gemm_scratch_bytes_for.restype = C.c_size_t
 lib.epara_decode_attention.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                        C.c_int, C.c_void_p, C.c_size_t]
@@ -250,8 +252,7 @@ class Context:
 
 
 # ----------------------------------------------------------------------------- single kernels
-def epara_grouped_gemm(problems: Sequence[Dict], stream_ptr: int, scratch, impl: int = GEMM_TCGEN05, device: int = 0):
-    """problems: dicts with torch tensors A [M, lda], W [N, ldw], C, optional bias, and M, N, K, epilogue."""
+def gemm_problem_array(problems: Sequence[Dict]):
     n = len(problems)
     arr = (GemmProblem * max(n, 1))()
     for i, p in enumerate(problems):
@@ -259,6 +260,17 @@ def epara_grouped_gemm(problems: Sequence[Dict], stream_ptr: int, scratch, impl:
                              p["bias"].data_ptr() if p.get("bias") is not None else None,
                              p["M"], p["N"], p["K"], p["A"].stride(0), p["W"].stride(0), p["C"].stride(0),
                              p.get("epilogue", 0))
+    return arr
+
+
+def epara_gemm_scratch_bytes_for(problems: Sequence[Dict]) -> int:
+    return lib.epara_gemm_scratch_bytes_for(gemm_problem_array(problems), len(problems))
+
+
+def epara_grouped_gemm(problems: Sequence[Dict], stream_ptr: int, scratch, impl: int = GEMM_TCGEN05, device: int = 0):
+    """problems: dicts with torch tensors A [M, lda], W [N, ldw], C, optional bias, and M, N, K, epilogue."""
+    n = len(problems)
+    arr = gemm_problem_array(problems)
     _check(lib.epara_grouped_gemm(device, C.c_void_p(stream_ptr), impl, arr, n, scratch.data_ptr(),
                                   scratch.numel() * scratch.element_size()), "epara_grouped_gemm")
 

@@ -34,6 +34,11 @@ GEMM_CASES = [
     (77, 768, 3072, ("bias", "resid")),
     (0, 64, 64, ()),                    # empty group
     (257, 136, 64, ("gelu", "bias")),   # single k-block, N tail of 8
+    (40, 1024, 1024, ("swiglu",)),      # split along K with a SwiGLU epilogue
+    (256, 2048, 4096, ("resid",)),      # two row tiles, long K
+    (64, 512, 8192, ("bias", "resid")), # few tiles, very long K: split along K with the last-arriver reduction
+    (20, 768, 4096, ("gelu", "bias")),  # split along K, bf16 output
+    (9, 256, 5120, ("swiglu",)),        # split along K, SwiGLU, uneven ranges
 ]
 
 
@@ -64,7 +69,7 @@ def _run_gemm(E, impl, cases, seed=0):
         if "resid" in fl:
             y = C0[:M, :N].double().cpu().numpy() + y
         refs.append(y)
-    scratch = torch.empty(E.lib.epara_gemm_scratch_bytes(len(probs)), dtype=torch.uint8, device=dev)
+    scratch = torch.empty(E.epara_gemm_scratch_bytes_for(probs), dtype=torch.uint8, device=dev)
     E.epara_grouped_gemm(probs, _stream(), scratch, impl=impl)
     torch.cuda.synchronize()
     status = int(scratch[:4].view(torch.int32).item())
