@@ -238,6 +238,33 @@ int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_s
                            int B, int Hq, int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes);
 size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len);
 
+/* Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart
+ * of this call; it exists for how this library gets embedded.)
+ *
+ * Some users of this library run where cudaMalloc is off limits: a serving process whose framework
+ * took the whole device for its own memory pool at start-up, so that a driver allocation now fails
+ * or forces the pool to shrink; or a latency-critical loop in which the implicit device-wide
+ * synchronisation of cudaMalloc/cudaFree would stall every stream.  Such callers cannot provide the
+ * scratch buffer epara_decode_attention asks for.  This variant takes the same inputs and outputs
+ * and keeps its scratch (request table and split-KV partials) in an array that is part of the
+ * library image: EPARA_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the library,
+ * held until the process exits.  It calls no cudaMalloc, cudaFree or any allocating routine.
+ *
+ * Same kernels, same results as epara_decode_attention.  Arguments as there, minus scratch.
+ * Returns EPARA_E_RESOURCE when 256 + roundup256(16 B) + B*Hq*ceil(max_len/256)*(hd+2)*4 bytes exceed
+ * EPARA_STATIC_SCRATCH_BYTES (nothing is launched), INVALID / UNSUPPORTED / CUDA as the other entry.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and caches
+ * it; make that first call outside any stream capture.  All calls on a device share the one array,
+ * which keeps whatever the previous call left in it (nothing needs to start at zero: every byte
+ * that is read is written first by the same call).  Two calls whose kernels may overlap on the GPU
+ * -- different streams without an ordering between them -- race on that array; order them. */
+#define EPARA_STATIC_SCRATCH_BYTES (8u << 20)
+int epara_decode_attention_static(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
+                                  const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out,
+                                  int B, int Hq, int Hkv, int hd, int max_len);
+size_t epara_static_scratch_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -9,6 +9,9 @@
 // kernel merges the chunks in order.
 //
 // Encoder (ViT): full bidirectional attention of T tokens per (image, head).
+#include <cstring>
+
+#include "../../include/epara.h"
 #include "common.cuh"
 #include "kernels.h"
 
@@ -398,3 +401,57 @@ cudaError_t launch_attn_encoder(const AttnEncGroup* groups, int n_groups, int to
 }
 
 }  // namespace epara
+
+// ------------------------------------------------------------------ decode attention without caller scratch
+// Scratch of epara_decode_attention_static: one array per GPU that loads this library, held until
+// the process exits.  Host code may not hand `g_static_scratch` itself to a kernel (on the host the
+// name is only a stand-in for the symbol); the device address is looked up once per device below.
+namespace {
+constexpr size_t STATIC_SCRATCH_BYTES = EPARA_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+constexpr int MAX_DEVICES = 64;
+unsigned char* g_static_ptr[MAX_DEVICES] = {nullptr};
+}  // namespace
+
+extern "C" int epara_decode_attention_static(int device, void* cuda_stream, const void* q, int q_stride,
+                                             const void* kv_layer, const int32_t* kv_lens, const int32_t* tables,
+                                             int table_stride, void* out, int B, int Hq, int Hkv, int hd, int max_len) {
+  using namespace epara;
+  if (!q || !kv_layer || !kv_lens || !tables || !out || B < 0 || Hkv <= 0 || Hq <= 0 || Hq % Hkv || max_len <= 0 || hd <= 0)
+    return EPARA_E_INVALID;
+  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(kv_layer) & 15) || (q_stride % 8))
+    return EPARA_E_INVALID;
+  if (device < 0 || device >= MAX_DEVICES) return EPARA_E_INVALID;
+  const int chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK;
+  const size_t req_bytes = ((size_t)B * sizeof(AttnReq) + 255) / 256 * 256;
+  const size_t need = 256 + req_bytes + (size_t)B * Hq * chunks * (hd + 2) * sizeof(float);
+  if (need > STATIC_SCRATCH_BYTES) return EPARA_E_RESOURCE;   // problem too large for the built-in scratch
+  if (B == 0) return EPARA_OK;
+  if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
+  if (!g_static_ptr[device]) {
+    // first call on this device: resolve the device address of the array (this device is current)
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return EPARA_E_CUDA;
+    g_static_ptr[device] = static_cast<unsigned char*>(p);
+  }
+  unsigned char* s = g_static_ptr[device];
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  AttnDecGroup g;
+  memset(&g, 0, sizeof(g));
+  AttnReq* reqs = reinterpret_cast<AttnReq*>(s + 256);
+  g.q = (const bf16*)q; g.q_stride = q_stride; g.kv_layer = (const bf16*)kv_layer; g.reqs = reqs; g.out = (bf16*)out;
+  g.partial = reinterpret_cast<float*>(s + 256 + req_bytes);
+  g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = chunks; g.req_start = 0;
+  // Nothing in the scratch has to start at zero: the descriptor and the request table are rewritten
+  // here, and every partial the combine kernel reads is written by the decode kernel of this call.
+  if (cudaMemcpyAsync(s, &g, sizeof(g), cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
+  launch_attn_fill_reqs(reqs, kv_lens, tables, table_stride, B, st);
+  cudaError_t e = launch_attn_decode(reinterpret_cast<const AttnDecGroup*>(s), 1, B, Hkv, chunks, hd, Hq / Hkv, st);
+  if (e == cudaErrorInvalidValue) return EPARA_E_UNSUPPORTED;
+  if (e != cudaSuccess) return EPARA_E_CUDA;
+  e = launch_attn_combine(reinterpret_cast<const AttnDecGroup*>(s), 1, B, Hq, hd, st);
+  return e == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
+}
+
+extern "C" size_t epara_static_scratch_bytes(void) { return STATIC_SCRATCH_BYTES; }
+

@@ -67,7 +67,8 @@ class GemmProblem(C.Structure):
 EXPORTS = ["epara_init", "epara_register_model", "epara_submit", "epara_submit_many", "epara_step", "epara_collect",
            "epara_step_profile", "epara_set_profile", "epara_destroy", "epara_strerror", "epara_model_workspace_bytes",
            "epara_dp_group_count", "epara_inter_request_count", "epara_admit_queue", "epara_grouped_gemm",
-           "epara_gemm_scratch_bytes", "epara_gemm_scratch_bytes_for", "epara_decode_attention", "epara_decode_attention_scratch_bytes"]
+           "epara_gemm_scratch_bytes", "epara_gemm_scratch_bytes_for", "epara_decode_attention", "epara_decode_attention_scratch_bytes",
+           "epara_decode_attention_static", "epara_static_scratch_bytes"]
 
 lib.epara_init.argtypes = [C.POINTER(Config), C.POINTER(C.c_void_p)]
 lib.epara_register_model.argtypes = [C.c_void_p, C.POINTER(ModelDesc), C.POINTER(C.c_int)]
@@ -99,6 +100,13 @@ lib.epara_decode_attention.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int,
                                        C.c_int, C.c_void_p, C.c_size_t]
 lib.epara_decode_attention_scratch_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
 lib.epara_decode_attention_scratch_bytes.restype = C.c_size_t
+
+
+lib.epara_decode_attention_static.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+                                              C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
+                                              C.c_int]
+lib.epara_static_scratch_bytes.argtypes = []
+lib.epara_static_scratch_bytes.restype = C.c_size_t
 
 
 class EparaError(RuntimeError):
@@ -282,3 +290,14 @@ def epara_decode_attention(q, kv_layer, kv_lens, tables, out, Hq: int, Hkv: int,
                                       kv_lens.data_ptr(), tables.data_ptr(), tables.stride(0), out.data_ptr(), B, Hq,
                                       Hkv, hd, max_len, scratch.data_ptr(),
                                       scratch.numel() * scratch.element_size()), "epara_decode_attention")
+
+
+def epara_decode_attention_static(q, kv_layer, kv_lens, tables, out, Hq: int, Hkv: int, hd: int, max_len: int,
+                                  stream_ptr: int, device: int = 0):
+    """Decode attention for callers that must not allocate: same arguments as epara_decode_attention
+    without the scratch tensor (the library's built-in per-GPU array is used instead)."""
+    B = q.shape[0]
+    _check(lib.epara_decode_attention_static(device, C.c_void_p(stream_ptr), q.data_ptr(), q.stride(0),
+                                             kv_layer.data_ptr(), kv_lens.data_ptr(), tables.data_ptr(),
+                                             tables.stride(0), out.data_ptr(), B, Hq, Hkv, hd, max_len),
+           "epara_decode_attention_static")
