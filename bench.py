@@ -313,12 +313,10 @@ def run_gpu(args):
     # per-kind device time of the last timed step (every step launches the same kernels)
     prof = srv.ctx.epara_step_profile()
     srv.ctx.epara_set_profile(False)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    from paper_2511_00603_b200 import dp
+    value = dp.whole_job_throughput(n_req * args.steps, ms_total, device=dev)   # all ranks' requests / slowest rank
+    ms_total = world * n_req * args.steps / value * 1e3
     ms_step = ms_total / args.steps
-    value = world * n_req * args.steps / (ms_total / 1e3)
 
     # ---- unprofiled repeat (shows what the event bracketing costs) ----
     barrier()
