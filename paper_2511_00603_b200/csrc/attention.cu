@@ -167,6 +167,201 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __
   }
 }
 
+// Tensor-core variant for hd 64 / 128.  Same work split (chunk, kv head, request; 4 warps, warp w
+// takes pages w, w+4, w+8, w+12 of the chunk) and the same partial format, but the pages are
+// brought into shared memory with 16-byte cp.async copies -- all of a warp's pages are in flight
+// at once and no registers are tied up by loads -- and Q K^T and P V run on mma.sync m16n8k16
+// with the G query heads of the kv head as the first G rows of the 16-row A operand.  Rows of a
+// staged tile are 128-byte segments whose 16-byte pieces are XOR-swizzled by the token index, so
+// ldmatrix reads are free of bank conflicts.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void mma_bf16_m16n8k16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t* r, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t* r, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+template <int HD, int G, int NSLOT>
+__global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup* __restrict__ groups, int n_groups) {
+  constexpr int ROWB = HD * 2;              // bytes per token row
+  constexpr int TILE = 16 * ROWB;           // bytes per (K or V) page tile
+  constexpr int CPR = HD / 8;               // 16-byte pieces per row
+  constexpr int KS = HD / 16;               // k-steps of Q K^T
+  constexpr float LOG2E = 1.4426950408889634f;
+  extern __shared__ __align__(128) unsigned char dsm[];
+
+  int gi = 0;
+  for (int i = 1; i < n_groups; ++i) if ((int)blockIdx.z >= groups[i].req_start) gi = i;
+  const AttnDecGroup& g = groups[gi];
+  const int b = blockIdx.z - g.req_start;
+  const int kvh = blockIdx.y;
+  if (kvh >= g.Hkv) return;
+  const AttnReq rq = g.reqs[b];
+  const int chunk = blockIdx.x;
+  const int t_begin = chunk * ATTN_CHUNK;
+  if (t_begin >= rq.len) return;
+  const int t_end = min(rq.len, t_begin + ATTN_CHUNK);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gq = lane >> 2, tq = lane & 3;
+  const int Hkv = g.Hkv;
+  const bf16* kv_layer = g.kv_layer;
+
+  // ---- issue all copies of this warp's pages (up to 4), one commit group per page
+  unsigned char* wsm = dsm + warp * (NSLOT * 2 * TILE);
+  const uint32_t wsm_u = (uint32_t)__cvta_generic_to_shared(wsm);
+  const int page_begin = t_begin / 16, page_end = (t_end + 15) / 16;
+  // page i of this warp goes to slot i % NSLOT; one commit group per page (empty past the end)
+  auto issue = [&](int i) {
+    const int pg = page_begin + warp + 4 * i;
+    if (i < 4 && pg < page_end) {
+      const int page = rq.table[pg];
+      const unsigned char* kt = reinterpret_cast<const unsigned char*>(kv_layer + (((size_t)page * 2 + 0) * Hkv + kvh) * 16 * HD);
+      const unsigned char* vt = reinterpret_cast<const unsigned char*>(kv_layer + (((size_t)page * 2 + 1) * Hkv + kvh) * 16 * HD);
+      const uint32_t kd = wsm_u + (i % NSLOT) * 2 * TILE, vd = kd + TILE;
+#pragma unroll
+      for (int j = 0; j < (16 * CPR) / 32; ++j) {
+        const int piece = j * 32 + lane, r = piece / CPR, c = piece % CPR;
+        const uint32_t off = r * ROWB + (c & ~7) * 16 + (((c & 7) ^ (r & 7)) << 4);
+        cp_async16(kd + off, kt + piece * 16);
+        cp_async16(vd + off, vt + piece * 16);
+      }
+    }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int i = 0; i < NSLOT; ++i) issue(i);
+
+  // ---- Q fragments: rows 0..G-1 of the A operand are the query heads of this kv head
+  uint32_t qa[KS][4];
+  {
+    const bf16* qrow = g.q + (size_t)b * g.q_stride + (size_t)(kvh * G + gq) * HD;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      qa[ks][0] = (gq < G) ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * tq) : 0u;
+      qa[ks][2] = (gq < G) ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * tq) : 0u;
+      qa[ks][1] = 0u;
+      qa[ks][3] = 0u;
+    }
+  }
+  const float scale = LOG2E * rsqrtf((float)HD);
+  float o[HD / 8][4];
+#pragma unroll
+  for (int n = 0; n < HD / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m_run = -1e30f, l_run = 0.f;
+  const int lm_row = lane & 7, lm_mat = lane >> 3;
+
+  auto process = [&](int i) {
+    const int pg = page_begin + warp + 4 * i;
+    if (pg >= page_end) return;
+    const uint32_t kd = wsm_u + (i % NSLOT) * 2 * TILE, vd = kd + TILE;
+    const int tok0 = pg * 16;
+    if (tok0 + 16 > t_end) {
+      // slots past the length may hold anything (NaN included): zero those V rows
+      const int valid = t_end - tok0;
+      for (int piece = lane; piece < 16 * CPR; piece += 32) {
+        const int r = piece / CPR, c = piece % CPR;
+        if (r >= valid)
+          *reinterpret_cast<uint4*>(wsm + (i % NSLOT) * 2 * TILE + TILE + r * ROWB + (c & ~7) * 16 + (((c & 7) ^ (r & 7)) << 4)) =
+              make_uint4(0, 0, 0, 0);
+      }
+      __syncwarp();
+    }
+    // S = Q K^T for 16 tokens: two 8-token tiles
+    float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const int r = (lm_mat >> 1) * 8 + lm_row, c = ks * 2 + (lm_mat & 1);
+      uint32_t kr[4];
+      ldsm_x4(kr, kd + r * ROWB + (c & ~7) * 16 + (((c & 7) ^ (r & 7)) << 4));
+      mma_bf16_m16n8k16(sc[0], qa[ks], kr[0], kr[1]);
+      mma_bf16_m16n8k16(sc[1], qa[ks], kr[2], kr[3]);
+    }
+    // row gq of the tile: tokens tok0 + j*8 + 2*tq (+1)
+    float s[4];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int t0 = tok0 + j * 8 + 2 * tq;
+      s[2 * j] = (t0 < t_end) ? sc[j][0] * scale : -INFINITY;
+      s[2 * j + 1] = (t0 + 1 < t_end) ? sc[j][1] * scale : -INFINITY;
+    }
+    float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float mn = fmaxf(m_run, mx);
+    const float resc = exp2f(m_run - mn);
+    m_run = mn;
+    l_run *= resc;
+#pragma unroll
+    for (int n = 0; n < HD / 8; ++n) { o[n][0] *= resc; o[n][1] *= resc; }
+    const float p0 = exp2f(s[0] - mn), p1 = exp2f(s[1] - mn), p2 = exp2f(s[2] - mn), p3 = exp2f(s[3] - mn);
+    l_run += (p0 + p1) + (p2 + p3);
+    uint32_t pa[4];
+    pa[0] = pack2(p0, p1); pa[1] = 0u; pa[2] = pack2(p2, p3); pa[3] = 0u;
+    // O += P V
+#pragma unroll
+    for (int np = 0; np < HD / 16; ++np) {
+      const int r = (lm_mat & 1) * 8 + lm_row, c = 2 * np + (lm_mat >> 1);
+      uint32_t vr[4];
+      ldsm_x4_trans(vr, vd + r * ROWB + (c & ~7) * 16 + (((c & 7) ^ (r & 7)) << 4));
+      mma_bf16_m16n8k16(o[2 * np], pa, vr[0], vr[1]);
+      mma_bf16_m16n8k16(o[2 * np + 1], pa, vr[2], vr[3]);
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    cp_async_wait<NSLOT - 1>();              // page i has landed (one group is committed per step)
+    __syncwarp();
+    process(i);
+    __syncwarp();                            // the slot is free again
+    issue(i + NSLOT);
+  }
+
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+
+  // ---- merge the 4 warps through shared memory, in warp order (same layout as the SIMT kernel)
+  __shared__ float sm_m[4][G], sm_l[4][G], sm_o[4][G][HD];
+  if (gq < G) {
+    if (tq == 0) { sm_m[warp][gq] = m_run; sm_l[warp][gq] = l_run; }
+#pragma unroll
+    for (int n = 0; n < HD / 8; ++n) {
+      sm_o[warp][gq][n * 8 + 2 * tq] = o[n][0];
+      sm_o[warp][gq][n * 8 + 2 * tq + 1] = o[n][1];
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < G * HD; idx += 128) {
+    const int h = idx / HD, e = idx % HD;
+    float mm = sm_m[0][h];
+#pragma unroll
+    for (int w = 1; w < 4; ++w) mm = fmaxf(mm, sm_m[w][h]);
+    float ll = 0.f, oo = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float a = exp2f(sm_m[w][h] - mm);
+      ll += sm_l[w][h] * a;
+      oo += sm_o[w][h][e] * a;
+    }
+    float* dst = g.partial + (((size_t)b * g.Hq + (kvh * G + h)) * g.max_chunks + chunk) * (HD + 2);
+    dst[2 + e] = oo;
+    if (e == 0) { dst[0] = mm; dst[1] = ll; }
+  }
+}
+
 // One block per (query head, request): merges the chunk partials in chunk order.
 __global__ void attn_combine_kernel(const AttnDecGroup* __restrict__ groups, int n_groups) {
   int gi = 0;
@@ -192,6 +387,17 @@ __global__ void attn_combine_kernel(const AttnDecGroup* __restrict__ groups, int
 }
 
 template <int HD, int G>
+static cudaError_t launch_dec_mma(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_chunks,
+                                  cudaStream_t st) {
+  constexpr int NSLOT = 2;                           // pages in flight per warp
+  constexpr int SMEM = 4 * NSLOT * 2 * 16 * HD * 2;  // 4 warps x NSLOT pages x (K + V) tiles
+  cudaError_t e = cudaFuncSetAttribute(attn_decode_mma_kernel<HD, G, NSLOT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e != cudaSuccess) return e;
+  attn_decode_mma_kernel<HD, G, NSLOT><<<dim3(max_chunks, max_Hkv, total_B), 128, SMEM, st>>>(groups, n_groups);
+  return cudaGetLastError();
+}
+
+template <int HD, int G>
 static cudaError_t launch_dec(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_chunks,
                               cudaStream_t st) {
   attn_decode_kernel<HD, G><<<dim3(max_chunks, max_Hkv, total_B), 128, 0, st>>>(groups, n_groups);
@@ -203,8 +409,10 @@ cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int tot
   if (n_groups == 0 || total_B == 0) return cudaSuccess;
   if (total_B > 65535 || max_Hkv > 65535) return cudaErrorInvalidValue;
 #define EPARA_DEC(HD_, G_) if (hd == HD_ && gqa == G_) return launch_dec<HD_, G_>(groups, n_groups, total_B, max_Hkv, max_chunks, st);
-  EPARA_DEC(64, 1) EPARA_DEC(64, 2) EPARA_DEC(64, 4) EPARA_DEC(64, 8)
-  EPARA_DEC(128, 1) EPARA_DEC(128, 2) EPARA_DEC(128, 4) EPARA_DEC(128, 8)
+#define EPARA_DEC_MMA(HD_, G_) if (hd == HD_ && gqa == G_) return launch_dec_mma<HD_, G_>(groups, n_groups, total_B, max_Hkv, max_chunks, st);
+  EPARA_DEC_MMA(64, 1) EPARA_DEC_MMA(64, 2) EPARA_DEC_MMA(64, 4) EPARA_DEC_MMA(64, 8)
+  EPARA_DEC_MMA(128, 1) EPARA_DEC_MMA(128, 2) EPARA_DEC_MMA(128, 4) EPARA_DEC_MMA(128, 8)
+#undef EPARA_DEC_MMA
   EPARA_DEC(16, 1) EPARA_DEC(16, 2) EPARA_DEC(16, 4)
   EPARA_DEC(32, 1) EPARA_DEC(32, 2) EPARA_DEC(32, 4)
 #undef EPARA_DEC
