@@ -309,8 +309,13 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
     for (int n = 0; n < HD / 8; ++n) { o[n][0] *= resc; o[n][1] *= resc; }
     const float p0 = exp2f(s[0] - mn), p1 = exp2f(s[1] - mn), p2 = exp2f(s[2] - mn), p3 = exp2f(s[3] - mn);
     l_run += (p0 + p1) + (p2 + p3);
-    uint32_t pa[4];
+    // P enters the tensor core as bf16; to keep fp32-level accuracy it is split into a bf16 head
+    // and a bf16 remainder (p = hi + lo up to 2^-17 relative), and P V is two MMAs per tile
+    uint32_t pa[4], pb[4];
     pa[0] = pack2(p0, p1); pa[1] = 0u; pa[2] = pack2(p2, p3); pa[3] = 0u;
+    pb[0] = pack2(p0 - __uint_as_float(pa[0] << 16), p1 - __uint_as_float(pa[0] & 0xffff0000u));
+    pb[2] = pack2(p2 - __uint_as_float(pa[2] << 16), p3 - __uint_as_float(pa[2] & 0xffff0000u));
+    pb[1] = 0u; pb[3] = 0u;
     // O += P V
 #pragma unroll
     for (int np = 0; np < HD / 16; ++np) {
@@ -319,6 +324,8 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
       ldsm_x4_trans(vr, vd + r * ROWB + (c & ~7) * 16 + (((c & 7) ^ (r & 7)) << 4));
       mma_bf16_m16n8k16(o[2 * np], pa, vr[0], vr[1]);
       mma_bf16_m16n8k16(o[2 * np + 1], pa, vr[2], vr[3]);
+      mma_bf16_m16n8k16(o[2 * np], pb, vr[0], vr[1]);
+      mma_bf16_m16n8k16(o[2 * np + 1], pb, vr[2], vr[3]);
     }
   };
 #pragma unroll
