@@ -185,6 +185,64 @@ def test_config3_shapes_shallow_strict(mods, n_layers):
     _decoder_case(E, server, p, B=5, lo=128, hi=4096, seed=22, n_check=3, deep=n_layers > 1)
 
 
+def test_config5_8b_layer_shapes_shallow_strict(mods):
+    """The 8B decoder's layer shapes (d 4096, 32/8 heads of 128, FFN 14336, vocab 32000) at depth 1,
+    KV lengths U[512, 8192]: strict element-wise tolerance."""
+    E, server = mods
+    p = synth.make_decoder(d=4096, n_layers=1, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=14336, vocab=32000,
+                           seed=4, device=DEV)
+    _decoder_case(E, server, p, B=3, lo=512, hi=8192, seed=41, n_check=2)
+
+
+def test_mixed_bench_workload_sampled_parity(mods):
+    """The benchmark's own configuration (8 co-resident instances, full batches, one step): sampled
+    requests of every instance against the oracle, plus properties that hold for all of them."""
+    E, server = mods
+    from paper_2511_00603_b200 import workloads as W
+    srv = server.Server(workspace_bytes=3 << 30)
+    insts = W.build_mixed(srv, seed=3)
+    pools0 = {i: synth.to_bits(inst.kv_pool) for i, inst in enumerate(insts) if inst.kind == "decoder" and inst.n_req <= 8}
+    for inst in insts:
+        inst.submit_all(srv.ctx)
+    info = srv.ctx.epara_step(torch.cuda.current_stream().cuda_stream, 0)
+    torch.cuda.synchronize()
+    assert info.admitted[0] == 12 and info.admitted[1] == 1280
+    for k, inst in enumerate(insts):
+        for t in inst.tickets:
+            assert srv.ctx.epara_collect(t)[0] == E.OK
+        lg = inst.logits.float()
+        assert torch.isfinite(lg).all()
+        # the argmax kernel agrees with its own logits for every request of the instance
+        assert torch.equal(inst.argmax.long(), lg.argmax(dim=1))
+        v = synth.bits_view({kk: inst.p[kk] for kk in inst.p if kk != "packed_layers"})
+        if inst.kind == "mlp":
+            for i in (0, inst.n_req // 2, inst.n_req - 1):
+                ref, _ = O.mlp_forward(synth.to_bits(inst.x[i]), v["W"], v["b"])
+                assert_close(inst.logits[i], ref, what=f"instance {k} MLP request {i}")
+        elif inst.kind == "vit":
+            for i in (0, inst.n_req - 1):
+                ref, _, _ = O.vit_forward(synth.to_bits(inst.x[i]), v)
+                assert_close(inst.logits[i], ref, what=f"instance {k} ViT-S image {i}")
+                check_argmax(int(inst.argmax[i]), inst.logits[i], ref)
+        elif k in pools0:
+            i = 0                                     # latency-sensitive decoder: its cache copy fits the host
+            pb = pools0[k]
+            tb = inst.tables[i]
+            ra = O.decoder_step(int(inst.tokens[i]), int(inst.lens[i]), tb, lambda l, pg: pb[l, pg], v)
+            rb = O.decoder_step(int(inst.tokens[i]), int(inst.lens[i]), tb, lambda l, pg: pb[l, pg], v, round_bf16=True)
+            assert_parity(inst.logits[i], ra["logits"], rb["logits"], what=f"instance {k} decoder request {i}", deep=True)
+        else:
+            # frequency-sensitive decoder (17 GB cache): the oracle reads one request's pages from the device
+            i = int(np.argmin(inst.lens))
+            tb = inst.tables[i]
+            fetch = lambda l, pg: synth.to_bits(inst.kv_pool[l, pg])
+            # the step appended this request's k, v at slot L: mask it out by giving the oracle L tokens only
+            rb = O.decoder_step(int(inst.tokens[i]), int(inst.lens[i]), tb, fetch, v, round_bf16=True)
+            ra = O.decoder_step(int(inst.tokens[i]), int(inst.lens[i]), tb, fetch, v)
+            assert_parity(inst.logits[i], ra["logits"], rb["logits"], what=f"instance {k} decoder request {i}", deep=True)
+    srv.close()
+
+
 def test_decoder_batch_invariance_and_mixed_models(mods):
     """One step holding an MLP, a ViT and a decoder: every request equals the oracle, and the decoder
     request's bits do not depend on the co-resident models (MT)."""
