@@ -433,6 +433,19 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
         g_end = g.tile_start + g.tiles_m * g.tiles_n * g.ksplit;
       }
       const Item it = decode_item(g, item - g.tile_start);
+      // bias of this warp's column half, 4 values per lane, requested before the accumulator is awaited
+      uint2 bias_reg = make_uint2(0u, 0u);
+      if (g.epi & EPI_BIAS) {
+        const int nb = it.n0 + half * (g.bn >> 1) + lane * 4;
+        if (nb + 4 <= g.N) {
+          bias_reg = __ldg(reinterpret_cast<const uint2*>(g.bias + nb));
+        } else {
+          unsigned short e[4] = {0, 0, 0, 0};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) if (nb + j < g.N) e[j] = __bfloat16_as_ushort(g.bias[nb + j]);
+          bias_reg = make_uint2((uint32_t)e[0] | ((uint32_t)e[1] << 16), (uint32_t)e[2] | ((uint32_t)e[3] << 16));
+        }
+      }
       bool got = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
       if (g.ksplit > 1) {
         // the split path uses block-level barriers among the epilogue warps: leave together
@@ -518,17 +531,13 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r32[j]);
             if (g.epi & EPI_BIAS) {
-              if (n + 32 <= g.N) {
+              // the 32 bias values of this chunk sit in 8 consecutive lanes of bias_reg (zero past N)
+              const int lane0 = (c - half * (g.bn >> 1)) >> 2;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  float bb[8];
-                  unpack8(__ldg(reinterpret_cast<const uint4*>(g.bias + n) + j), bb);
-#pragma unroll
-                  for (int e = 0; e < 8; ++e) v[8 * j + e] += bb[e];
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) if (n + j < g.N) v[j] += bf2f(g.bias[n + j]);
+              for (int jj = 0; jj < 16; ++jj) {
+                const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
+                v[2 * jj] += __uint_as_float(w << 16);
+                v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
               }
             }
             if (g.epi & EPI_GELU) {
