@@ -445,12 +445,12 @@ void launch_attn_fill_reqs(AttnReq* reqs, const int32_t* kv_lens, const int32_t*
 }
 
 // ------------------------------------------------------------------ encoder attention
-// One block per (image, head, block of up to 256 query rows); one warp per 16 query rows.
+// One block per (image, head, block of up to 112 query rows); one warp per 16 query rows.
 // K and V of the head are staged once in shared memory (bf16, rows padded to 72 elements so
 // that ldmatrix rows fall in distinct banks); each warp runs a flash-style loop over 64-key
 // blocks with mma.sync m16n8k16 (bf16 in, fp32 accumulate): S = Q K^T, online softmax in the
 // exp2 domain, O += P V.  Keys beyond T are masked; their padded rows are zero.
-constexpr int ENC_ROWS = 256;      // query rows per block
+constexpr int ENC_ROWS = 112;      // query rows per block (7 warps): two blocks share an SM
 constexpr int ENC_LD = 72;         // padded row length of K and V in shared memory
 int attn_encoder_q_blocks(int T) { return (T + ENC_ROWS - 1) / ENC_ROWS; }
 static int enc_key_pad(int T) { return (T + 63) / 64 * 64; }
@@ -469,7 +469,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, uint32_t addr) {
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
 
-__global__ void __launch_bounds__(512, 1) attn_encoder_kernel(const AttnEncGroup* __restrict__ groups, int n_groups) {
+__global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const AttnEncGroup* __restrict__ groups, int n_groups) {
   constexpr int HD = 64;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   int gi = 0;

@@ -114,10 +114,80 @@ __device__ __forceinline__ void norm_row(const NormGroup& g, int row, float* red
   }
 }
 
+// Narrow rows (d <= 512): one warp takes ROWS rows at once, all their loads in flight together.
+constexpr int NORM_NARROW_D = 512;
+constexpr int NORM_NARROW_ROWS = 4;
+__device__ __forceinline__ void norm_rows_narrow(const NormGroup& g, int row0) {
+  const int lane = threadIdx.x & 31;
+  const int nvec = g.d >> 2;
+  float4 v[NORM_NARROW_ROWS][4];
+#pragma unroll
+  for (int r = 0; r < NORM_NARROW_ROWS; ++r) {
+    const float4* x = reinterpret_cast<const float4*>(g.x + (size_t)(row0 + r) * g.x_stride);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = lane + i * 32;
+      v[r][i] = (row0 + r < g.M && c < nvec) ? x[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  const float inv_d = 1.0f / (float)g.d;
+  const uint2* gm = reinterpret_cast<const uint2*>(g.gamma);
+  const uint2* bt = reinterpret_cast<const uint2*>(g.beta);
+#pragma unroll
+  for (int r = 0; r < NORM_NARROW_ROWS; ++r) {
+    if (row0 + r >= g.M) break;                  // uniform across the warp
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      s += (g.kind == NORM_LN) ? (v[r][i].x + v[r][i].y) + (v[r][i].z + v[r][i].w)
+                               : (v[r][i].x * v[r][i].x + v[r][i].y * v[r][i].y) + (v[r][i].z * v[r][i].z + v[r][i].w * v[r][i].w);
+    s = warp_sum(s);
+    float mean = 0.f, rstd;
+    if (g.kind == NORM_LN) {
+      mean = s * inv_d;
+      float q = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (lane + i * 32 < nvec) {
+          const float a = v[r][i].x - mean, b = v[r][i].y - mean, cc = v[r][i].z - mean, dd = v[r][i].w - mean;
+          q += (a * a + b * b) + (cc * cc + dd * dd);
+        }
+      }
+      q = warp_sum(q);
+      rstd = 1.0f / sqrtf(q * inv_d + g.eps);
+    } else {
+      rstd = 1.0f / sqrtf(s * inv_d + g.eps);
+    }
+    uint2* y = reinterpret_cast<uint2*>(g.y + (size_t)(row0 + r) * g.d);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = lane + i * 32;
+      if (c < nvec) {
+        const uint2 gg = __ldg(gm + c);
+        const float ga[4] = {__uint_as_float(gg.x << 16), __uint_as_float(gg.x & 0xffff0000u),
+                             __uint_as_float(gg.y << 16), __uint_as_float(gg.y & 0xffff0000u)};
+        float be[4] = {0.f, 0.f, 0.f, 0.f};
+        if (g.kind == NORM_LN) {
+          const uint2 bb = __ldg(bt + c);
+          be[0] = __uint_as_float(bb.x << 16); be[1] = __uint_as_float(bb.x & 0xffff0000u);
+          be[2] = __uint_as_float(bb.y << 16); be[3] = __uint_as_float(bb.y & 0xffff0000u);
+        }
+        uint2 o;
+        o.x = pack2((v[r][i].x - mean) * rstd * ga[0] + be[0], (v[r][i].y - mean) * rstd * ga[1] + be[1]);
+        o.y = pack2((v[r][i].z - mean) * rstd * ga[2] + be[2], (v[r][i].w - mean) * rstd * ga[3] + be[3]);
+        y[c] = o;
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(NORM_THREADS) norm_kernel(const NormGroup* __restrict__ groups) {
   __shared__ float red[32];
   const NormGroup g = groups[blockIdx.y];
-  if (g.d <= NORM_WARP_D) {
+  if (g.d <= NORM_NARROW_D) {
+    const int row0 = (blockIdx.x * (NORM_THREADS / 32) + (threadIdx.x >> 5)) * NORM_NARROW_ROWS;
+    if (row0 < g.M) norm_rows_narrow(g, row0);
+  } else if (g.d <= NORM_WARP_D) {
     const int row = blockIdx.x * (NORM_THREADS / 32) + (threadIdx.x >> 5);
     if (row < g.M) norm_row<true>(g, row, red);
   } else {
@@ -126,7 +196,11 @@ __global__ void __launch_bounds__(NORM_THREADS) norm_kernel(const NormGroup* __r
 }
 
 // Blocks a group of M rows of width d needs.
-int norm_blocks(int M, int d) { return d <= NORM_WARP_D ? (M + NORM_THREADS / 32 - 1) / (NORM_THREADS / 32) : M; }
+int norm_blocks(int M, int d) {
+  const int wpb = NORM_THREADS / 32;
+  if (d <= NORM_NARROW_D) return (M + wpb * NORM_NARROW_ROWS - 1) / (wpb * NORM_NARROW_ROWS);
+  return d <= NORM_WARP_D ? (M + wpb - 1) / wpb : M;
+}
 
 void launch_norm(const NormGroup* groups, int n_groups, int max_blocks, cudaStream_t st) {
   if (n_groups == 0 || max_blocks == 0) return;
