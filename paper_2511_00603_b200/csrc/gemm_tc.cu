@@ -10,8 +10,8 @@
 //   warp 1 (one lane)  MMA issuer: tcgen05.mma (M 128, N bn, K 16) from shared memory into one
 //                      of two TMEM accumulators (256 columns each), releasing stages with
 //                      tcgen05.commit;
-//   warps 2..9         epilogue: tcgen05.ld of the finished accumulator (two warps per TMEM lane
-//                      quarter, alternating 32-column chunks), bias / GELU / SwiGLU / fp32 residual
+//   warps 2..17        epilogue: tcgen05.ld of the finished accumulator (four warps per TMEM lane
+//                      quarter, a quarter of the tile's columns each), bias / GELU / SwiGLU / fp32 residual
 //                      update, bf16 store -- while the MMA warp already fills the other accumulator.
 // Split-k (weight-streaming groups with few tiles): every k range of a tile writes its fp32
 // partial; the range that finishes last (an atomic counter per tile, no waiting) adds the partials
@@ -32,9 +32,9 @@ constexpr int B_BYTES_MAX = TC_BN_MAX * TC_BK * 2;  // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES_MAX;
 constexpr int ACC_COLS = TC_BN_MAX;                 // TMEM columns per accumulator
 constexpr int TMEM_COLS = 2 * ACC_COLS;             // 512: the whole TMEM of the SM
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_WARPS = 16;
 constexpr int N_THREADS = 64 + EPI_WARPS * 32;
-constexpr int STAGE_OUT_BYTES = 128 * 256;          // epilogue staging: 128 rows x 256 bytes
+constexpr int STAGE_OUT_BYTES = EPI_WARPS * 2048;    // epilogue staging: 2 KB (32 rows x 64 bytes) per warp
 constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + STAGE_OUT_BYTES + 256;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
@@ -65,6 +65,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
+    if (it >= 8) __nanosleep(32);             // a long wait: stop competing with the epilogue warps for issue slots
     if ((it & 1023u) == 1023u) {
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer();
@@ -117,6 +118,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -415,11 +424,11 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
       if (!ok) *abort_flag = 1;
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..9)
+    // ------------------------------------------------------------ epilogue (warps 2..17)
     const int ew = warp - 2;
     const int et = threadIdx.x - 64;          // 0..255 among the epilogue threads
     const int quarter = warp & 3;             // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int half = ew >> 2;                 // which of the two warps of the quarter: 32-column chunks half, half+2, ...
+    const int part = ew >> 2;                 // which quarter of the tile's columns this warp owns
     const int row = quarter * 32 + lane;      // row of the tile this thread reads from TMEM
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -433,11 +442,13 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
         g_end = g.tile_start + g.tiles_m * g.tiles_n * g.ksplit;
       }
       const Item it = decode_item(g, item - g.tile_start);
-      // bias of this warp's column half, 4 values per lane, requested before the accumulator is awaited
+      // bias of this warp's columns, 4 values per lane, requested before the accumulator is awaited
       uint2 bias_reg = make_uint2(0u, 0u);
       if (g.epi & EPI_BIAS) {
-        const int nb = it.n0 + half * (g.bn >> 1) + lane * 4;
-        if (nb + 4 <= g.N) {
+        const int nb = it.n0 + part * (g.bn >> 2) + lane * 4;
+        if (lane * 4 >= (g.bn >> 2)) {
+          // beyond this warp's columns
+        } else if (nb + 4 <= g.N) {
           bias_reg = __ldg(reinterpret_cast<const uint2*>(g.bias + nb));
         } else {
           unsigned short e[4] = {0, 0, 0, 0};
@@ -461,16 +472,16 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
       const bool split = g.ksplit > 1;
       const size_t pld = (size_t)g.tiles_n * g.bn;                                   // partial row length
       if (split) {
-        float* part = g.partial + ((size_t)it.split * g.tiles_m * TC_BM + m) * pld + it.n0;
+        float* pdst = g.partial + ((size_t)it.split * g.tiles_m * TC_BM + m) * pld + it.n0;
 #pragma unroll 1
-        for (int c = half * 32; c < g.bn; c += 64) {
+        for (int c = part * 32; c < g.bn; c += 128) {
           if (it.n0 + c >= g.N) break;           // uniform across the warp
           uint32_t r[32];
           tmem_ld32(taddr + (uint32_t)c, r);
           if (m < g.M) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
-              __stcg(reinterpret_cast<float4*>(part + c + j),
+              __stcg(reinterpret_cast<float4*>(pdst + c + j),
                      make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
                                  __uint_as_float(r[j + 3])));
           }
@@ -498,33 +509,77 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
         }
         epi_barrier();                         // last_flag may be rewritten only after everyone read it
       } else {
-        // direct epilogue, warp by warp with no block-level barrier.  Warp (quarter, half) owns rows
-        // quarter*32..+31 and the half-th half of the tile's columns, in sub-passes of 64 accumulator
-        // columns (32 for an fp32 residual).  Phase 1: each lane turns its row's chunk into output
-        // values and parks them in the warp's 4 KB staging area (16-byte pieces XOR-swizzled by row);
-        // phase 2: the warp writes the 32 rows out with 128-byte row segments.
+        // direct epilogue, warp by warp with no block-level barrier.  Warp (quarter, part) owns rows
+        // quarter*32..+31 and the part-th quarter of the tile's columns.  Per chunk (32 accumulator
+        // columns; 16 for an fp32 residual) each lane turns its row's values into outputs and parks
+        // them in the warp's 2 KB staging area (64-byte rows, 16-byte pieces XOR-swizzled by row); then
+        // the warp writes the 32 rows out in 64-byte row segments.  Sixteen epilogue warps (four per
+        // scheduler) hide each other's TMEM, shuffle and arithmetic latencies.
         const bool f32 = (g.epi & EPI_RESID_F32) != 0, swi = (g.epi & EPI_SWIGLU) != 0;
         const int rows = min(32, g.M - it.m0 - quarter * 32);  // valid rows of this warp (may be <= 0)
-        unsigned char* wst = stage_out + ew * 4096;
-        unsigned char* srow = wst + lane * 128;
-        const int c_end = min((half + 1) * (g.bn >> 1), g.N - it.n0);
-        for (int g0 = half * (g.bn >> 1); g0 < c_end; g0 += 64) {
-#pragma unroll
-          for (int h2 = 0; h2 < 2; ++h2) {
-            const int c = g0 + 32 * h2;
-            if (c >= c_end) break;
+        unsigned char* wst = stage_out + ew * 2048;
+        unsigned char* srow = wst + lane * 64;
+        const int sw = (lane >> 1) & 3;                        // swizzle of this lane's staged row
+        const int c_begin = part * (g.bn >> 2);
+        const int c_end = min(c_begin + (g.bn >> 2), g.N - it.n0);
+        if (f32) {
+#pragma unroll 1
+          for (int c = c_begin; c < c_end; c += 16) {
             const int n = it.n0 + c;
-            const int acc_valid = min(32, g.N - n);              // valid accumulator columns of this chunk
-            float4 cpre[8];
-            if (f32) {                                           // residual values of this chunk, requested early
-              const float* Cr = reinterpret_cast<const float*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + n;
+            const int acc_valid = min(16, g.N - n);
+            float* C = reinterpret_cast<float*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + n;
+            float4 cpre[4];                                      // residual values, requested before the TMEM read
 #pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const int idx = lane + k * 32, r2 = idx >> 3, col = (idx & 7) << 2;
-                cpre[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (r2 < rows && col + 4 <= acc_valid) cpre[k] = *reinterpret_cast<const float4*>(Cr + (size_t)r2 * g.ldc + col);
+            for (int k = 0; k < 4; ++k) {
+              const int idx = lane + k * 32, r2 = idx >> 2, col = (idx & 3) << 2;
+              cpre[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (r2 < rows && col + 4 <= acc_valid) cpre[k] = *reinterpret_cast<const float4*>(C + (size_t)r2 * g.ldc + col);
+            }
+            uint32_t r16[16];
+            tmem_ld16(taddr + (uint32_t)c, r16);
+            float v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r16[j]);
+            if (g.epi & EPI_BIAS) {
+              const int lane0 = (c - c_begin) >> 2;
+#pragma unroll
+              for (int jj = 0; jj < 8; ++jj) {
+                const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
+                v[2 * jj] += __uint_as_float(w << 16);
+                v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
               }
             }
+            if (g.epi & EPI_GELU) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] = gelu_erf(v[j]);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              *reinterpret_cast<float4*>(srow + ((k ^ sw) << 4)) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+            __syncwarp();
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const int idx = lane + k * 32, r2 = idx >> 2, pp = idx & 3, col = pp << 2;
+              if (r2 >= rows || col >= acc_valid) continue;
+              const float4 a = *reinterpret_cast<const float4*>(wst + r2 * 64 + ((pp ^ ((r2 >> 1) & 3)) << 4));
+              float* cp = C + (size_t)r2 * g.ldc + col;
+              if (col + 4 <= acc_valid) {
+                float4 cv = cpre[k];
+                cv.x += a.x; cv.y += a.y; cv.z += a.z; cv.w += a.w;
+                *reinterpret_cast<float4*>(cp) = cv;
+              } else {
+                const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (col + j < acc_valid) cp[j] += av[j];
+              }
+            }
+            __syncwarp();                        // the staging area is reused by the next chunk
+          }
+        } else {
+#pragma unroll 1
+          for (int c = c_begin; c < c_end; c += 32) {
+            const int n = it.n0 + c;
+            const int acc_valid = min(32, g.N - n);
             uint32_t r32[32];
             tmem_ld32(taddr + (uint32_t)c, r32);
             float v[32];
@@ -532,7 +587,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r32[j]);
             if (g.epi & EPI_BIAS) {
               // the 32 bias values of this chunk sit in 8 consecutive lanes of bias_reg (zero past N)
-              const int lane0 = (c - half * (g.bn >> 1)) >> 2;
+              const int lane0 = (c - c_begin) >> 2;
 #pragma unroll
               for (int jj = 0; jj < 16; ++jj) {
                 const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
@@ -544,31 +599,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
 #pragma unroll
               for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
             }
-            if (f32) {
-#pragma unroll
-              for (int k = 0; k < 8; ++k)
-                *reinterpret_cast<float4*>(srow + ((k ^ (lane & 7)) << 4)) =
-                    make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
-              __syncwarp();
-              float* C = reinterpret_cast<float*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + n;
-#pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const int idx = lane + k * 32, r2 = idx >> 3, pp = idx & 7, col = pp << 2;
-                if (r2 >= rows || col >= acc_valid) continue;
-                const float4 a = *reinterpret_cast<const float4*>(wst + r2 * 128 + ((pp ^ (r2 & 7)) << 4));
-                float* cp = C + (size_t)r2 * g.ldc + col;
-                if (col + 4 <= acc_valid) {
-                  float4 cv = cpre[k];
-                  cv.x += a.x; cv.y += a.y; cv.z += a.z; cv.w += a.w;
-                  *reinterpret_cast<float4*>(cp) = cv;
-                } else {
-                  const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) if (col + j < acc_valid) cp[j] += av[j];
-                }
-              }
-              __syncwarp();                      // the staging area is reused by the next chunk
-            } else if (swi) {
+            if (swi) {
 #pragma unroll
               for (int k = 0; k < 2; ++k) {                      // 32 columns -> 16 outputs -> 2 pieces
                 uint4 o;
@@ -576,7 +607,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
                 o.y = pack2(silu_f(v[16 * k + 4]) * v[16 * k + 5], silu_f(v[16 * k + 6]) * v[16 * k + 7]);
                 o.z = pack2(silu_f(v[16 * k + 8]) * v[16 * k + 9], silu_f(v[16 * k + 10]) * v[16 * k + 11]);
                 o.w = pack2(silu_f(v[16 * k + 12]) * v[16 * k + 13], silu_f(v[16 * k + 14]) * v[16 * k + 15]);
-                *reinterpret_cast<uint4*>(srow + (((2 * h2 + k) ^ (lane & 7)) << 4)) = o;
+                *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
               }
             } else {
 #pragma unroll
@@ -584,24 +615,20 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
                 uint4 o;
                 o.x = pack2(v[8 * k], v[8 * k + 1]); o.y = pack2(v[8 * k + 2], v[8 * k + 3]);
                 o.z = pack2(v[8 * k + 4], v[8 * k + 5]); o.w = pack2(v[8 * k + 6], v[8 * k + 7]);
-                *reinterpret_cast<uint4*>(srow + (((4 * h2 + k) ^ (lane & 7)) << 4)) = o;
+                *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
               }
             }
-          }
-          if (!f32) {
             __syncwarp();
-            // write the 32 rows x 64 accumulator columns out with 128-byte (SwiGLU: 64-byte) row segments
-            const int acc_valid = min(64, g.N - it.n0 - g0);
+            // write the 32 rows out: 64-byte (SwiGLU: 32-byte) row segments
             const int out_valid = swi ? (acc_valid >> 1) : acc_valid;
-            const int ppr = swi ? 4 : 8;                         // 8-element pieces per staged row
-            bf16* C = reinterpret_cast<bf16*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc +
-                      (swi ? ((it.n0 + g0) >> 1) : (it.n0 + g0));
+            const int ppr = swi ? 2 : 4;                         // 8-element pieces per staged row
+            bf16* C = reinterpret_cast<bf16*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + (swi ? (n >> 1) : n);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < 4; ++k) {
               const int idx = lane + k * 32;
-              const int r2 = swi ? (idx >> 2) : (idx >> 3), pp = swi ? (idx & 3) : (idx & 7), col = pp << 3;
+              const int r2 = swi ? (idx >> 1) : (idx >> 2), pp = swi ? (idx & 1) : (idx & 3), col = pp << 3;
               if (idx >= 32 * ppr || r2 >= rows || col >= out_valid) continue;
-              const uint4 a = *reinterpret_cast<const uint4*>(wst + r2 * 128 + ((pp ^ (r2 & 7)) << 4));
+              const uint4 a = *reinterpret_cast<const uint4*>(wst + r2 * 64 + ((pp ^ ((r2 >> 1) & 3)) << 4));
               bf16* cp = C + (size_t)r2 * g.ldc + col;
               if (col + 8 <= out_valid) {
                 *reinterpret_cast<uint4*>(cp) = a;
@@ -612,7 +639,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
                   if (col + j < out_valid) cp[j] = __ushort_as_bfloat16((unsigned short)(aw[j >> 1] >> ((j & 1) * 16)));
               }
             }
-            __syncwarp();                        // the staging area is reused by the next 64 columns
+            __syncwarp();                        // the staging area is reused by the next chunk
           }
         }
         // the accumulator is drained by this warp: hand it back to the MMA warp
