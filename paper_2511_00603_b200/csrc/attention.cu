@@ -178,6 +178,10 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// 16-byte copy that writes zeros instead when `valid` is false (the source is not read then)
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, bool valid) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
+}
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -483,20 +487,25 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
   bf16* Ks = reinterpret_cast<bf16*>(smem_raw);
   bf16* Vs = Ks + (size_t)Tp * ENC_LD;
   const bf16* base = g.qkv + (size_t)b * T * 3 * d + (size_t)h * HD;
-  for (int i = threadIdx.x; i < Tp * (HD / 8); i += blockDim.x) {
-    const int t = i >> 3, cc = i & 7;
-    uint4 kk = make_uint4(0, 0, 0, 0), vv = kk;
-    if (t < T) {
-      kk = *reinterpret_cast<const uint4*>(base + (size_t)t * 3 * d + d + cc * 8);
-      vv = *reinterpret_cast<const uint4*>(base + (size_t)t * 3 * d + 2 * d + cc * 8);
+  // K and V are brought in by cp.async, one commit group per block of 64 keys, all in flight at once;
+  // the loop below waits for block after block, so the first scores start while later keys still load
+  const int nblk = Tp >> 6;
+  {
+    const uint32_t ks_u = (uint32_t)__cvta_generic_to_shared(Ks), vs_u = (uint32_t)__cvta_generic_to_shared(Vs);
+    for (int blk = 0; blk < nblk; ++blk) {
+      for (int i = threadIdx.x; i < 64 * (HD / 8); i += blockDim.x) {
+        const int t = blk * 64 + (i >> 3), cc = i & 7;
+        const bool valid = t < T;
+        const bf16* src = base + (size_t)(valid ? t : 0) * 3 * d + cc * 8;
+        cp_async16_zfill(ks_u + (uint32_t)(t * ENC_LD + cc * 8) * 2u, src + d, valid);
+        cp_async16_zfill(vs_u + (uint32_t)(t * ENC_LD + cc * 8) * 2u, src + 2 * d, valid);
+      }
+      cp_async_commit();
     }
-    *reinterpret_cast<uint4*>(Ks + (size_t)t * ENC_LD + cc * 8) = kk;
-    *reinterpret_cast<uint4*>(Vs + (size_t)t * ENC_LD + cc * 8) = vv;
   }
-  __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row0 = qb * ENC_ROWS + warp * 16;
-  if (row0 >= T) return;
+  const bool active = row0 < T;             // idle warps still take part in the block barriers below
   const int gq = lane >> 2, tq = lane & 3;
   // Q fragments of the warp's 16 rows: 4 k-steps of 16
   uint32_t qa[4][4];
@@ -522,6 +531,19 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
   // ldmatrix lane addressing: lanes 0-7 rows of matrix 0, 8-15 matrix 1, 16-23 matrix 2, 24-31 matrix 3
   const int lm_row = lane & 7, lm_mat = lane >> 3;
   for (int kb = 0; kb < Tp; kb += 64) {
+    // at most (blocks after this one) copy groups may still be pending
+    switch (nblk - 1 - (kb >> 6)) {
+      case 0: cp_async_wait<0>(); break;
+      case 1: cp_async_wait<1>(); break;
+      case 2: cp_async_wait<2>(); break;
+      case 3: cp_async_wait<3>(); break;
+      case 4: cp_async_wait<4>(); break;
+      case 5: cp_async_wait<5>(); break;
+      case 6: cp_async_wait<6>(); break;
+      default: cp_async_wait<7>(); break;
+    }
+    __syncthreads();
+    if (!active) continue;
     float sc[8][4];
 #pragma unroll
     for (int n = 0; n < 8; ++n) { sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f; }
@@ -585,6 +607,7 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
       }
     }
   }
+  if (!active) return;
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
