@@ -210,7 +210,8 @@ int epara_admit_queue(int n, const uint64_t* tickets, const long long* deadline_
 typedef struct {
   const void* A;      /* bf16 [M, lda]  */
   const void* W;      /* bf16 [N, ldw], K contiguous */
-  void* C;            /* bf16 [M, ldc] (or fp32 when EPARA_EPI_RESID_F32); SwiGLU: [M, N/2] */
+  void* C;            /* bf16 [M, ldc] (or fp32 when EPARA_EPI_RESID_F32); SwiGLU: [M, N/2].  Pad columns
+                         between N and the next multiple of 8 may be overwritten. */
   const void* bias;   /* bf16 [N] or NULL */
   int M, N, K;
   int lda, ldw, ldc;  /* elements; multiples of 8 */

@@ -32,6 +32,9 @@ struct ReqDesc {
 struct alignas(64) GemmGroup {
   CUtensorMap tmA;
   CUtensorMap tmW;
+  CUtensorMap tmC;   // output, written by TMA from the epilogue's staging rows: bf16 [rows, N] with a
+                     // 32 x 32 box (SwiGLU: [rows, N/2], 16 x 32), or fp32 [rows, N] with a 16 x 32 box
+                     // for the residual update (TMA reduce-add)
   const bf16* A;
   const bf16* W;
   void* C;
@@ -44,6 +47,8 @@ struct alignas(64) GemmGroup {
   int bn, ksplit;  // tensor-core kernel only: tile width (128 or 256), k ranges per tile
   float* partial;  // [ksplit][tiles_m * 128][tiles_n * bn] fp32, ksplit > 1 only
   int* counters;   // [tiles_m * tiles_n], zero between launches
+  int c_rows;      // row extent of tmC (rows at and beyond it are never written)
+  int pad0, pad1, pad2;
 };
 
 struct GemmLaunch {      // header followed by groups

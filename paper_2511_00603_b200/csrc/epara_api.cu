@@ -65,6 +65,22 @@ bool make_tmap(CUtensorMap* tm, const void* ptr, long long rows, long long cols,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Output map of a GEMM for the epilogue's TMA stores: rows of 64 bytes (SwiGLU: 32 bytes) per box row,
+// matching swizzle, 32 rows per box.
+bool make_tmap_c(CUtensorMap* tm, void* C, long long rows, int N, int ldc, int epi) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const bool f32 = (epi & EPI_RESID_F32) != 0, swi = (epi & EPI_SWIGLU) != 0;
+  const int cols = swi ? N / 2 : N;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ldc * (f32 ? 4 : 2)};
+  cuuint32_t box[2] = {(cuuint32_t)(f32 ? 16 : (swi ? 16 : 32)), 32};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, C, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swi ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct Op {
   int kind;           // EPARA_K_*
   int rows_per_req;   // rows of this op = batch * rows_per_req
@@ -194,7 +210,9 @@ bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap,
   if (bl.c) {
     if (!make_tmap(&g.tmA, A, rows_cap, K, lda, TC_BM)) return false;
     if (!make_tmap(&g.tmW, W, N, K, K, g.bn)) return false;
+    if (!make_tmap_c(&g.tmC, C, rows_cap, N, ldc, g.epi)) return false;
   }
+  g.c_rows = (int)rows_cap;
   m->ops.push_back(op);
   return true;
 }
@@ -987,7 +1005,9 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
     if (!simt && q.M > 0) {
       if (!make_tmap(&g.tmA, q.A, q.M, q.K, q.lda, TC_BM)) return EPARA_E_CUDA;
       if (!make_tmap(&g.tmW, q.W, q.N, q.K, q.ldw, g.bn)) return EPARA_E_CUDA;
+      if (!make_tmap_c(&g.tmC, q.C, q.M, q.N, q.ldc, q.epilogue)) return EPARA_E_CUDA;
     }
+    g.c_rows = q.M;
     if (g.ksplit > 1) {
       soff = align_up(soff, 256);
       g.partial = (float*)((unsigned char*)scratch + soff);

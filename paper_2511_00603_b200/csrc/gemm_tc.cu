@@ -80,6 +80,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+// TMA store / reduce-add of one staged box (32 rows) to the output tensor; rows and columns outside
+// the tensor are clipped by the hardware.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tm), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tm), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tensormap_acquire(const CUtensorMap* tm) {
   asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tm) : "memory");
 }
@@ -162,13 +175,15 @@ struct GView {
   void* C;
   float* partial;
   int* counters;
-  int M, N, K, ldc, epi, tile_start, tiles_m, tiles_n, bn, ksplit;
+  const CUtensorMap* tmC;
+  int M, N, K, ldc, epi, tile_start, tiles_m, tiles_n, bn, ksplit, c_rows;
 };
 __device__ __forceinline__ GView load_view(const GemmGroup* g) {
   GView v;
   v.bias = g->bias; v.C = g->C; v.partial = g->partial; v.counters = g->counters;
   v.M = g->M; v.N = g->N; v.K = g->K; v.ldc = g->ldc; v.epi = g->epi; v.tile_start = g->tile_start;
   v.tiles_m = g->tiles_m; v.tiles_n = g->tiles_n; v.bn = g->bn; v.ksplit = g->ksplit;
+  v.tmC = &g->tmC; v.c_rows = g->c_rows;
   return v;
 }
 
@@ -440,6 +455,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
       if (item >= g_end || item < g.tile_start) {
         g = load_view(groups + find_group_tc(groups, n_groups, item));
         g_end = g.tile_start + g.tiles_m * g.tiles_n * g.ksplit;
+        if (lane == 0) tensormap_acquire(g.tmC);
       }
       const Item it = decode_item(g, item - g.tile_start);
       // bias of this warp's columns, 4 values per lane, requested before the accumulator is awaited
@@ -512,134 +528,87 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
         // direct epilogue, warp by warp with no block-level barrier.  Warp (quarter, part) owns rows
         // quarter*32..+31 and the part-th quarter of the tile's columns.  Per chunk (32 accumulator
         // columns; 16 for an fp32 residual) each lane turns its row's values into outputs and parks
-        // them in the warp's 2 KB staging area (64-byte rows, 16-byte pieces XOR-swizzled by row); then
-        // the warp writes the 32 rows out in 64-byte row segments.  Sixteen epilogue warps (four per
-        // scheduler) hide each other's TMEM, shuffle and arithmetic latencies.
+        // them in the warp's 2 KB staging area (64-byte rows, SwiGLU 32-byte rows, 16-byte pieces in
+        // the TMA swizzle pattern, which also keeps the stores free of bank conflicts); one lane then
+        // hands the 32-row box to the TMA unit: a plain store for bf16 outputs, a reduce-add for the
+        // fp32 residual (the addition happens at L2; the SM never reads C).  The hardware clips rows
+        // and columns outside the tensor.  Sixteen epilogue warps hide each other's latencies.
         const bool f32 = (g.epi & EPI_RESID_F32) != 0, swi = (g.epi & EPI_SWIGLU) != 0;
-        const int rows = min(32, g.M - it.m0 - quarter * 32);  // valid rows of this warp (may be <= 0)
         unsigned char* wst = stage_out + ew * 2048;
-        unsigned char* srow = wst + lane * 64;
-        const int sw = (lane >> 1) & 3;                        // swizzle of this lane's staged row
+        const uint32_t wst_u = smem_u32(wst);
+        const int y0 = it.m0 + quarter * 32;
+        const bool box_ok = y0 < g.c_rows;                     // some row of this warp's box is inside the tensor
         const int c_begin = part * (g.bn >> 2);
         const int c_end = min(c_begin + (g.bn >> 2), g.N - it.n0);
-        if (f32) {
+        const int cw = f32 ? 16 : 32;                          // accumulator columns per chunk
 #pragma unroll 1
-          for (int c = c_begin; c < c_end; c += 16) {
-            const int n = it.n0 + c;
-            const int acc_valid = min(16, g.N - n);
-            float* C = reinterpret_cast<float*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + n;
-            float4 cpre[4];                                      // residual values, requested before the TMEM read
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const int idx = lane + k * 32, r2 = idx >> 2, col = (idx & 3) << 2;
-              cpre[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (r2 < rows && col + 4 <= acc_valid) cpre[k] = *reinterpret_cast<const float4*>(C + (size_t)r2 * g.ldc + col);
-            }
+        for (int c = c_begin; c < c_end; c += cw) {
+          const int n = it.n0 + c;
+          float v[32];
+          if (f32) {
             uint32_t r16[16];
             tmem_ld16(taddr + (uint32_t)c, r16);
-            float v[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r16[j]);
-            if (g.epi & EPI_BIAS) {
-              const int lane0 = (c - c_begin) >> 2;
+          } else {
+            uint32_t r32[32];
+            tmem_ld32(taddr + (uint32_t)c, r32);
 #pragma unroll
-              for (int jj = 0; jj < 8; ++jj) {
-                const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
-                v[2 * jj] += __uint_as_float(w << 16);
-                v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
-              }
-            }
-            if (g.epi & EPI_GELU) {
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r32[j]);
+          }
+          if (g.epi & EPI_BIAS) {
+            // the bias values of this chunk sit in consecutive lanes of bias_reg (zero past N)
+            const int lane0 = (c - c_begin) >> 2;
 #pragma unroll
-              for (int j = 0; j < 16; ++j) v[j] = gelu_erf(v[j]);
+            for (int jj = 0; jj < 16; ++jj) {
+              if (f32 && jj >= 8) break;
+              const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
+              v[2 * jj] += __uint_as_float(w << 16);
+              v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
             }
+          }
+          if (g.epi & EPI_GELU) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (!f32 || j < 16) v[j] = gelu_erf(v[j]);
+          }
+          // the previous box of this warp must have been read out of the staging area
+          if (lane == 0) bulk_wait_read0();
+          __syncwarp();
+          if (f32) {
+            unsigned char* srow = wst + lane * 64;
+            const int sw = (lane >> 1) & 3;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
               *reinterpret_cast<float4*>(srow + ((k ^ sw) << 4)) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
-            __syncwarp();
+          } else if (swi) {
+            unsigned char* srow = wst + lane * 32;             // 32 columns -> 16 outputs -> 2 pieces
+            const int sw = (lane >> 2) & 1;
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              uint4 o;
+              o.x = pack2(silu_f(v[16 * k]) * v[16 * k + 1], silu_f(v[16 * k + 2]) * v[16 * k + 3]);
+              o.y = pack2(silu_f(v[16 * k + 4]) * v[16 * k + 5], silu_f(v[16 * k + 6]) * v[16 * k + 7]);
+              o.z = pack2(silu_f(v[16 * k + 8]) * v[16 * k + 9], silu_f(v[16 * k + 10]) * v[16 * k + 11]);
+              o.w = pack2(silu_f(v[16 * k + 12]) * v[16 * k + 13], silu_f(v[16 * k + 14]) * v[16 * k + 15]);
+              *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
+            }
+          } else {
+            unsigned char* srow = wst + lane * 64;             // 32 columns -> 4 pieces
+            const int sw = (lane >> 1) & 3;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              const int idx = lane + k * 32, r2 = idx >> 2, pp = idx & 3, col = pp << 2;
-              if (r2 >= rows || col >= acc_valid) continue;
-              const float4 a = *reinterpret_cast<const float4*>(wst + r2 * 64 + ((pp ^ ((r2 >> 1) & 3)) << 4));
-              float* cp = C + (size_t)r2 * g.ldc + col;
-              if (col + 4 <= acc_valid) {
-                float4 cv = cpre[k];
-                cv.x += a.x; cv.y += a.y; cv.z += a.z; cv.w += a.w;
-                *reinterpret_cast<float4*>(cp) = cv;
-              } else {
-                const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) if (col + j < acc_valid) cp[j] += av[j];
-              }
+              uint4 o;
+              o.x = pack2(v[8 * k], v[8 * k + 1]); o.y = pack2(v[8 * k + 2], v[8 * k + 3]);
+              o.z = pack2(v[8 * k + 4], v[8 * k + 5]); o.w = pack2(v[8 * k + 6], v[8 * k + 7]);
+              *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
             }
-            __syncwarp();                        // the staging area is reused by the next chunk
           }
-        } else {
-#pragma unroll 1
-          for (int c = c_begin; c < c_end; c += 32) {
-            const int n = it.n0 + c;
-            const int acc_valid = min(32, g.N - n);
-            uint32_t r32[32];
-            tmem_ld32(taddr + (uint32_t)c, r32);
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r32[j]);
-            if (g.epi & EPI_BIAS) {
-              // the 32 bias values of this chunk sit in 8 consecutive lanes of bias_reg (zero past N)
-              const int lane0 = (c - c_begin) >> 2;
-#pragma unroll
-              for (int jj = 0; jj < 16; ++jj) {
-                const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
-                v[2 * jj] += __uint_as_float(w << 16);
-                v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
-              }
-            }
-            if (g.epi & EPI_GELU) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-            }
-            if (swi) {
-#pragma unroll
-              for (int k = 0; k < 2; ++k) {                      // 32 columns -> 16 outputs -> 2 pieces
-                uint4 o;
-                o.x = pack2(silu_f(v[16 * k]) * v[16 * k + 1], silu_f(v[16 * k + 2]) * v[16 * k + 3]);
-                o.y = pack2(silu_f(v[16 * k + 4]) * v[16 * k + 5], silu_f(v[16 * k + 6]) * v[16 * k + 7]);
-                o.z = pack2(silu_f(v[16 * k + 8]) * v[16 * k + 9], silu_f(v[16 * k + 10]) * v[16 * k + 11]);
-                o.w = pack2(silu_f(v[16 * k + 12]) * v[16 * k + 13], silu_f(v[16 * k + 14]) * v[16 * k + 15]);
-                *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
-              }
-            } else {
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {                      // 32 columns -> 4 pieces
-                uint4 o;
-                o.x = pack2(v[8 * k], v[8 * k + 1]); o.y = pack2(v[8 * k + 2], v[8 * k + 3]);
-                o.z = pack2(v[8 * k + 4], v[8 * k + 5]); o.w = pack2(v[8 * k + 6], v[8 * k + 7]);
-                *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
-              }
-            }
-            __syncwarp();
-            // write the 32 rows out: 64-byte (SwiGLU: 32-byte) row segments
-            const int out_valid = swi ? (acc_valid >> 1) : acc_valid;
-            const int ppr = swi ? 2 : 4;                         // 8-element pieces per staged row
-            bf16* C = reinterpret_cast<bf16*>(g.C) + (size_t)(it.m0 + quarter * 32) * g.ldc + (swi ? (n >> 1) : n);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const int idx = lane + k * 32;
-              const int r2 = swi ? (idx >> 1) : (idx >> 2), pp = swi ? (idx & 1) : (idx & 3), col = pp << 3;
-              if (idx >= 32 * ppr || r2 >= rows || col >= out_valid) continue;
-              const uint4 a = *reinterpret_cast<const uint4*>(wst + r2 * 64 + ((pp ^ ((r2 >> 1) & 3)) << 4));
-              bf16* cp = C + (size_t)r2 * g.ldc + col;
-              if (col + 8 <= out_valid) {
-                *reinterpret_cast<uint4*>(cp) = a;
-              } else {
-                const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                  if (col + j < out_valid) cp[j] = __ushort_as_bfloat16((unsigned short)(aw[j >> 1] >> ((j & 1) * 16)));
-              }
-            }
-            __syncwarp();                        // the staging area is reused by the next chunk
+          fence_async_smem();                    // the staged values must be visible to the TMA unit
+          __syncwarp();
+          if (lane == 0 && box_ok) {
+            if (f32) tma_reduce_add_2d(g.tmC, wst_u, n, y0);
+            else tma_store_2d(g.tmC, wst_u, swi ? (n >> 1) : n, y0);
+            bulk_commit();
           }
         }
         // the accumulator is drained by this warp: hand it back to the MMA warp
@@ -649,6 +618,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) bulk_wait_read0();       // staged boxes still being read by the TMA unit
     if (!ok) *abort_flag = 1;
   }
   tc_fence_before();
