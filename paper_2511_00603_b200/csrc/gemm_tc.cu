@@ -639,9 +639,6 @@ void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int
   if (rows_cap <= 0) { *bn = 128; *ksplit = 1; return; }
   if (rows_cap > 256) {                       // dense: tensor-bound; a 128 x 256 MMA runs at about twice the
     *bn = (N > 128) ? 256 : 128;              // efficiency of a 128 x 128 one, which outweighs padded columns
-    // ... except for the fp32 residual update, which is bound by its read-modify-write of C: there
-    // padded columns cost more than narrow MMAs
-    if ((epi & EPI_RESID_F32) && padded(128) < padded(256)) *bn = 128;
     *ksplit = 1;
     return;
   }
