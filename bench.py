@@ -492,12 +492,44 @@ def run_micro(args):
         kvb = float(lens.sum()) * 2 * Hkv * hd * 2
         print(json.dumps({"kernel": "attn_decode+combine", "B": B, "Hq": Hq, "Hkv": Hkv, "hd": hd, "tokens": int(lens.sum()),
                           "ms": ms, "kv_gbs": kvb / (ms / 1e3) / 1e9, "frac_hbm": kvb / (ms / 1e3) / 1e9 / peaks["hbm_gbs"]}))
+    elif args.micro == "decode_step":
+        # whole decode steps of one decoder (configs[2] / the decoder of configs[4]) through the step API
+        from paper_2511_00603_b200 import server, workloads as W
+        cfgm = W.DEC_8B if args.case == "dec_8b" else W.DEC_1B
+        hi = 8192 if args.case == "dec_8b" else 4096
+        lo = 512 if args.case == "dec_8b" else 128
+        B = args.m or 128
+        srv = server.Server(device=0, workspace_bytes=2 << 30)
+        inst = W.Instance(srv, synth.make_decoder(seed=2, device=dev, **cfgm), E.CAT_FS, B, seed=21, kv_lo=lo, kv_hi=hi)
+        srv.ctx.epara_set_profile(True)
+        times = []
+        for i in range(args.steps + 3):
+            flush.zero_()
+            inst.submit_all(srv.ctx)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            info = srv.ctx.epara_step(stream.cuda_stream, 0)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            for t in inst.tickets:
+                srv.ctx.epara_collect(t)
+            if i >= 3:
+                times.append(e0.elapsed_time(e1))
+        prof = srv.ctx.epara_step_profile()
+        ms = sorted(times)[len(times) // 2]
+        byt = info.weight_bytes + info.kv_bytes
+        print(json.dumps({"kernel": "decode step", "case": args.case, "B": B, "ms": ms, "launches": info.launches,
+                          "weight_gb": info.weight_bytes / 1e9, "kv_gb": info.kv_bytes / 1e9,
+                          "hbm_gbs": byt / (ms / 1e3) / 1e9, "frac_hbm": byt / (ms / 1e3) / 1e9 / peaks["hbm_gbs"],
+                          "tokens_per_s": B / (ms / 1e3),
+                          "per_kind_ms": {k: round(v[0], 4) for k, v in prof.items() if v[1]}}))
+        srv.close()
     return 0
 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["gemm", "attn_dec"], help="time one kernel instead of the step")
+    ap.add_argument("--micro", default=None, choices=["gemm", "attn_dec", "decode_step"], help="time one kernel instead of the step")
     ap.add_argument("--case", default="vit_s")
     ap.add_argument("--m", type=int, default=0, help="override M (gemm) or B (attn_dec) of the micro case")
     ap.add_argument("--gpus", type=int, default=1)
