@@ -645,8 +645,10 @@ void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int
   // weight streaming: the widest tile (most W bytes in flight per stage).  Splitting K pays only when
   // a handful of tiles would each stream a very long K: measured on B200, the fixed cost of a split
   // item (partials, counter, reduction) exceeds the gain for K < 4096.
+  // One CTA streams only about 80 GB/s through its 4-stage ring, so when 256-wide tiles would leave
+  // SMs without work, 128-wide tiles (twice as many CTAs) stream faster.
   const int tiles_m = (int)((rows_cap + TC_BM - 1) / TC_BM);
-  *bn = (N > 128) ? 256 : 128;
+  *bn = (N > 128 && tiles_m * (padded(256) / 256) * 10 >= sm_count * 7) ? 256 : 128;
   const int tiles = tiles_m * (padded(*bn) / *bn);
   int ks = 1;
   if (kblocks >= 64 && tiles * 8 <= sm_count) {
