@@ -314,6 +314,101 @@ __device__ __forceinline__ void splitk_reduce(const GView& g, const Item& it, in
   }
 }
 
+// Direct epilogue of one warp for one tile, with no block-level barrier.  Warp (quarter, part) owns
+// rows quarter*32..+31 and the part-th quarter of the tile's columns.  Per chunk (32 accumulator
+// columns; 16 for an fp32 residual) each lane turns its row's values into outputs and parks them in
+// the warp's 2 KB staging area (64-byte rows, SwiGLU 32-byte rows, 16-byte pieces in the TMA swizzle
+// pattern, which also keeps the stores free of bank conflicts); one lane then hands the 32-row box to
+// the TMA unit: a plain store for bf16 outputs, a reduce-add for the fp32 residual (the addition
+// happens at L2; the SM never reads C).  The hardware clips rows and columns outside the tensor.
+// The accumulator is handed back to the MMA warp as soon as this warp's last chunk has left TMEM.
+// MODE: 0 bf16 output, 1 SwiGLU, 2 fp32 residual.
+template <int MODE>
+__device__ __forceinline__ void epi_direct(const GView& g, const Item& it, uint32_t taddr, unsigned char* wst, int quarter,
+                                           int part, int lane, uint2 bias_reg, uint32_t tempty) {
+  constexpr int CW = (MODE == 2) ? 16 : 32;                  // accumulator columns per chunk
+  const uint32_t wst_u = smem_u32(wst);
+  const int y0 = it.m0 + quarter * 32;
+  const bool box_ok = y0 < g.c_rows;                         // some row of this warp's box is inside the tensor
+  const int c_begin = part * (g.bn >> 2);
+  const int c_end = min(c_begin + (g.bn >> 2), g.N - it.n0);
+  if (c_begin >= c_end) {                                    // nothing to do for this warp: release at once
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(tempty);
+    return;
+  }
+#pragma unroll 1
+  for (int c = c_begin; c < c_end; c += CW) {
+    const int n = it.n0 + c;
+    float v[CW];
+    {
+      uint32_t r[CW];
+      if (MODE == 2) tmem_ld16(taddr + (uint32_t)c, r); else tmem_ld32(taddr + (uint32_t)c, r);
+#pragma unroll
+      for (int j = 0; j < CW; ++j) v[j] = __uint_as_float(r[j]);
+    }
+    if (c + CW >= c_end) {                                   // that was this warp's last read of the accumulator
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty);
+    }
+    if (g.epi & EPI_BIAS) {
+      // the bias values of this chunk sit in consecutive lanes of bias_reg (zero past N)
+      const int lane0 = (c - c_begin) >> 2;
+#pragma unroll
+      for (int jj = 0; jj < CW / 2; ++jj) {
+        const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
+        v[2 * jj] += __uint_as_float(w << 16);
+        v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
+      }
+    }
+    if (g.epi & EPI_GELU) {
+#pragma unroll
+      for (int j = 0; j < CW; ++j) v[j] = gelu_erf(v[j]);
+    }
+    // the previous box of this warp must have been read out of the staging area
+    if (lane == 0) bulk_wait_read0();
+    __syncwarp();
+    if (MODE == 2) {
+      unsigned char* srow = wst + lane * 64;
+      const int sw = (lane >> 1) & 3;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        *reinterpret_cast<float4*>(srow + ((k ^ sw) << 4)) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+    } else if (MODE == 1) {
+      unsigned char* srow = wst + lane * 32;                 // 32 columns -> 16 outputs -> 2 pieces
+      const int sw = (lane >> 2) & 1;
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        uint4 o;
+        o.x = pack2(silu_f(v[16 * k]) * v[16 * k + 1], silu_f(v[16 * k + 2]) * v[16 * k + 3]);
+        o.y = pack2(silu_f(v[16 * k + 4]) * v[16 * k + 5], silu_f(v[16 * k + 6]) * v[16 * k + 7]);
+        o.z = pack2(silu_f(v[16 * k + 8]) * v[16 * k + 9], silu_f(v[16 * k + 10]) * v[16 * k + 11]);
+        o.w = pack2(silu_f(v[16 * k + 12]) * v[16 * k + 13], silu_f(v[16 * k + 14]) * v[16 * k + 15]);
+        *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
+      }
+    } else {
+      unsigned char* srow = wst + lane * 64;                 // 32 columns -> 4 pieces
+      const int sw = (lane >> 1) & 3;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint4 o;
+        o.x = pack2(v[8 * k], v[8 * k + 1]); o.y = pack2(v[8 * k + 2], v[8 * k + 3]);
+        o.z = pack2(v[8 * k + 4], v[8 * k + 5]); o.w = pack2(v[8 * k + 6], v[8 * k + 7]);
+        *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
+      }
+    }
+    fence_async_smem();                      // the staged values must be visible to the TMA unit
+    __syncwarp();
+    if (lane == 0 && box_ok) {
+      if (MODE == 2) tma_reduce_add_2d(g.tmC, wst_u, n, y0);
+      else tma_store_2d(g.tmC, wst_u, MODE == 1 ? (n >> 1) : n, y0);
+      bulk_commit();
+    }
+  }
+}
+
 __global__ void __launch_bounds__(N_THREADS, 1)
 gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status) {
   extern __shared__ unsigned char smem_dyn[];
@@ -525,96 +620,11 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
         }
         epi_barrier();                         // last_flag may be rewritten only after everyone read it
       } else {
-        // direct epilogue, warp by warp with no block-level barrier.  Warp (quarter, part) owns rows
-        // quarter*32..+31 and the part-th quarter of the tile's columns.  Per chunk (32 accumulator
-        // columns; 16 for an fp32 residual) each lane turns its row's values into outputs and parks
-        // them in the warp's 2 KB staging area (64-byte rows, SwiGLU 32-byte rows, 16-byte pieces in
-        // the TMA swizzle pattern, which also keeps the stores free of bank conflicts); one lane then
-        // hands the 32-row box to the TMA unit: a plain store for bf16 outputs, a reduce-add for the
-        // fp32 residual (the addition happens at L2; the SM never reads C).  The hardware clips rows
-        // and columns outside the tensor.  Sixteen epilogue warps hide each other's latencies.
-        const bool f32 = (g.epi & EPI_RESID_F32) != 0, swi = (g.epi & EPI_SWIGLU) != 0;
+        // direct epilogue (see epi_direct), specialised by output mode
         unsigned char* wst = stage_out + ew * 2048;
-        const uint32_t wst_u = smem_u32(wst);
-        const int y0 = it.m0 + quarter * 32;
-        const bool box_ok = y0 < g.c_rows;                     // some row of this warp's box is inside the tensor
-        const int c_begin = part * (g.bn >> 2);
-        const int c_end = min(c_begin + (g.bn >> 2), g.N - it.n0);
-        const int cw = f32 ? 16 : 32;                          // accumulator columns per chunk
-#pragma unroll 1
-        for (int c = c_begin; c < c_end; c += cw) {
-          const int n = it.n0 + c;
-          float v[32];
-          if (f32) {
-            uint32_t r16[16];
-            tmem_ld16(taddr + (uint32_t)c, r16);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r16[j]);
-          } else {
-            uint32_t r32[32];
-            tmem_ld32(taddr + (uint32_t)c, r32);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r32[j]);
-          }
-          if (g.epi & EPI_BIAS) {
-            // the bias values of this chunk sit in consecutive lanes of bias_reg (zero past N)
-            const int lane0 = (c - c_begin) >> 2;
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-              if (f32 && jj >= 8) break;
-              const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, lane0 + (jj >> 1));
-              v[2 * jj] += __uint_as_float(w << 16);
-              v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
-            }
-          }
-          if (g.epi & EPI_GELU) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) if (!f32 || j < 16) v[j] = gelu_erf(v[j]);
-          }
-          // the previous box of this warp must have been read out of the staging area
-          if (lane == 0) bulk_wait_read0();
-          __syncwarp();
-          if (f32) {
-            unsigned char* srow = wst + lane * 64;
-            const int sw = (lane >> 1) & 3;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              *reinterpret_cast<float4*>(srow + ((k ^ sw) << 4)) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
-          } else if (swi) {
-            unsigned char* srow = wst + lane * 32;             // 32 columns -> 16 outputs -> 2 pieces
-            const int sw = (lane >> 2) & 1;
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-              uint4 o;
-              o.x = pack2(silu_f(v[16 * k]) * v[16 * k + 1], silu_f(v[16 * k + 2]) * v[16 * k + 3]);
-              o.y = pack2(silu_f(v[16 * k + 4]) * v[16 * k + 5], silu_f(v[16 * k + 6]) * v[16 * k + 7]);
-              o.z = pack2(silu_f(v[16 * k + 8]) * v[16 * k + 9], silu_f(v[16 * k + 10]) * v[16 * k + 11]);
-              o.w = pack2(silu_f(v[16 * k + 12]) * v[16 * k + 13], silu_f(v[16 * k + 14]) * v[16 * k + 15]);
-              *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
-            }
-          } else {
-            unsigned char* srow = wst + lane * 64;             // 32 columns -> 4 pieces
-            const int sw = (lane >> 1) & 3;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              uint4 o;
-              o.x = pack2(v[8 * k], v[8 * k + 1]); o.y = pack2(v[8 * k + 2], v[8 * k + 3]);
-              o.z = pack2(v[8 * k + 4], v[8 * k + 5]); o.w = pack2(v[8 * k + 6], v[8 * k + 7]);
-              *reinterpret_cast<uint4*>(srow + ((k ^ sw) << 4)) = o;
-            }
-          }
-          fence_async_smem();                    // the staged values must be visible to the TMA unit
-          __syncwarp();
-          if (lane == 0 && box_ok) {
-            if (f32) tma_reduce_add_2d(g.tmC, wst_u, n, y0);
-            else tma_store_2d(g.tmC, wst_u, swi ? (n >> 1) : n, y0);
-            bulk_commit();
-          }
-        }
-        // the accumulator is drained by this warp: hand it back to the MMA warp
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (g.epi & EPI_RESID_F32) epi_direct<2>(g, it, taddr, wst, quarter, part, lane, bias_reg, tempty_bar(acc));
+        else if (g.epi & EPI_SWIGLU) epi_direct<1>(g, it, taddr, wst, quarter, part, lane, bias_reg, tempty_bar(acc));
+        else epi_direct<0>(g, it, taddr, wst, quarter, part, lane, bias_reg, tempty_bar(acc));
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
