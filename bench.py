@@ -501,9 +501,10 @@ def run_micro(args):
         B = args.m or 128
         srv = server.Server(device=0, workspace_bytes=2 << 30)
         inst = W.Instance(srv, synth.make_decoder(seed=2, device=dev, **cfgm), E.CAT_FS, B, seed=21, kv_lo=lo, kv_hi=hi)
-        srv.ctx.epara_set_profile(True)
         times = []
-        for i in range(args.steps + 3):
+        for i in range(args.steps + 4):
+            if i == args.steps + 3:
+                srv.ctx.epara_set_profile(True)      # one more step, bracketed per launch, for the per-kind split
             flush.zero_()
             inst.submit_all(srv.ctx)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -513,7 +514,7 @@ def run_micro(args):
             torch.cuda.synchronize()
             for t in inst.tickets:
                 srv.ctx.epara_collect(t)
-            if i >= 3:
+            if 3 <= i < args.steps + 3:
                 times.append(e0.elapsed_time(e1))
         prof = srv.ctx.epara_step_profile()
         ms = sorted(times)[len(times) // 2]

@@ -233,7 +233,8 @@ size_t epara_gemm_scratch_bytes_for(const epara_gemm_problem* problems, int n);
 /* Split-KV paged decode attention with GQA (one layer).  q: bf16 [B, q_stride] (head h at
  * column h*hd); kv_layer: bf16 [pages][2][Hkv][16][hd]; kv_lens int32 [B] = tokens to attend
  * (cached + appended); tables: int32 [B, table_stride]; out bf16 [B, Hq*hd];
- * scratch: at least epara_decode_attention_scratch_bytes(B, Hq, hd, max_len) bytes. */
+ * scratch: at least epara_decode_attention_scratch_bytes(B, Hq, hd, max_len) bytes (request table,
+ * fp32 chunk partials, chunk counters; the call clears the counters itself). */
 int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
                            const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out,
                            int B, int Hq, int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes);
@@ -252,13 +253,15 @@ size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len);
  * held until the process exits.  It calls no cudaMalloc, cudaFree or any allocating routine.
  *
  * Same kernels, same results as epara_decode_attention.  Arguments as there, minus scratch.
- * Returns EPARA_E_RESOURCE when 256 + roundup256(16 B) + B*Hq*ceil(max_len/256)*(hd+2)*4 bytes exceed
- * EPARA_STATIC_SCRATCH_BYTES (nothing is launched), INVALID / UNSUPPORTED / CUDA as the other entry.
+ * Returns EPARA_E_RESOURCE when 256 + roundup256(16 B) + roundup256(B*Hq*ceil(max_len/256)*(hd+2)*4) +
+ * 4*B*Hq bytes exceed EPARA_STATIC_SCRATCH_BYTES (nothing is launched), INVALID / UNSUPPORTED / CUDA as
+ * the other entry.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and caches
  * it; make that first call outside any stream capture.  All calls on a device share the one array,
- * which keeps whatever the previous call left in it (nothing needs to start at zero: every byte
- * that is read is written first by the same call).  Two calls whose kernels may overlap on the GPU
+ * which keeps whatever the previous call left in it: the request table and the partials are written
+ * before they are read, and the per-(request, kv head) chunk counters, the one part that must start
+ * at zero, are cleared on the stream by every call.  Two calls whose kernels may overlap on the GPU
  * -- different streams without an ordering between them -- race on that array; order them. */
 #define EPARA_STATIC_SCRATCH_BYTES (8u << 20)
 int epara_decode_attention_static(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,

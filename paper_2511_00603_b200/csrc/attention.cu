@@ -5,8 +5,8 @@
 // all G query heads that share the kv head, so every K/V byte is read once.  The chunk size is
 // a constant, hence a request's reduction order never depends on what else is in the step.
 // A page's (K or V, head) tile is 16 x hd contiguous bf16; a warp reads it with 128-bit loads,
-// lanes covering consecutive 16-byte pieces.  Partials (m, l, o) go to scratch and a second
-// kernel merges the chunks in order.
+// lanes covering consecutive 16-byte pieces.  Partials (m, l, o) go to scratch; the block of a
+// (request, kv head) that finishes last merges the chunks in chunk order (finish_chunk).
 //
 // Encoder (ViT): full bidirectional attention of T tokens per (image, head).
 #include <cstring>
@@ -24,8 +24,95 @@ __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
   return v;
 }
 
+// Merge of the chunk partials of one (request, query head) element e, in chunk order.  Every load is
+// independent of the running sums: unrolled, they are all in flight together.
+template <int HD>
+__device__ __forceinline__ float merge_chunks(const float* p, int n_chunks, int e) {
+  float mm = -1e30f;
+#pragma unroll 8
+  for (int ch = 0; ch < n_chunks; ++ch) mm = fmaxf(mm, __ldcg(p + (size_t)ch * (HD + 2)));
+  float ll = 0.f, oo = 0.f;
+#pragma unroll 8
+  for (int ch = 0; ch < n_chunks; ++ch) {
+    const float* pc = p + (size_t)ch * (HD + 2);
+    const float a = exp2f(__ldcg(pc) - mm);
+    ll += __ldcg(pc + 1) * a;
+    oo += __ldcg(pc + 2 + e) * a;
+  }
+  return oo / ll;
+}
+
+// Last step of a decode-attention block: the four warps' (m, l, o) of this chunk sit in shared
+// memory.  They are merged in warp order.  A request of a single chunk is finished right here.
+// Otherwise the chunk's partial goes to scratch.  With `fused` a per-(request, kv head) counter is
+// bumped and the block that arrives last (no block waits for another) merges all chunks in chunk
+// order, writes the output and leaves the counter at zero for the next launch; without it a second
+// kernel (attn_combine_kernel) does the same merge.  The arithmetic and its order are the same in both
+// cases, so the result depends neither on which block is last nor on the mode.
 template <int HD, int G>
-__global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __restrict__ groups, int n_groups) {
+__device__ __forceinline__ void finish_chunk(const AttnDecGroup& g, int b, int kvh, int chunk, int len, int fused,
+                                             const float (*sm_m)[G], const float (*sm_l)[G],
+                                             const float (*sm_o)[G][HD]) {
+  __shared__ int s_last;
+  const int n_chunks = (len + ATTN_CHUNK - 1) / ATTN_CHUNK;
+  for (int idx = threadIdx.x; idx < G * HD; idx += 128) {
+    const int h = idx / HD, e = idx % HD;
+    float mm = sm_m[0][h];
+#pragma unroll
+    for (int w = 1; w < 4; ++w) mm = fmaxf(mm, sm_m[w][h]);
+    float ll = 0.f, oo = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float a = exp2f(sm_m[w][h] - mm);
+      ll += sm_l[w][h] * a;
+      oo += sm_o[w][h][e] * a;
+    }
+    if (n_chunks == 1) {
+      g.out[((size_t)b * g.Hq + (kvh * G + h)) * HD + e] = f2bf(oo / ll);
+    } else {
+      float* dst = g.partial + (((size_t)b * g.Hq + (kvh * G + h)) * g.max_chunks + chunk) * (HD + 2);
+      __stcg(dst + 2 + e, oo);
+      if (e == 0) { __stcg(dst, mm); __stcg(dst + 1, ll); }
+    }
+  }
+  if (n_chunks == 1 || !fused) return;
+  __syncthreads();                      // all partials of the block are written ...
+  if (threadIdx.x == 0) {
+    __threadfence();                    // ... and visible device-wide before the arrival is counted
+    int* cnt = g.counters + (size_t)b * g.Hkv + kvh;
+    const int last = (atomicAdd(cnt, 1) == n_chunks - 1);
+    if (last) atomicExch(cnt, 0);
+    s_last = last;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int idx = threadIdx.x; idx < G * HD; idx += 128) {
+    const int h = idx / HD, e = idx % HD;
+    const float* p = g.partial + ((size_t)b * g.Hq + (kvh * G + h)) * g.max_chunks * (HD + 2);
+    g.out[((size_t)b * g.Hq + (kvh * G + h)) * HD + e] = f2bf(merge_chunks<HD>(p, n_chunks, e));
+  }
+}
+
+// Separate merge for launches with many blocks: one block per (query head, request) of more than one chunk.
+template <int HD>
+__global__ void __launch_bounds__(HD) attn_combine_kernel(const AttnDecGroup* __restrict__ groups, int n_groups) {
+  pdl_launch_dependents();
+  int gi = 0;
+  for (int i = 1; i < n_groups; ++i) if ((int)blockIdx.y >= groups[i].req_start) gi = i;
+  const AttnDecGroup& g = groups[gi];
+  const int b = blockIdx.y - g.req_start, hq = blockIdx.x;
+  pdl_wait();
+  if (hq >= g.Hq) return;
+  const int n_chunks = (g.reqs[b].len + ATTN_CHUNK - 1) / ATTN_CHUNK;
+  if (n_chunks == 1) return;            // finished by the attention kernel itself
+  const float* p = g.partial + ((size_t)b * g.Hq + hq) * g.max_chunks * (HD + 2);
+  const int e = threadIdx.x;
+  g.out[((size_t)b * g.Hq + hq) * HD + e] = f2bf(merge_chunks<HD>(p, n_chunks, e));
+}
+
+template <int HD, int G>
+__global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __restrict__ groups, int n_groups, int fused) {
   constexpr int LPT = HD / 8;        // lanes per token row
   constexpr int TPW = 32 / LPT;      // tokens per warp-wide load
   constexpr int NL = 16 / TPW;       // loads per page tile
@@ -37,6 +124,9 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __
   const int b = blockIdx.z - g.req_start;
   const int kvh = blockIdx.y;
   if (kvh >= g.Hkv) return;
+  if (g.reqs_stable && blockIdx.x * ATTN_CHUNK >= g.reqs[b].len) return;   // nothing to do and nothing to wait for
+  pdl_launch_dependents();
+  pdl_wait();                 // q, the appended K/V row and (single-kernel entry) the request table come from earlier kernels
   const AttnReq rq = g.reqs[b];
   const int chunk = blockIdx.x;
   const int t_begin = chunk * ATTN_CHUNK;
@@ -149,22 +239,7 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __
     }
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < G * HD; idx += 128) {
-    const int h = idx / HD, e = idx % HD;
-    float mm = sm_m[0][h];
-#pragma unroll
-    for (int w = 1; w < 4; ++w) mm = fmaxf(mm, sm_m[w][h]);
-    float ll = 0.f, oo = 0.f;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float a = exp2f(sm_m[w][h] - mm);
-      ll += sm_l[w][h] * a;
-      oo += sm_o[w][h][e] * a;
-    }
-    float* dst = g.partial + (((size_t)b * g.Hq + (kvh * G + h)) * g.max_chunks + chunk) * (HD + 2);
-    dst[2 + e] = oo;
-    if (e == 0) { dst[0] = mm; dst[1] = ll; }
-  }
+  finish_chunk<HD, G>(g, b, kvh, chunk, rq.len, fused, sm_m, sm_l, sm_o);
 }
 
 // Tensor-core variant for hd 64 / 128.  Same work split (chunk, kv head, request; 4 warps, warp w
@@ -200,7 +275,7 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t* r, uint32_t addr) {
 }
 
 template <int HD, int G, int NSLOT>
-__global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup* __restrict__ groups, int n_groups) {
+__global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup* __restrict__ groups, int n_groups, int fused) {
   constexpr int ROWB = HD * 2;              // bytes per token row
   constexpr int TILE = 16 * ROWB;           // bytes per (K or V) page tile
   constexpr int CPR = HD / 8;               // 16-byte pieces per row
@@ -214,6 +289,9 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
   const int b = blockIdx.z - g.req_start;
   const int kvh = blockIdx.y;
   if (kvh >= g.Hkv) return;
+  if (g.reqs_stable && blockIdx.x * ATTN_CHUNK >= g.reqs[b].len) return;   // nothing to do and nothing to wait for
+  pdl_launch_dependents();
+  pdl_wait();                 // q, the appended K/V row and (single-kernel entry) the request table come from earlier kernels
   const AttnReq rq = g.reqs[b];
   const int chunk = blockIdx.x;
   const int t_begin = chunk * ATTN_CHUNK;
@@ -355,86 +433,54 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
     }
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < G * HD; idx += 128) {
-    const int h = idx / HD, e = idx % HD;
-    float mm = sm_m[0][h];
-#pragma unroll
-    for (int w = 1; w < 4; ++w) mm = fmaxf(mm, sm_m[w][h]);
-    float ll = 0.f, oo = 0.f;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float a = exp2f(sm_m[w][h] - mm);
-      ll += sm_l[w][h] * a;
-      oo += sm_o[w][h][e] * a;
-    }
-    float* dst = g.partial + (((size_t)b * g.Hq + (kvh * G + h)) * g.max_chunks + chunk) * (HD + 2);
-    dst[2 + e] = oo;
-    if (e == 0) { dst[0] = mm; dst[1] = ll; }
-  }
-}
-
-// One block per (query head, request): merges the chunk partials in chunk order.
-__global__ void attn_combine_kernel(const AttnDecGroup* __restrict__ groups, int n_groups) {
-  int gi = 0;
-  for (int i = 1; i < n_groups; ++i) if ((int)blockIdx.y >= groups[i].req_start) gi = i;
-  const AttnDecGroup& g = groups[gi];
-  const int b = blockIdx.y - g.req_start, hq = blockIdx.x;
-  if (hq >= g.Hq) return;
-  const int HD = g.hd;
-  const int n_chunks = (g.reqs[b].len + ATTN_CHUNK - 1) / ATTN_CHUNK;
-  const float* p = g.partial + ((size_t)b * g.Hq + hq) * g.max_chunks * (HD + 2);
-  float mm = -1e30f;
-  for (int ch = 0; ch < n_chunks; ++ch) mm = fmaxf(mm, p[(size_t)ch * (HD + 2)]);
-  for (int e = threadIdx.x; e < HD; e += blockDim.x) {
-    float ll = 0.f, oo = 0.f;
-    for (int ch = 0; ch < n_chunks; ++ch) {
-      const float* pc = p + (size_t)ch * (HD + 2);
-      const float a = exp2f(pc[0] - mm);
-      ll += pc[1] * a;
-      oo += pc[2 + e] * a;
-    }
-    g.out[((size_t)b * g.Hq + hq) * HD + e] = f2bf(oo / ll);
-  }
+  finish_chunk<HD, G>(g, b, kvh, chunk, rq.len, fused, sm_m, sm_l, sm_o);
 }
 
 template <int HD, int G>
 static cudaError_t launch_dec_mma(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_chunks,
-                                  cudaStream_t st) {
+                                  int fused, cudaStream_t st) {
   constexpr int NSLOT = 2;                           // pages in flight per warp
   constexpr int SMEM = 4 * NSLOT * 2 * 16 * HD * 2;  // 4 warps x NSLOT pages x (K + V) tiles
   cudaError_t e = cudaFuncSetAttribute(attn_decode_mma_kernel<HD, G, NSLOT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
-  attn_decode_mma_kernel<HD, G, NSLOT><<<dim3(max_chunks, max_Hkv, total_B), 128, SMEM, st>>>(groups, n_groups);
-  return cudaGetLastError();
+  return launch_pdl(attn_decode_mma_kernel<HD, G, NSLOT>, dim3(max_chunks, max_Hkv, total_B), dim3(128), SMEM, st, groups, n_groups, fused);
 }
 
 template <int HD, int G>
 static cudaError_t launch_dec(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_chunks,
-                              cudaStream_t st) {
-  attn_decode_kernel<HD, G><<<dim3(max_chunks, max_Hkv, total_B), 128, 0, st>>>(groups, n_groups);
-  return cudaGetLastError();
+                              int fused, cudaStream_t st) {
+  return launch_pdl(attn_decode_kernel<HD, G>, dim3(max_chunks, max_Hkv, total_B), dim3(128), 0, st, groups, n_groups, fused);
 }
 
-cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_chunks,
-                               int hd, int gqa, cudaStream_t st) {
+// Few blocks (up to two waves): the last block of a (request, kv head) merges the chunks itself and the
+// step saves a launch.  Many blocks: the counter round trip at the end of every block costs more than
+// a second kernel, so the merge runs as attn_combine_kernel.
+bool attn_decode_fused(int total_B, int max_Hkv, int max_chunks, int sm_count) {
+  return (long long)total_B * max_Hkv * max_chunks <= 10ll * sm_count;
+}
+
+cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_Hq,
+                               int max_chunks, int hd, int gqa, int fused, cudaStream_t st) {
   if (n_groups == 0 || total_B == 0) return cudaSuccess;
   if (total_B > 65535 || max_Hkv > 65535) return cudaErrorInvalidValue;
-#define EPARA_DEC(HD_, G_) if (hd == HD_ && gqa == G_) return launch_dec<HD_, G_>(groups, n_groups, total_B, max_Hkv, max_chunks, st);
-#define EPARA_DEC_MMA(HD_, G_) if (hd == HD_ && gqa == G_) return launch_dec_mma<HD_, G_>(groups, n_groups, total_B, max_Hkv, max_chunks, st);
+  cudaError_t e = cudaErrorInvalidValue;
+#define EPARA_DEC(HD_, G_) if (hd == HD_ && gqa == G_) e = launch_dec<HD_, G_>(groups, n_groups, total_B, max_Hkv, max_chunks, fused, st);
+#define EPARA_DEC_MMA(HD_, G_) if (hd == HD_ && gqa == G_) e = launch_dec_mma<HD_, G_>(groups, n_groups, total_B, max_Hkv, max_chunks, fused, st);
   EPARA_DEC_MMA(64, 1) EPARA_DEC_MMA(64, 2) EPARA_DEC_MMA(64, 4) EPARA_DEC_MMA(64, 8)
   EPARA_DEC_MMA(128, 1) EPARA_DEC_MMA(128, 2) EPARA_DEC_MMA(128, 4) EPARA_DEC_MMA(128, 8)
 #undef EPARA_DEC_MMA
   EPARA_DEC(16, 1) EPARA_DEC(16, 2) EPARA_DEC(16, 4)
   EPARA_DEC(32, 1) EPARA_DEC(32, 2) EPARA_DEC(32, 4)
 #undef EPARA_DEC
+  if (e != cudaSuccess || fused || max_chunks <= 1) return e;
+  const dim3 grid(max_Hq, total_B);
+  switch (hd) {
+    case 16: return launch_pdl(attn_combine_kernel<16>, grid, dim3(16), 0, st, groups, n_groups);
+    case 32: return launch_pdl(attn_combine_kernel<32>, grid, dim3(32), 0, st, groups, n_groups);
+    case 64: return launch_pdl(attn_combine_kernel<64>, grid, dim3(64), 0, st, groups, n_groups);
+    case 128: return launch_pdl(attn_combine_kernel<128>, grid, dim3(128), 0, st, groups, n_groups);
+  }
   return cudaErrorInvalidValue;
-}
-
-cudaError_t launch_attn_combine(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hq, int hd,
-                                cudaStream_t st) {
-  if (n_groups == 0 || total_B == 0) return cudaSuccess;
-  attn_combine_kernel<<<dim3(max_Hq, total_B), hd < 32 ? 32 : hd, 0, st>>>(groups, n_groups);
-  return cudaGetLastError();
 }
 
 __global__ void attn_fill_reqs_kernel(AttnReq* reqs, const int32_t* kv_lens, const int32_t* tables, int stride, int B) {
@@ -476,9 +522,11 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, uint32_t addr) {
 __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const AttnEncGroup* __restrict__ groups, int n_groups) {
   constexpr int HD = 64;
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_launch_dependents();
   int gi = 0;
   for (int i = 1; i < n_groups; ++i) if ((int)blockIdx.x >= groups[i].blk_start) gi = i;
   const AttnEncGroup& g = groups[gi];
+  pdl_wait();
   const int local = blockIdx.x - g.blk_start;
   const int qb = local % g.q_blocks, bh = local / g.q_blocks;
   const int h = bh % g.H, b = bh / g.H;
@@ -544,12 +592,15 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
     }
     __syncthreads();
     if (!active) continue;
+    // the last block of keys is ragged (197 = 3 x 64 + 5): only its 16-key groups that hold real keys are computed
+    const int np_lim = (min(64, T - kb) + 15) >> 4;
     float sc[8][4];
 #pragma unroll
     for (int n = 0; n < 8; ++n) { sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f; }
     // S = Q K^T : for key tiles (pairs of 8 keys) and k-steps
 #pragma unroll
     for (int np = 0; np < 4; ++np) {        // key tiles 2np, 2np+1
+      if (np >= np_lim) continue;
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {
         // matrices: (keys 2np*8.., k lo), (keys 2np*8.., k hi), (keys (2np+1)*8.., k lo), (.., k hi)
@@ -585,6 +636,7 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
     uint32_t pa[4][4];                       // P as A fragments: 4 k-steps of 16 keys
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
+      if ((n >> 1) >= np_lim) continue;      // all keys of the group are masked: never read below
       const float p0 = exp2f(sc[n][0] - m_lo), p1 = exp2f(sc[n][1] - m_lo);
       const float p2 = exp2f(sc[n][2] - m_hi), p3 = exp2f(sc[n][3] - m_hi);
       l_lo += p0 + p1;
@@ -595,6 +647,7 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
     // O += P V : k = keys (4 steps of 16), n = head dims (8 tiles of 8)
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks) {
+      if (ks >= np_lim) continue;
 #pragma unroll
       for (int np = 0; np < 4; ++np) {      // dim tiles 2np, 2np+1
         // matrices: (keys lo 8, dims 2np*8..), (keys hi 8, dims 2np*8..), (keys lo, dims (2np+1)*8..), (keys hi, ..)
@@ -634,8 +687,7 @@ cudaError_t launch_attn_encoder(const AttnEncGroup* groups, int n_groups, int to
   if (e != cudaSuccess) return e;
   const int rows = max_T < ENC_ROWS ? max_T : ENC_ROWS;
   const int warps = (rows + 15) / 16;
-  attn_encoder_kernel<<<total_blocks, warps * 32, smem, st>>>(groups, n_groups);
-  return cudaGetLastError();
+  return launch_pdl(attn_encoder_kernel, dim3(total_blocks), dim3(warps * 32), smem, st, groups, n_groups);
 }
 
 }  // namespace epara
@@ -662,7 +714,8 @@ extern "C" int epara_decode_attention_static(int device, void* cuda_stream, cons
   if (device < 0 || device >= MAX_DEVICES) return EPARA_E_INVALID;
   const int chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK;
   const size_t req_bytes = ((size_t)B * sizeof(AttnReq) + 255) / 256 * 256;
-  const size_t need = 256 + req_bytes + (size_t)B * Hq * chunks * (hd + 2) * sizeof(float);
+  const size_t part_bytes = ((size_t)B * Hq * chunks * (hd + 2) * sizeof(float) + 255) / 256 * 256;
+  const size_t need = 256 + req_bytes + part_bytes + (size_t)B * Hq * sizeof(int);
   if (need > STATIC_SCRATCH_BYTES) return EPARA_E_RESOURCE;   // problem too large for the built-in scratch
   if (B == 0) return EPARA_OK;
   if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
@@ -679,15 +732,17 @@ extern "C" int epara_decode_attention_static(int device, void* cuda_stream, cons
   AttnReq* reqs = reinterpret_cast<AttnReq*>(s + 256);
   g.q = (const bf16*)q; g.q_stride = q_stride; g.kv_layer = (const bf16*)kv_layer; g.reqs = reqs; g.out = (bf16*)out;
   g.partial = reinterpret_cast<float*>(s + 256 + req_bytes);
+  g.counters = reinterpret_cast<int*>(s + 256 + req_bytes + part_bytes);
   g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = chunks; g.req_start = 0;
-  // Nothing in the scratch has to start at zero: the descriptor and the request table are rewritten
-  // here, and every partial the combine kernel reads is written by the decode kernel of this call.
+  // The array keeps the previous call's contents.  The descriptor and the request table are rewritten
+  // here and every partial that is read is written first by this call's kernel; only the chunk
+  // counters must start at zero, so they are cleared on the stream before the kernel.
+  if (cudaMemsetAsync(g.counters, 0, (size_t)B * Hq * sizeof(int), st) != cudaSuccess) return EPARA_E_CUDA;
   if (cudaMemcpyAsync(s, &g, sizeof(g), cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
   launch_attn_fill_reqs(reqs, kv_lens, tables, table_stride, B, st);
-  cudaError_t e = launch_attn_decode(reinterpret_cast<const AttnDecGroup*>(s), 1, B, Hkv, chunks, hd, Hq / Hkv, st);
+  cudaError_t e = launch_attn_decode(reinterpret_cast<const AttnDecGroup*>(s), 1, B, Hkv, Hq, chunks, hd, Hq / Hkv,
+                                     attn_decode_fused(B, Hkv, chunks, 148) ? 1 : 0, st);
   if (e == cudaErrorInvalidValue) return EPARA_E_UNSUPPORTED;
-  if (e != cudaSuccess) return EPARA_E_CUDA;
-  e = launch_attn_combine(reinterpret_cast<const AttnDecGroup*>(s), 1, B, Hq, hd, st);
   return e == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
 }
 

@@ -6,6 +6,35 @@
 
 namespace epara {
 
+// Programmatic dependent launch.  Every kernel of a step is launched with programmatic stream
+// serialisation: it may become resident while the kernel before it in the stream is still running,
+// which hides launch latency and set-up.  pdl_launch_dependents() lets the next kernel start
+// launching; pdl_wait() returns once all earlier kernels have completed and their writes are
+// visible.  Rule: a kernel touches nothing that an earlier kernel of the stream writes or reads
+// before its pdl_wait(); weights and the step's descriptors (uploaded by a copy that completes
+// before the first kernel) may be read earlier.  Every kernel waits at least once, so completion
+// is transitive along the stream.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// (one thread per block is enough; a block that exits counts as having triggered)
+__device__ __forceinline__ void pdl_launch_dependents() {
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ float bf2f(bf16 v) { return __bfloat162float(v); }
 __device__ __forceinline__ bf16 f2bf(float v) { return __float2bfloat16_rn(v); }
 

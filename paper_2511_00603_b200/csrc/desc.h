@@ -48,7 +48,9 @@ struct alignas(64) GemmGroup {
   float* partial;  // [ksplit][tiles_m * 128][tiles_n * bn] fp32, ksplit > 1 only
   int* counters;   // [tiles_m * tiles_n], zero between launches
   int c_rows;      // row extent of tmC (rows at and beyond it are never written)
-  int pad0, pad1, pad2;
+  int stream;      // 1: at most 16 rows ever, runs in the weight-streaming kernel (16 W rows per block,
+                   // tiles_n = ceil(N / 16), no TMA maps); 0: tensor-core tiles
+  int pad1, pad2;
 };
 
 struct GemmLaunch {      // header followed by groups
@@ -82,7 +84,7 @@ struct RopeGroup {
   bf16* qkv;             // [B, (Hq+2Hkv)*hd], q rotated in place
   bf16* kv_layer;        // [pages][2][Hkv][16][hd]
   const ReqDesc* reqs;
-  const double* inv_freq;  // [hd/2]
+  const float2* cs;      // [max position + 1][hd/2]: (cos, sin) of position * 10000^(-2j/hd)
   int B, Hq, Hkv, hd;
 };
 
@@ -97,12 +99,14 @@ struct AttnDecGroup {
   const bf16* kv_layer;
   const AttnReq* reqs;
   bf16* out;             // [B, Hq*hd]
-  float* partial;        // [B][Hq][max_chunks][hd + 2]  (m, l, o[hd])
+  float* partial;        // [B][Hq][max_chunks][hd + 2]  (m, l, o[hd]); requests of more than one chunk
+  int* counters;         // [B][Hkv] chunks that have arrived; zero between launches
   int q_stride;
   int B, Hq, Hkv, hd;
   int max_chunks;
   int req_start;         // first grid.z index of this group
-  int pad;
+  int reqs_stable;       // 1: `reqs` was uploaded before the step's first kernel (a block past a request's
+                         // length may leave without the dependency wait); 0: an earlier kernel writes it
 };
 
 struct AttnEncGroup {

@@ -182,6 +182,7 @@ struct Builder {
   size_t need;
   bool fail;
   int sm_count;
+  int gemm_impl;
   void* get(size_t bytes) {
     if (!c) { carve_size(need, bytes); return reinterpret_cast<void*>(size_t(256)); }
     void* p = carve(c, bytes);
@@ -193,6 +194,7 @@ struct Builder {
 bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap, const void* W, int N, int K,
               void* C, int ldc, const void* bias, int epi, int rows_per_req) {
   const int sm_count = bl.sm_count;
+  const long long max_rows = (long long)m->max_batch * rows_per_req;   // the most rows this op ever sees
   Op op;
   memset(&op, 0, sizeof(op));
   op.kind = EPARA_K_GEMM;
@@ -202,12 +204,15 @@ bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap,
   g.N = N; g.K = K; g.lda = lda; g.ldw = K; g.ldc = ldc; g.epi = epi | (bias ? EPI_BIAS : 0);
   op.weight_bytes = 2.0 * N * K;
   gemm_tc_config(rows_cap, N, K, g.epi, sm_count, &g.bn, &g.ksplit);
+  if (max_rows <= GEMM_STREAM_MAX_ROWS && bl.gemm_impl == EPARA_GEMM_TCGEN05) {
+    g.stream = 1; g.bn = 16; g.ksplit = 1;
+  }
   if (g.ksplit > 1) {
     const size_t tiles_m = (size_t)((rows_cap + TC_BM - 1) / TC_BM), tiles_n = (size_t)((N + g.bn - 1) / g.bn);
     m->splitk_bytes = std::max(m->splitk_bytes, (size_t)g.ksplit * tiles_m * TC_BM * tiles_n * g.bn * 4);
     m->splitk_tiles = std::max(m->splitk_tiles, tiles_m * tiles_n);
   }
-  if (bl.c) {
+  if (bl.c && !g.stream) {
     if (!make_tmap(&g.tmA, A, rows_cap, K, lda, TC_BM)) return false;
     if (!make_tmap(&g.tmW, W, N, K, K, g.bn)) return false;
     if (!make_tmap_c(&g.tmC, C, rows_cap, N, ldc, g.epi)) return false;
@@ -364,12 +369,22 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
   const int ldl = round_up(d.vocab, 8);
   bf16* logits = (bf16*)bl.get((size_t)Bcap * ldl * 2);
   float* partial = (float*)bl.get((size_t)B * Hq * m->max_chunks * (hd + 2) * 4);
-  double* inv_freq = (double*)bl.get((size_t)(hd / 2) * 8);
+  int* chunk_counters = (int*)bl.get((size_t)B * Hkv * sizeof(int));
+  float2* rope_cs = (float2*)bl.get((size_t)(d.max_kv_len + 1) * (hd / 2) * sizeof(float2));
   if (bl.fail) return EPARA_E_RESOURCE;
   if (bl.c) {
-    std::vector<double> f64(hd / 2);
-    for (int j = 0; j < hd / 2; ++j) f64[j] = std::pow(10000.0, -2.0 * j / hd);
-    if (cudaMemcpy(inv_freq, f64.data(), f64.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess) return EPARA_E_CUDA;
+    // rotation table: angles in fp64 on the host, (cos, sin) rounded once to fp32
+    const int half = hd / 2;
+    std::vector<double> inv_freq(half);
+    for (int j = 0; j < half; ++j) inv_freq[j] = std::pow(10000.0, -2.0 * j / hd);
+    std::vector<float2> cs((size_t)(d.max_kv_len + 1) * half);
+    for (int p = 0; p <= d.max_kv_len; ++p)
+      for (int j = 0; j < half; ++j) {
+        const double ang = (double)p * inv_freq[j];
+        cs[(size_t)p * half + j] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+      }
+    if (cudaMemcpy(rope_cs, cs.data(), cs.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess) return EPARA_E_CUDA;
+    if (cudaMemset(chunk_counters, 0, (size_t)B * Hkv * sizeof(int)) != cudaSuccess) return EPARA_E_CUDA;
   }
   Op g;
   memset(&g, 0, sizeof(g));
@@ -385,14 +400,16 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
     Op r;
     memset(&r, 0, sizeof(r));
     r.kind = EPARA_K_ROPE; r.rows_per_req = 1;
-    r.rope.qkv = qkv; r.rope.kv_layer = kv_layer; r.rope.inv_freq = inv_freq;
+    r.rope.qkv = qkv; r.rope.kv_layer = kv_layer; r.rope.cs = rope_cs;
     r.rope.Hq = Hq; r.rope.Hkv = Hkv; r.rope.hd = hd;
     m->ops.push_back(r);
     Op at;
     memset(&at, 0, sizeof(at));
     at.kind = EPARA_K_ATTN_DEC; at.rows_per_req = 1;
     at.adec.q = qkv; at.adec.q_stride = nq; at.adec.kv_layer = kv_layer; at.adec.out = a; at.adec.partial = partial;
+    at.adec.counters = chunk_counters;
     at.adec.Hq = Hq; at.adec.Hkv = Hkv; at.adec.hd = hd; at.adec.max_chunks = m->max_chunks;
+    at.adec.reqs_stable = 1;
     m->ops.push_back(at);
     if (!add_gemm(bl, m, a, Hq * hd, Bcap, w[2], dm, Hq * hd, x, dm, nullptr, EPI_RESID_F32, 1)) return EPARA_E_CUDA;
     add_norm(m, x, dm, h, w[3], nullptr, dm, NORM_RMS, 1e-5f, 1);
@@ -511,7 +528,7 @@ size_t epara_model_workspace_bytes(const epara_config* cfg, const epara_model_de
   m.tensors.assign(d->tensors, d->tensors + d->n_tensors);
   if (d->kind == EPARA_MODEL_MLP) m.dims.assign(d->mlp_dims, d->mlp_dims + d->n_layers + 1);
   m.max_batch = effective_max_batch(*cfg, *d);
-  Builder bl{nullptr, 0, false, 148};
+  Builder bl{nullptr, 0, false, 148, cfg->gemm_impl};
   build_model(bl, &m, *cfg);
   finish_model(bl, &m);
   return bl.need + 256;
@@ -589,7 +606,7 @@ int epara_register_model(epara_ctx* c, const epara_model_desc* d, int* model_id)
   m->max_chunks = 0;
   m->kv_bytes_per_token = 0;
   const size_t mark = c->ws_used;
-  Builder bl{c, 0, false, c->sm_count};
+  Builder bl{c, 0, false, c->sm_count, c->cfg.gemm_impl};
   int r = build_model(bl, m, c->cfg);
   if (r == EPARA_OK) r = finish_model(bl, m);
   if (r != EPARA_OK) {
@@ -734,10 +751,16 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
         if (a.cursor < a.m->ops.size() && a.m->ops[a.cursor].kind == kind) who.push_back(&a);
       if (who.empty()) continue;
       more = true;
+      // GEMM groups go out in up to two launches: tensor-core tiles (pass 0) and the weight-streaming
+      // kernel for groups that never exceed 16 rows (pass 1)
+      const int n_pass = (kind == EPARA_K_GEMM) ? 2 : 1;
+      for (int pass = 0; pass < n_pass; ++pass) {
       Launch L;
       memset(&L, 0, sizeof(L));
       L.kind = kind;
       L.n_groups = (int)who.size();
+      L.p2 = pass;
+      int n_put = 0;
       off = align_up(off, 64);
       L.off = off;
       if (kind == EPARA_K_ATTN_DEC) {
@@ -766,11 +789,8 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
               max_chunks = std::max(max_chunks, (a->reqs[b].in.kv_len + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK);
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
           }
-          LL.p0 = total_B; LL.p1 = max_hkv; LL.p2 = max_chunks; LL.p3 = (hd << 8) | G;
+          LL.p0 = total_B; LL.p1 = max_hkv | (max_hq << 16); LL.p2 = max_chunks; LL.p3 = (hd << 8) | G;
           launches.push_back(LL);
-          Launch LC = LL;
-          LC.kind = EPARA_K_ATTN_COMBINE; LC.p1 = max_hq;
-          launches.push_back(LC);
           rest.swap(other);
         }
         for (Active* a : who) a->cursor++;
@@ -804,11 +824,21 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           }
           case EPARA_K_GEMM: {
             GemmGroup g = op.gemm;
+            if ((g.stream != 0) != (pass == 1)) break;         // the other pass takes it
             g.M = rows;
-            const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : g.bn;
-            g.tiles_m = (rows + tm - 1) / tm; g.tiles_n = (g.N + tn - 1) / tn;
-            g.tile_start = total;
-            total += g.tiles_m * g.tiles_n * (simt ? 1 : g.ksplit);
+            if (g.stream) {
+              g.tiles_m = 1; g.tiles_n = gemm_stream_tiles(g.N);
+              g.tile_start = total;
+              total += g.tiles_n;
+              mx = std::max(mx, rows);
+            } else {
+              const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : g.bn;
+              g.tiles_m = (rows + tm - 1) / tm; g.tiles_n = (g.N + tn - 1) / tn;
+              g.tile_start = total;
+              total += g.tiles_m * g.tiles_n * (simt ? 1 : g.ksplit);
+              L.p3 = std::max(L.p3, g.bn);
+            }
+            ++n_put;
             inf.gemm_groups++;
             inf.gemm_flops += 2.0 * rows * g.N * g.K;
             inf.weight_bytes += op.weight_bytes;
@@ -838,10 +868,15 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
             break;
           }
         }
-        a->cursor++;
+        if (pass == n_pass - 1) a->cursor++;
       }
       L.p0 = total; L.p1 = mx;
+      if (kind == EPARA_K_GEMM) {
+        L.n_groups = n_put;
+        if (n_put == 0) continue;
+      }
       launches.push_back(L);
+      }
     }
   }
   if (overflow) {
@@ -866,8 +901,10 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
     slot.prof_kind.clear();
   }
   cudaError_t err = cudaSuccess;
-  int li = 0;
+  int li = 0, n_kernels = 0;
   for (const Launch& L : launches) {
+    n_kernels += 1 + ((L.kind == EPARA_K_ATTN_DEC && L.p2 > 1 &&
+                       !attn_decode_fused(L.p0, L.p1 & 0xffff, L.p2, c->sm_count)) ? 1 : 0);
     const unsigned char* gp = slot.dev + L.off;
     if (prof) { cudaEventRecord(slot.prof[2 * li], st); slot.prof_kind.push_back(L.kind); }
     switch (L.kind) {
@@ -875,15 +912,14 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       case EPARA_K_ASSEMBLE: launch_assemble((const AssembleGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_NORM: launch_norm((const NormGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_GEMM:
-        if (simt) launch_gemm_simt((const GemmGroup*)gp, L.n_groups, L.p0, st);
-        else err = launch_gemm_tc((const GemmGroup*)gp, L.n_groups, L.p0, c->dev_status, c->sm_count, st);
+        if (L.p2 == 1) err = launch_gemm_stream((const GemmGroup*)gp, L.n_groups, L.p0, L.p1, st);
+        else if (simt) launch_gemm_simt((const GemmGroup*)gp, L.n_groups, L.p0, st);
+        else err = launch_gemm_tc((const GemmGroup*)gp, L.n_groups, L.p0, L.p3, c->dev_status, c->sm_count, st);
         break;
       case EPARA_K_ROPE: launch_rope_append((const RopeGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_ATTN_DEC:
-        err = launch_attn_decode((const AttnDecGroup*)gp, L.n_groups, L.p0, L.p1, L.p2, L.p3 >> 8, L.p3 & 255, st);
-        break;
-      case EPARA_K_ATTN_COMBINE:
-        err = launch_attn_combine((const AttnDecGroup*)gp, L.n_groups, L.p0, L.p1, L.p3 >> 8, st);
+        err = launch_attn_decode((const AttnDecGroup*)gp, L.n_groups, L.p0, L.p1 & 0xffff, L.p1 >> 16, L.p2, L.p3 >> 8,
+                                 L.p3 & 255, attn_decode_fused(L.p0, L.p1 & 0xffff, L.p2, c->sm_count) ? 1 : 0, st);
         break;
       case EPARA_K_ATTN_ENC: err = launch_attn_encoder((const AttnEncGroup*)gp, L.n_groups, L.p0, L.p1, st); break;
       case EPARA_K_OUTPUT: launch_output((const OutputGroup*)gp, L.n_groups, L.p1, st); break;
@@ -898,7 +934,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
   slot.busy = true;
   slot.step_id = step_id;
   c->last_step_slot = step_id % N_SLOTS;
-  inf.launches = (int)launches.size();
+  inf.launches = n_kernels;
   if (info) *info = inf;
   return err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
 }
@@ -980,8 +1016,8 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
   if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool simt = impl == EPARA_GEMM_SIMT;
-  std::vector<GemmGroup> gs(n);
-  int total = 0;
+  std::vector<GemmGroup> gs, gs_stream;      // tensor-core (or CUDA-core) groups; weight-streaming groups (M <= 16)
+  int total = 0, total_stream = 0, max_rows_stream = 0;
   size_t soff = epara_gemm_scratch_bytes(n);
   for (int i = 0; i < n; ++i) {
     const epara_gemm_problem& q = p[i];
@@ -992,11 +1028,21 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
       return EPARA_E_INVALID;
     if ((q.epilogue & EPARA_EPI_SWIGLU) && (q.N % 2 || (q.epilogue & EPARA_EPI_RESID_F32))) return EPARA_E_INVALID;
     if ((q.epilogue & EPARA_EPI_BIAS) && !q.bias) return EPARA_E_INVALID;
-    GemmGroup& g = gs[i];
+    GemmGroup g;
     memset(&g, 0, sizeof(g));
     g.A = (const bf16*)q.A; g.W = (const bf16*)q.W; g.C = q.C; g.bias = (const bf16*)q.bias;
     g.M = q.M; g.N = q.N; g.K = q.K; g.lda = q.lda; g.ldw = q.ldw; g.ldc = q.ldc; g.epi = q.epilogue;
     g.bn = 128; g.ksplit = 1;
+    g.c_rows = q.M;
+    if (!simt && q.M <= GEMM_STREAM_MAX_ROWS && q.K % 8 == 0) {
+      g.stream = 1; g.bn = 16;
+      g.tiles_m = 1; g.tiles_n = gemm_stream_tiles(q.N);
+      g.tile_start = total_stream;
+      if (q.M > 0) total_stream += g.tiles_n;
+      max_rows_stream = std::max(max_rows_stream, q.M);
+      gs_stream.push_back(g);
+      continue;
+    }
     if (!simt) gemm_tc_config(q.M, q.N, q.K, q.epilogue, 148, &g.bn, &g.ksplit);
     const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : g.bn;
     g.tiles_m = (q.M + tm - 1) / tm; g.tiles_n = (q.N + tn - 1) / tn;
@@ -1007,7 +1053,6 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
       if (!make_tmap(&g.tmW, q.W, q.N, q.K, q.ldw, g.bn)) return EPARA_E_CUDA;
       if (!make_tmap_c(&g.tmC, q.C, q.M, q.N, q.ldc, q.epilogue)) return EPARA_E_CUDA;
     }
-    g.c_rows = q.M;
     if (g.ksplit > 1) {
       soff = align_up(soff, 256);
       g.partial = (float*)((unsigned char*)scratch + soff);
@@ -1017,28 +1062,39 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
       if (cudaMemsetAsync(g.counters, 0, (size_t)g.tiles_m * g.tiles_n * sizeof(int), st) != cudaSuccess) return EPARA_E_CUDA;
       soff += (size_t)g.tiles_m * g.tiles_n * sizeof(int);
     }
+    gs.push_back(g);
   }
   int* status = (int*)scratch;
   GemmGroup* dev_groups = (GemmGroup*)((unsigned char*)scratch + 256);
+  GemmGroup* dev_stream = dev_groups + gs.size();
   if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) return EPARA_E_CUDA;
-  if (cudaMemcpyAsync(dev_groups, gs.data(), gs.size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
+  // (a copy from pageable host memory is staged before cudaMemcpyAsync returns, so the vectors may go out of scope)
+  if (!gs.empty() &&
+      cudaMemcpyAsync(dev_groups, gs.data(), gs.size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return EPARA_E_CUDA;
-  // (a copy from pageable host memory is staged before cudaMemcpyAsync returns, so gs may go out of scope)
+  if (!gs_stream.empty() &&
+      cudaMemcpyAsync(dev_stream, gs_stream.data(), gs_stream.size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return EPARA_E_CUDA;
   cudaError_t err = cudaSuccess;
   if (simt) {
-    launch_gemm_simt(dev_groups, n, total, st);
+    launch_gemm_simt(dev_groups, (int)gs.size(), total, st);
     err = cudaGetLastError();
   } else {
     int sm = 0;
     cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device);
-    err = launch_gemm_tc(dev_groups, n, total, status, sm, st);
+    int max_bn = 0;
+    for (const GemmGroup& g : gs) max_bn = std::max(max_bn, g.bn);
+    err = launch_gemm_tc(dev_groups, (int)gs.size(), total, max_bn, status, sm, st);
+    if (err == cudaSuccess)
+      err = launch_gemm_stream(dev_stream, (int)gs_stream.size(), total_stream, max_rows_stream, st);
   }
   return err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
 }
 
 size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len) {
   const int chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK;
-  return 256 + align_up((size_t)B * sizeof(AttnReq), 256) + (size_t)B * Hq * chunks * (hd + 2) * 4;
+  return 256 + align_up((size_t)B * sizeof(AttnReq), 256) + align_up((size_t)B * Hq * chunks * (hd + 2) * 4, 256) +
+         (size_t)B * Hq * sizeof(int);
 }
 
 int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
@@ -1056,16 +1112,18 @@ int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_s
   unsigned char* s = (unsigned char*)scratch;
   AttnDecGroup g;
   memset(&g, 0, sizeof(g));
+  const int g_chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK;
   AttnReq* reqs = (AttnReq*)(s + 256);
   g.q = (const bf16*)q; g.q_stride = q_stride; g.kv_layer = (const bf16*)kv_layer; g.reqs = reqs; g.out = (bf16*)out;
   g.partial = (float*)(s + 256 + align_up((size_t)B * sizeof(AttnReq), 256));
+  g.counters = (int*)((unsigned char*)g.partial + align_up((size_t)B * Hq * g_chunks * (hd + 2) * 4, 256));
+  if (cudaMemsetAsync(g.counters, 0, (size_t)B * Hq * sizeof(int), st) != cudaSuccess) return EPARA_E_CUDA;
   g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK; g.req_start = 0;
   if (cudaMemcpyAsync(s, &g, sizeof(g), cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
   launch_attn_fill_reqs(reqs, kv_lens, tables, table_stride, B, st);
-  cudaError_t e = launch_attn_decode((const AttnDecGroup*)s, 1, B, Hkv, g.max_chunks, hd, Hq / Hkv, st);
+  cudaError_t e = launch_attn_decode((const AttnDecGroup*)s, 1, B, Hkv, Hq, g.max_chunks, hd, Hq / Hkv,
+                                     attn_decode_fused(B, Hkv, g.max_chunks, 148) ? 1 : 0, st);
   if (e == cudaErrorInvalidValue) return EPARA_E_UNSUPPORTED;
-  if (e != cudaSuccess) return EPARA_E_CUDA;
-  e = launch_attn_combine((const AttnDecGroup*)s, 1, B, Hq, hd, st);
   return e == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
 }
 

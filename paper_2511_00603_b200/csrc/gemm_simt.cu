@@ -18,6 +18,8 @@ __device__ __forceinline__ int find_group(const GemmGroup* groups, int n, int ti
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmGroup* __restrict__ groups, int n_groups) {
   __shared__ float As[16][SIMT_TILE + 4];
   __shared__ float Ws[16][SIMT_TILE + 4];
+  pdl_launch_dependents();
+  pdl_wait();
   const int gi = find_group(groups, n_groups, blockIdx.x);
   const GemmGroup& g = groups[gi];
   const int local = blockIdx.x - g.tile_start;

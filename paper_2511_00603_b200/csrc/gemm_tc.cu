@@ -26,16 +26,19 @@ namespace epara {
 
 namespace {
 
-constexpr int STAGES = 4;
+// The operand ring holds 192 KB: 4 stages of 48 KB (A 128 x 64 + W 256 x 64) when some group of the
+// launch has 256-wide tiles, 6 stages of 32 KB when all tiles are 128 wide (more loads in flight for
+// the weight-streaming groups).  The geometry is a launch parameter.
+constexpr int MAX_STAGES = 6;
 constexpr int A_BYTES = TC_BM * TC_BK * 2;          // 16 KB
 constexpr int B_BYTES_MAX = TC_BN_MAX * TC_BK * 2;  // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES_MAX;
+constexpr int RING_BYTES = 4 * (A_BYTES + B_BYTES_MAX);
 constexpr int ACC_COLS = TC_BN_MAX;                 // TMEM columns per accumulator
 constexpr int TMEM_COLS = 2 * ACC_COLS;             // 512: the whole TMEM of the SM
 constexpr int EPI_WARPS = 16;
 constexpr int N_THREADS = 64 + EPI_WARPS * 32;
 constexpr int STAGE_OUT_BYTES = EPI_WARPS * 2048;    // epilogue staging: 2 KB (32 rows x 64 bytes) per warp
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + STAGE_OUT_BYTES + 256;
+constexpr size_t SMEM_BYTES = 1024 + (size_t)RING_BYTES + STAGE_OUT_BYTES + 256;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -92,6 +95,8 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, uint32_
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// waits until the bulk stores / reductions of this thread have been performed in global memory
+__device__ __forceinline__ void bulk_wait_done0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tensormap_acquire(const CUtensorMap* tm) {
   asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tm) : "memory");
@@ -410,23 +415,25 @@ __device__ __forceinline__ void epi_direct(const GView& g, const Item& it, uint3
 }
 
 __global__ void __launch_bounds__(N_THREADS, 1)
-gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status) {
+gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status,
+               int STAGES, int STAGE_BYTES) {
   extern __shared__ unsigned char smem_dyn[];
   // 1024-byte aligned tile area (128-byte swizzle atoms are 1024 bytes)
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
-  unsigned char* stage_out = base_ptr + STAGES * STAGE_BYTES;
-  const uint32_t bars = base + STAGES * STAGE_BYTES + STAGE_OUT_BYTES;
+  unsigned char* stage_out = base_ptr + RING_BYTES;
+  const uint32_t bars = base + RING_BYTES + STAGE_OUT_BYTES;
   auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
-  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * STAGE_BYTES + STAGE_OUT_BYTES + 8 * (2 * STAGES + 4));
+  auto empty_bar = [&](int s) { return bars + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * MAX_STAGES + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + RING_BYTES + STAGE_OUT_BYTES + 8 * (2 * MAX_STAGES + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
   volatile int* votes = reinterpret_cast<volatile int*>(tmem_slot + 4);   // one per epilogue warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), EPI_WARPS); }
@@ -445,6 +452,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
 
   if (warp == 0) {
     if (lane != 0) {
+      pdl_wait();
       // ---------------------------------------------------------- L2 prefetch of residual tiles
       // The fp32 residual epilogue reads C before it adds to it; these lanes ask L2 for the C tiles of
       // this CTA's items ahead of time so that those reads do not wait on HBM.
@@ -470,6 +478,31 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
       const GemmGroup* g_prev = nullptr;
       GroupCache gc;
       gc.g = nullptr;
+      // Weights are never written by a kernel: the W tiles of this CTA's first k-blocks (the stages are
+      // all free) are requested before the wait on the earlier kernels of the stream, the A tiles after it.
+      int npre = 0;
+      if ((int)blockIdx.x < total_items) {
+        group_cache(gc, groups, n_groups, blockIdx.x);
+        const GemmGroup* g = gc.g;
+        const Item it = decode_item(gc, blockIdx.x);
+        tensormap_acquire(&g->tmA);
+        tensormap_acquire(&g->tmW);
+        g_prev = g;
+        const uint32_t bytes = A_BYTES + (uint32_t)gc.bn * TC_BK * 2;
+        npre = min(STAGES, it.kb1 - it.kb0);
+        for (int i = 0; i < npre; ++i) {
+          mbar_expect_tx(full_bar(i), bytes);
+          tma_load_2d(base + i * STAGE_BYTES + A_BYTES, &g->tmW, (it.kb0 + i) * TC_BK, it.n0, full_bar(i));
+        }
+        pdl_wait();
+        for (int i = 0; i < npre; ++i) {
+          tma_load_2d(base + i * STAGE_BYTES, &g->tmA, (it.kb0 + i) * TC_BK, it.m0, full_bar(i));
+          issued_mask |= 1u << i;
+        }
+        if (npre == STAGES) { stage = 0; phase = 1u; } else { stage = npre; }
+      } else {
+        pdl_wait();
+      }
       for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
         group_cache(gc, groups, n_groups, item);
         const GemmGroup* g = gc.g;
@@ -480,7 +513,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
           g_prev = g;
         }
         const uint32_t bytes = A_BYTES + (uint32_t)gc.bn * TC_BK * 2;
-        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+        for (int kb = it.kb0 + npre; kb < it.kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 1); break; }
           mbar_expect_tx(full_bar(stage), bytes);
           const uint32_t sa = base + stage * STAGE_BYTES;
@@ -490,6 +523,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
           last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
+        npre = 0;
       }
       if (!ok) {
         *abort_flag = 1;
@@ -535,6 +569,7 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..17)
+    pdl_wait();
     const int ew = warp - 2;
     const int et = threadIdx.x - 64;          // 0..255 among the epilogue threads
     const int quarter = warp & 3;             // TMEM lanes 32*quarter .. +31 belong to this warp
@@ -628,7 +663,9 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
-    if (lane == 0) bulk_wait_read0();       // staged boxes still being read by the TMA unit
+    // The kernel that follows may already be resident and is released the moment this grid completes:
+    // the staged boxes must have reached global memory, not merely have left shared memory.
+    if (lane == 0) bulk_wait_done0();
     if (!ok) *abort_flag = 1;
   }
   tc_fence_before();
@@ -653,8 +690,9 @@ void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int
     return;
   }
   // weight streaming: the widest tile (most W bytes in flight per stage).  Splitting K pays only when
-  // a handful of tiles would each stream a very long K: measured on B200, the fixed cost of a split
-  // item (partials, counter, reduction) exceeds the gain for K < 4096.
+  // a handful of tiles would each stream a very long K: measured on B200 (whole decode steps of the 1B
+  // decoder at batch 32 and 128), splitting from K = 1024 or 2048 on, into 4 to 8 ranges, changed the
+  // step time by -2 % to +9 %: the fixed cost of a split item (partials, counter, reduction) eats the gain.
   // One CTA streams only about 80 GB/s through its 4-stage ring, so when 256-wide tiles would leave
   // SMs without work, 128-wide tiles (twice as many CTAs) stream faster.
   const int tiles_m = (int)((rows_cap + TC_BM - 1) / TC_BM);
@@ -669,14 +707,16 @@ void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int
   *ksplit = ks;
 }
 
-cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
+cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int max_bn, int* status, int sm_count,
                            cudaStream_t st) {
   if (n_groups == 0 || total_items == 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int grid = total_items < sm_count ? total_items : sm_count;
-  gemm_tc_kernel<<<grid, N_THREADS, SMEM_BYTES, st>>>(groups, n_groups, total_items, status);
-  return cudaGetLastError();
+  const int stages = max_bn <= 128 ? 6 : 4;
+  const int stage_bytes = RING_BYTES / stages;
+  return launch_pdl(gemm_tc_kernel, dim3(grid), dim3(N_THREADS), SMEM_BYTES, st, groups, n_groups, total_items, status,
+                    stages, stage_bytes);
 }
 
 }  // namespace epara

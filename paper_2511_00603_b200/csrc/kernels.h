@@ -23,15 +23,23 @@ constexpr int TC_BM = 128;
 constexpr int TC_BN_MAX = 256;
 constexpr int TC_BK = 64;
 void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int* bn, int* ksplit);
-cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
-                           cudaStream_t st);
+cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int max_bn, int* status,
+                           int sm_count, cudaStream_t st);   // max_bn: widest tile among the groups
 
-// Decode attention (split-KV over 256-token chunks) and the combine of the chunk partials.
+// Weight-streaming GEMM for groups that never exceed 16 rows (GemmGroup::stream): one block per 16
+// rows of W over the whole K, mma.sync, no tensor maps.  total_items = sum of gemm_stream_tiles(N).
+constexpr int GEMM_STREAM_MAX_ROWS = 16;
+int gemm_stream_tiles(int N);
+cudaError_t launch_gemm_stream(const GemmGroup* groups, int n_groups, int total_items, int max_rows, cudaStream_t st);
+
+// Decode attention, split-KV over 256-token chunks.  fused = 1: the block of a (request, kv head) that
+// finishes last merges the chunk partials (AttnDecGroup::counters must be zero at launch and is left
+// zero); fused = 0: a second kernel merges them.  attn_decode_fused() is the rule that picks the mode
+// from the launch's block count; both modes give the same bits.
 constexpr int ATTN_CHUNK = 256;
-cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_chunks,
-                               int hd, int gqa, cudaStream_t st);
-cudaError_t launch_attn_combine(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hq, int hd,
-                                cudaStream_t st);
+bool attn_decode_fused(int total_B, int max_Hkv, int max_chunks, int sm_count);
+cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_Hq,
+                               int max_chunks, int hd, int gqa, int fused, cudaStream_t st);
 // Fills AttnReq[b] = {tables + b*stride, kv_lens[b]} on the device.
 void launch_attn_fill_reqs(AttnReq* reqs, const int32_t* kv_lens, const int32_t* tables, int stride, int B,
                            cudaStream_t st);

@@ -10,7 +10,9 @@ namespace epara {
 // ------------------------------------------------------------------ gather
 __global__ void __launch_bounds__(128) gather_kernel(const GatherGroup* __restrict__ groups) {
   const GatherGroup g = groups[blockIdx.y];
-  if ((int)blockIdx.x >= g.blocks) return;
+  if ((int)blockIdx.x >= g.blocks) return;      // (descriptors are not written by kernels: no wait needed to leave)
+  pdl_launch_dependents();
+  pdl_wait();
   if (g.kind == GATHER_ROWS) {
     const int b = blockIdx.x;
     const uint4* src = reinterpret_cast<const uint4*>(g.reqs[b].input);
@@ -45,7 +47,7 @@ __global__ void __launch_bounds__(128) gather_kernel(const GatherGroup* __restri
 
 void launch_gather(const GatherGroup* groups, int n_groups, int max_blocks, cudaStream_t st) {
   if (n_groups == 0 || max_blocks == 0) return;
-  gather_kernel<<<dim3(max_blocks, n_groups), 128, 0, st>>>(groups);
+  launch_pdl(gather_kernel, dim3(max_blocks, n_groups), dim3(128), 0, st, groups);
 }
 
 // ------------------------------------------------------------------ norms
@@ -181,9 +183,19 @@ __device__ __forceinline__ void norm_rows_narrow(const NormGroup& g, int row0) {
   }
 }
 
+// Blocks a group of M rows of width d needs (device copy of norm_blocks).
+__device__ __forceinline__ int norm_blocks_dev(int M, int d) {
+  constexpr int wpb = NORM_THREADS / 32;
+  if (d <= NORM_NARROW_D) return (M + wpb * NORM_NARROW_ROWS - 1) / (wpb * NORM_NARROW_ROWS);
+  return d <= NORM_WARP_D ? (M + wpb - 1) / wpb : M;
+}
+
 __global__ void __launch_bounds__(NORM_THREADS) norm_kernel(const NormGroup* __restrict__ groups) {
   __shared__ float red[32];
   const NormGroup g = groups[blockIdx.y];
+  if ((int)blockIdx.x >= norm_blocks_dev(g.M, g.d)) return;   // beyond this group's rows: nothing to wait for
+  pdl_launch_dependents();
+  pdl_wait();
   if (g.d <= NORM_NARROW_D) {
     const int row0 = (blockIdx.x * (NORM_THREADS / 32) + (threadIdx.x >> 5)) * NORM_NARROW_ROWS;
     if (row0 < g.M) norm_rows_narrow(g, row0);
@@ -191,7 +203,7 @@ __global__ void __launch_bounds__(NORM_THREADS) norm_kernel(const NormGroup* __r
     const int row = blockIdx.x * (NORM_THREADS / 32) + (threadIdx.x >> 5);
     if (row < g.M) norm_row<true>(g, row, red);
   } else {
-    if ((int)blockIdx.x < g.M) norm_row<false>(g, blockIdx.x, red);
+    norm_row<false>(g, blockIdx.x, red);
   }
 }
 
@@ -204,35 +216,31 @@ int norm_blocks(int M, int d) {
 
 void launch_norm(const NormGroup* groups, int n_groups, int max_blocks, cudaStream_t st) {
   if (n_groups == 0 || max_blocks == 0) return;
-  norm_kernel<<<dim3(max_blocks, n_groups), NORM_THREADS, 0, st>>>(groups);
+  launch_pdl(norm_kernel, dim3(max_blocks, n_groups), dim3(NORM_THREADS), 0, st, groups);
 }
 
 // ------------------------------------------------------------------ RoPE + KV append
 // One block per request.  The new token sits at position kv_len: q and k are rotated there
-// (interleaved pairs, angle pos * inv_freq[j], fp64 angle), q in place, k and v written to the
-// cache page table[pos/16], slot pos%16.
-__global__ void __launch_bounds__(128) rope_append_kernel(const RopeGroup* __restrict__ groups) {
-  __shared__ float cs[128], sn[128];
+// (interleaved pairs; cos and sin come from the model's table, computed from fp64 angles when the
+// model was placed), q in place, k and v written to the cache page table[pos/16], slot pos%16.
+__global__ void __launch_bounds__(256) rope_append_kernel(const RopeGroup* __restrict__ groups) {
   const RopeGroup g = groups[blockIdx.y];
   const int b = blockIdx.x;
   if (b >= g.B) return;
+  pdl_launch_dependents();
+  pdl_wait();
   const ReqDesc r = g.reqs[b];
   const int pos = r.kv_len, hd = g.hd, half = hd >> 1;
-  for (int j = threadIdx.x; j < half; j += blockDim.x) {
-    double s, c;
-    sincos((double)pos * g.inv_freq[j], &s, &c);
-    cs[j] = (float)c;
-    sn[j] = (float)s;
-  }
-  __syncthreads();
+  const float2* cs = g.cs + (size_t)pos * half;
   const int page = r.table[pos / 16], slot = pos % 16;
   bf16* row = g.qkv + (size_t)b * (g.Hq + 2 * g.Hkv) * hd;
   const int n_rot = (g.Hq + g.Hkv) * half;
   for (int e = threadIdx.x; e < n_rot; e += blockDim.x) {
     const int h = e / half, j = e % half;
+    const float2 t = __ldg(cs + j);
     __nv_bfloat162* p2 = reinterpret_cast<__nv_bfloat162*>(row + (size_t)h * hd) + j;
     const float2 v = __bfloat1622float2(*p2);
-    const float x0 = v.x * cs[j] - v.y * sn[j], x1 = v.x * sn[j] + v.y * cs[j];
+    const float x0 = v.x * t.x - v.y * t.y, x1 = v.x * t.y + v.y * t.x;
     const __nv_bfloat162 o = __floats2bfloat162_rn(x0, x1);
     if (h < g.Hq) {
       *p2 = o;
@@ -252,7 +260,7 @@ __global__ void __launch_bounds__(128) rope_append_kernel(const RopeGroup* __res
 
 void launch_rope_append(const RopeGroup* groups, int n_groups, int max_B, cudaStream_t st) {
   if (n_groups == 0 || max_B == 0) return;
-  rope_append_kernel<<<dim3(max_B, n_groups), 128, 0, st>>>(groups);
+  launch_pdl(rope_append_kernel, dim3(max_B, n_groups), dim3(256), 0, st, groups);
 }
 
 // ------------------------------------------------------------------ ViT token assembly
@@ -260,6 +268,8 @@ __global__ void __launch_bounds__(128) assemble_kernel(const AssembleGroup* __re
   const AssembleGroup g = groups[blockIdx.y];
   const int row = blockIdx.x;
   if (row >= g.B * g.T) return;
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = row / g.T, t = row % g.T;
   const bf16* src = (t == 0) ? g.cls : g.E + ((size_t)b * (g.T - 1) + (t - 1)) * g.d;
   const bf16* pos = g.pos + (size_t)t * g.d;
@@ -275,24 +285,44 @@ __global__ void __launch_bounds__(128) assemble_kernel(const AssembleGroup* __re
 
 void launch_assemble(const AssembleGroup* groups, int n_groups, int max_rows, cudaStream_t st) {
   if (n_groups == 0 || max_rows == 0) return;
-  assemble_kernel<<<dim3(max_rows, n_groups), 128, 0, st>>>(groups);
+  launch_pdl(assemble_kernel, dim3(max_rows, n_groups), dim3(128), 0, st, groups);
 }
 
 // ------------------------------------------------------------------ output scatter + argmax
 // One block per request: copies its logits row to the request's buffer and writes the index of
-// the maximum (lowest index on ties; NaNs never win).
-__global__ void __launch_bounds__(256) output_kernel(const OutputGroup* __restrict__ groups) {
-  __shared__ float sv[8];
-  __shared__ int si[8];
+// the maximum (lowest index on ties; NaNs never win).  Rows are read 8 values (16 bytes) at a time.
+constexpr int OUT_THREADS = 512;
+__global__ void __launch_bounds__(OUT_THREADS) output_kernel(const OutputGroup* __restrict__ groups) {
+  __shared__ float sv[OUT_THREADS / 32];
+  __shared__ int si[OUT_THREADS / 32];
   const OutputGroup g = groups[blockIdx.y];
   const int b = blockIdx.x;
   if (b >= g.B) return;
+  pdl_launch_dependents();
+  pdl_wait();
   const ReqDesc r = g.reqs[b];
-  const bf16* src = g.logits + (size_t)b * g.ld;
+  const bf16* src = g.logits + (size_t)b * g.ld;          // 16-byte aligned: ld is a multiple of 8
   bf16* dst = reinterpret_cast<bf16*>(r.out_logits);
+  const bool dst_vec = dst && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
   float best = -INFINITY;
   int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < g.N; i += blockDim.x) {
+  const int nvec = g.N >> 3;
+  for (int i = threadIdx.x; i < nvec; i += OUT_THREADS) {
+    const uint4 u = reinterpret_cast<const uint4*>(src)[i];
+    if (dst_vec) {
+      reinterpret_cast<uint4*>(dst)[i] = u;
+    } else if (dst) {
+      const bf16* e = reinterpret_cast<const bf16*>(&u);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) dst[i * 8 + k] = e[k];
+    }
+    float f[8];
+    unpack8(u, f);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (f[k] > best || (f[k] == best && bi == 0x7fffffff)) { best = f[k]; bi = i * 8 + k; }   // ascending index: the first maximum stays
+  }
+  for (int i = (nvec << 3) + threadIdx.x; i < g.N; i += OUT_THREADS) {   // ragged end
     const bf16 v = src[i];
     if (dst) dst[i] = v;
     const float f = bf2f(v);
@@ -308,7 +338,7 @@ __global__ void __launch_bounds__(256) output_kernel(const OutputGroup* __restri
   if (l == 0) { sv[w] = best; si[w] = bi; }
   __syncthreads();
   if (threadIdx.x == 0) {
-    for (int k = 1; k < 8; ++k)
+    for (int k = 1; k < OUT_THREADS / 32; ++k)
       if (sv[k] > best || (sv[k] == best && si[k] < bi)) { best = sv[k]; bi = si[k]; }
     if (bi == 0x7fffffff) bi = 0;
     if (r.out_argmax) *r.out_argmax = bi;
@@ -317,7 +347,7 @@ __global__ void __launch_bounds__(256) output_kernel(const OutputGroup* __restri
 
 void launch_output(const OutputGroup* groups, int n_groups, int max_B, cudaStream_t st) {
   if (n_groups == 0 || max_B == 0) return;
-  output_kernel<<<dim3(max_B, n_groups), 256, 0, st>>>(groups);
+  launch_pdl(output_kernel, dim3(max_B, n_groups), dim3(OUT_THREADS), 0, st, groups);
 }
 
 }  // namespace epara

@@ -39,6 +39,13 @@ GEMM_CASES = [
     (64, 512, 8192, ("bias", "resid")), # few tiles, very long K: split along K with the last-arriver reduction
     (20, 768, 4096, ("gelu", "bias")),  # split along K, bf16 output
     (9, 256, 5120, ("swiglu",)),        # split along K, SwiGLU, uneven ranges
+    # at most 16 rows: the weight-streaming kernel (16 W rows per block, k-blocks of 32 dealt to 8 warps)
+    (16, 1000, 776, ("bias",)),         # ragged N, K not a multiple of 32
+    (3, 10, 512, ("bias",)),            # N below one block
+    (5, 64, 8, ()),                     # a single 16-byte piece of K
+    (12, 2048, 8192, ("resid",)),       # long K, fp32 residual
+    (2, 512, 2048, ("swiglu",)),
+    (1, 32000, 2048, ()),               # LM head of one request
 ]
 
 

@@ -3,7 +3,8 @@
 epara_decode_attention_static is for embedders that cannot hand the library a scratch buffer
 because they cannot allocate one (the device belongs to a framework's memory pool, or a
 cudaMalloc would stall a latency-critical loop).  It must give what epara_decode_attention gives,
-call after call, although all its calls share one built-in scratch array that is never cleared.
+call after call, although all its calls share one built-in scratch array that keeps the previous
+call's contents (only its chunk counters are cleared per call).
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test.
 """
