@@ -27,6 +27,8 @@ METRIC = "mixed-category requests/s"
 UNIT = "requests/s"
 WORKLOAD = ("mixed co-resident step (configs[3], saturated): 3x MLP-A, 3x ViT-S/16, 2x 1B decoder; per family "
             "instance 0 latency-sensitive batch 4, others frequency-sensitive batch 256; decoder KV ~U[128,4096]")
+WORKLOAD_STRESS = ("stress step (configs[4]): 8B-shaped decoder (d 4096, 32 layers, 32/8 heads, FFN 14336) decoding batch "
+                   "256 with KV ~U[512,{kv_hi}], co-resident with 16x ViT-B/16 at batch 32, all frequency-sensitive")
 
 
 def read_peaks():
@@ -255,8 +257,24 @@ def run_gpu(args):
     from paper_2511_00603_b200 import epara as E, server, workloads as W
     peaks = read_peaks()
     dev = torch.device("cuda", local)
-    srv = server.Server(device=local, workspace_bytes=3 << 30)
-    insts = W.build_mixed(srv, seed=3)
+    stress = args.workload == "stress"
+    workload, clamp = WORKLOAD, None
+    if stress:
+        # size the KV cache to what the device has: lower the upper length bound in steps of 512 until the
+        # whole configuration (plus 6 GB of slack for the framework's context and temporaries) fits
+        free, total = torch.cuda.mem_get_info(dev)
+        kv_hi = W.STRESS_KV_HI
+        while kv_hi > 1024 and W.stress_bytes(kv_hi)["total"] + (6 << 30) > free:
+            kv_hi -= 512
+        need = W.stress_bytes(kv_hi)
+        if kv_hi != W.STRESS_KV_HI:
+            clamp = {"kv_hi": kv_hi, "free_bytes": free, "needed_bytes_at_8192": W.stress_bytes(W.STRESS_KV_HI)["total"]}
+        srv = server.Server(device=local, workspace_bytes=int(need["workspace"]))
+        insts = W.build_stress(srv, seed=4, kv_hi=kv_hi)
+        workload = WORKLOAD_STRESS.format(kv_hi=kv_hi)
+    else:
+        srv = server.Server(device=local, workspace_bytes=3 << 30)
+        insts = W.build_mixed(srv, seed=3)
     n_req = sum(i.n_req for i in insts)
     stream = torch.cuda.current_stream(dev)
 
@@ -382,11 +400,11 @@ def run_gpu(args):
         kernels["attn_dec"]["kv_gbs"] = per_step(kvbytes) / (prof["attn_dec"][0] / 1e3) / 1e9
 
     poisson = None
-    if not args.no_poisson:
+    if not args.no_poisson and not stress:
         poisson = poisson_phase(srv, insts, E, W, torch)
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and not stress:
         smp = OracleSampler()
         t, cores = smp.sample(), smp.cores
         rps, step_s = oracle_rps(t, mixed_counts())
@@ -398,8 +416,9 @@ def run_gpu(args):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "requests_per_step": n_req, "l2": "inputs larger than L2 (17 GB of KV and 4.6 GB of weights per step)",
-                       "parallelism": f"replicas x{world}, no collective"},
+            "config": {"workload": workload, "requests_per_step": n_req,
+                       "l2": f"inputs larger than L2 ({kvbytes / args.steps / 1e9:.0f} GB of KV and {wbytes / args.steps / 1e9:.1f} GB of weights per step)",
+                       "parallelism": f"replicas x{world}, no collective", "kv_clamp": clamp},
             "clocks": clocks, "gpu_launches": launches,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "ms_per_step_unprofiled": ms_plain,
@@ -492,6 +511,38 @@ def run_micro(args):
         kvb = float(lens.sum()) * 2 * Hkv * hd * 2
         print(json.dumps({"kernel": "attn_decode+combine", "B": B, "Hq": Hq, "Hkv": Hkv, "hd": hd, "tokens": int(lens.sum()),
                           "ms": ms, "kv_gbs": kvb / (ms / 1e3) / 1e9, "frac_hbm": kvb / (ms / 1e3) / 1e9 / peaks["hbm_gbs"]}))
+    elif args.micro == "vit_step":
+        # whole steps of one ViT (configs[1]: ViT-B/16 at batch 1 / 8 / 64, each its own frequency-sensitive step)
+        from paper_2511_00603_b200 import server, workloads as W
+        cfgm = W.VIT_S if args.case == "vit_s" else W.VIT_B
+        B = args.m or 64
+        srv = server.Server(device=0, workspace_bytes=2 << 30)
+        inst = W.Instance(srv, synth.make_vit(seed=1, device=dev, **cfgm), E.CAT_FS, B, seed=11)
+        times = []
+        for i in range(args.steps + 4):
+            if i == args.steps + 3:
+                srv.ctx.epara_set_profile(True)
+            flush.zero_()
+            inst.submit_all(srv.ctx)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            info = srv.ctx.epara_step(stream.cuda_stream, 0)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            for t in inst.tickets:
+                srv.ctx.epara_collect(t)
+            if 3 <= i < args.steps + 3:
+                times.append(e0.elapsed_time(e1))
+        prof = srv.ctx.epara_step_profile()
+        ms = sorted(times)[len(times) // 2]
+        d, L, T, F = cfgm["d"], cfgm["n_layers"], 197, cfgm["mlp"]
+        attn_flops = 4.0 * T * T * d * L * B
+        print(json.dumps({"kernel": "vit step", "case": args.case or "vit_b", "B": B, "ms": ms, "launches": info.launches,
+                          "images_per_s": B / (ms / 1e3), "gemm_tflop": info.gemm_flops / 1e12,
+                          "tflops_step": (info.gemm_flops + attn_flops) / (ms / 1e3) / 1e12,
+                          "frac_tensor_sustained": (info.gemm_flops + attn_flops) / (ms / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
+                          "per_kind_ms": {k: round(v[0], 4) for k, v in prof.items() if v[1]}}))
+        srv.close()
     elif args.micro == "decode_step":
         # whole decode steps of one decoder (configs[2] / the decoder of configs[4]) through the step API
         from paper_2511_00603_b200 import server, workloads as W
@@ -530,13 +581,15 @@ def run_micro(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["gemm", "attn_dec", "decode_step"], help="time one kernel instead of the step")
+    ap.add_argument("--micro", default=None, choices=["gemm", "attn_dec", "decode_step", "vit_step"], help="time one kernel instead of the step")
     ap.add_argument("--case", default="vit_s")
     ap.add_argument("--m", type=int, default=0, help="override M (gemm) or B (attn_dec) of the micro case")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="epara", choices=["epara", "reference"])
+    ap.add_argument("--workload", default="mixed", choices=["mixed", "stress"],
+                    help="mixed: the co-resident step the metric is quoted on; stress: 8B decoder batch 256 + 16 ViT-B")
     ap.add_argument("--no-poisson", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

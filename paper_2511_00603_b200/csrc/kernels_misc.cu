@@ -116,9 +116,11 @@ __device__ __forceinline__ void norm_row(const NormGroup& g, int row, float* red
   }
 }
 
-// Narrow rows (d <= 512): one warp takes ROWS rows at once, all their loads in flight together.
+// Narrow rows (d <= 512): one warp takes ROWS rows at once, all their loads in flight together.  Two rows
+// keep the kernel at 64 registers, so four blocks (32 warps) share an SM: with more registers per
+// thread the occupancy, not the loads per warp, limited the bandwidth.
 constexpr int NORM_NARROW_D = 512;
-constexpr int NORM_NARROW_ROWS = 4;
+constexpr int NORM_NARROW_ROWS = 2;
 __device__ __forceinline__ void norm_rows_narrow(const NormGroup& g, int row0) {
   const int lane = threadIdx.x & 31;
   const int nvec = g.d >> 2;
@@ -190,7 +192,7 @@ __device__ __forceinline__ int norm_blocks_dev(int M, int d) {
   return d <= NORM_WARP_D ? (M + wpb - 1) / wpb : M;
 }
 
-__global__ void __launch_bounds__(NORM_THREADS) norm_kernel(const NormGroup* __restrict__ groups) {
+__global__ void __launch_bounds__(NORM_THREADS, 4) norm_kernel(const NormGroup* __restrict__ groups) {
   __shared__ float red[32];
   const NormGroup g = groups[blockIdx.y];
   if ((int)blockIdx.x >= norm_blocks_dev(g.M, g.d)) return;   // beyond this group's rows: nothing to wait for

@@ -128,6 +128,20 @@ def make_kv_pool(n_layers: int, num_pages: int, n_kv_heads: int, head_dim: int, 
     return pool
 
 
+def make_kv_pool_replicated(n_layers: int, num_pages: int, n_kv_heads: int, head_dim: int, seed: int,
+                            device="cpu") -> torch.Tensor:
+    """Pool of the same shape and distribution for very large caches: layer 0 is drawn N(0,1) as in
+    make_kv_pool; layer l holds layer 0's pages rotated by 7919 * l positions (a copy, not a new draw),
+    so filling 100+ GB takes seconds and any page of any layer can be recomputed from layer 0."""
+    pool = torch.empty((n_layers, num_pages, 2, n_kv_heads, PAGE, head_dim), device=device, dtype=torch.bfloat16)
+    pool[0] = make_kv_pool(1, num_pages, n_kv_heads, head_dim, seed, device=device)[0]
+    for l in range(1, n_layers):
+        sh = (7919 * l) % num_pages
+        pool[l, sh:] = pool[0, :num_pages - sh]
+        pool[l, :sh] = pool[0, num_pages - sh:]
+    return pool
+
+
 def make_decode_batch(batch: int, len_lo: int, len_hi: int, vocab: int, seed: int
                       ) -> Tuple[np.ndarray, np.ndarray, List[np.ndarray], int]:
     """Tokens ~U[0,vocab), KV lengths ~U[len_lo,len_hi] (inclusive), and per-request block

@@ -35,7 +35,7 @@ class Instance:
     """One placed model with a pool of ready-made requests (inputs, outputs, ctypes descriptors)."""
 
     def __init__(self, srv, p: Dict, category: int, n_req: int, seed: int, kv_lo: int = 128, kv_hi: int = 4096,
-                 max_batch: int = 0):
+                 max_batch: int = 0, kv_replicate_layers: bool = False):
         dev = srv.device
         self.p, self.category, self.n_req, self.kind = p, category, n_req, p["kind"]
         self.kv_pool = None
@@ -50,7 +50,12 @@ class Instance:
             self.x = None
             self.n_out = p["vocab"]
             self.tokens, self.lens, self.tables, npages = synth.make_decode_batch(n_req, kv_lo, kv_hi, p["vocab"], seed)
-            self.kv_pool = synth.make_kv_pool(p["n_layers"], npages, p["n_kv_heads"], p["head_dim"], seed + 1, device=dev)
+            if kv_replicate_layers:
+                self.kv_pool = synth.make_kv_pool_replicated(p["n_layers"], npages, p["n_kv_heads"], p["head_dim"],
+                                                             seed + 1, device=dev)
+            else:
+                self.kv_pool = synth.make_kv_pool(p["n_layers"], npages, p["n_kv_heads"], p["head_dim"], seed + 1,
+                                                  device=dev)
             flat = np.concatenate(self.tables)
             self.tables_dev = torch.as_tensor(flat, device=dev)
             self.table_off = np.concatenate([[0], np.cumsum([len(t) for t in self.tables])])
@@ -111,4 +116,47 @@ def build_mixed(srv, seed: int = 3, ls_batch: int = 4, fs_batch: int = 256, kv_l
         out.append(Instance(srv, synth.make_decoder(seed=seed * 100 + k, device=dev, **DEC_1B), cat, n,
                             seed * 1000 + k, kv_lo=kv_lo, kv_hi=kv_hi))
         k += 1
+    return out
+
+
+# ------------------------------------------------------------------ stress step
+STRESS_VITS, STRESS_VIT_BATCH, STRESS_DEC_BATCH = 16, 32, 256
+STRESS_KV_LO, STRESS_KV_HI = 512, 8192
+
+
+def stress_bytes(kv_hi: int, n_vits: int = STRESS_VITS, vit_batch: int = STRESS_VIT_BATCH,
+                 dec_batch: int = STRESS_DEC_BATCH, kv_lo: int = STRESS_KV_LO) -> Dict[str, float]:
+    """Device bytes the stress step needs for a KV upper bound (expected value of the seeded lengths)."""
+    d = DEC_8B
+    per_tok = 2 * d["n_kv_heads"] * d["head_dim"] * 2 * d["n_layers"]
+    mean_pages = ((kv_lo + kv_hi) / 2 + 1 + synth.PAGE) / synth.PAGE
+    kv = dec_batch * mean_pages * synth.PAGE * per_tok
+    dec_w = 2.0 * (2 * d["vocab"] * d["d"] + d["n_layers"] * (
+        (d["n_q_heads"] + 2 * d["n_kv_heads"]) * d["head_dim"] * d["d"] + d["d"] * d["n_q_heads"] * d["head_dim"] +
+        3 * d["ffn"] * d["d"]))
+    vit_w = n_vits * 2.0 * 86.6e6
+    rows = vit_batch * 197 + 128
+    ws = n_vits * rows * (768 * 4 + 768 * 2 * 2 + 2304 * 2 + 3072 * 2) + (dec_batch + 128) * (
+        4096 * 6 + 6144 * 2 + 14336 * 2 + 32000 * 2) + dec_batch * 32 * (kv_hi // 256 + 2) * 130 * 4 + (256 << 20)
+    imgs = n_vits * vit_batch * 3 * 224 * 224 * 2
+    return {"kv": kv, "decoder_weights": dec_w, "vit_weights": vit_w, "workspace": float(ws), "images": float(imgs),
+            "total": kv + dec_w + vit_w + ws + imgs}
+
+
+def build_stress(srv, seed: int = 4, kv_hi: int = STRESS_KV_HI, n_vits: int = STRESS_VITS,
+                 vit_batch: int = STRESS_VIT_BATCH, dec_batch: int = STRESS_DEC_BATCH, kv_lo: int = STRESS_KV_LO
+                 ) -> List[Instance]:
+    """The stress configuration: one 8B-shaped decoder decoding `dec_batch` sequences with KV lengths
+    ~U[kv_lo, kv_hi], co-resident with `n_vits` ViT-B/16 instances at batch `vit_batch`, all
+    frequency-sensitive.  The decoder's unpacked weight copies are dropped once the packed layout exists;
+    the KV pool is drawn for layer 0 and rotated for the other layers (see make_kv_pool_replicated)."""
+    dev = srv.device
+    out: List[Instance] = []
+    p = synth.make_decoder(seed=seed * 100, device=dev, **DEC_8B)
+    p["packed_layers"] = [synth.pack_decoder_layer(L) for L in p["layers"]]
+    p["layers"] = None                      # the packed layout is all the library reads
+    out.append(Instance(srv, p, E.CAT_FS, dec_batch, seed * 1000, kv_lo=kv_lo, kv_hi=kv_hi, kv_replicate_layers=True))
+    for i in range(n_vits):
+        out.append(Instance(srv, synth.make_vit(seed=seed * 100 + 1 + i, device=dev, **VIT_B), E.CAT_FS, vit_batch,
+                            seed * 1000 + 1 + i))
     return out
