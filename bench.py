@@ -23,6 +23,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) per GEMM launch of the mixed step, from one ncu pass over the 130 GEMM launches
+# of a step (65 tensor-core + 65 weight-streaming: 16.10 + 8.77 GB and 2.08 + 0.0005 GB; see
+# profiles/gemm_kernels_mixed_step_dram_traffic.md).  Set to None when the GEMM kernels change.
+GEMM_TRAFFIC_PER_LAUNCH_MIXED = (16104832768 + 8773382144 + 2083244288 + 522240) / 130
+
 METRIC = "mixed-category requests/s"
 UNIT = "requests/s"
 WORKLOAD = ("mixed co-resident step (configs[3], saturated): 3x MLP-A, 3x ViT-S/16, 2x 1B decoder; per family "
@@ -274,7 +279,7 @@ def run_gpu(args):
         workload = WORKLOAD_STRESS.format(kv_hi=kv_hi)
     else:
         srv = server.Server(device=local, workspace_bytes=3 << 30)
-        insts = W.build_mixed(srv, seed=3)
+        insts = W.build_mixed(srv, seed=3, kv_hi=args.kv_hi)
     n_req = sum(i.n_req for i in insts)
     stream = torch.cuda.current_stream(dev)
 
@@ -352,16 +357,49 @@ def run_gpu(args):
              for i in insts]
     h2d = sum(x.numel() * x.element_size() for _, x in h_in)
     d2h = sum(l.numel() * 2 + a.numel() * 4 for _, l, a in h_out)
+    # Two device input buffers per instance: while step s computes, the inputs of step s + 1 travel on a
+    # copy stream.  Every step still uploads all of its inputs and reads all of its results back into
+    # pinned host memory; the host does not wait for a step before it submits the next one (the library
+    # rotates its descriptor slots), so planning and launching overlap the previous step's kernels.
+    for i in insts:
+        i.make_alt()
+    copy_stream = torch.cuda.Stream(dev)
+    ev_in = [torch.cuda.Event(), torch.cuda.Event()]
+    ev_free = [None, None]
+
+    def upload(buf):
+        with torch.cuda.stream(copy_stream):
+            if ev_free[buf] is not None:
+                copy_stream.wait_event(ev_free[buf])      # the step that read this buffer has finished
+            # in pieces of about 4 MB: a copy engine serves its queue in order, and the small descriptor
+            # upload of the step that starts meanwhile must not wait behind 150 MB of images
+            for i, hx in h_in:
+                dst = i.x_alt if buf else i.x
+                rows = max(1, (4 << 20) // max(1, hx[0].numel() * hx.element_size()))
+                for r0 in range(0, hx.shape[0], rows):
+                    dst[r0:r0 + rows].copy_(hx[r0:r0 + rows], non_blocking=True)
+            ev_in[buf].record(copy_stream)
+
     barrier()
     t0 = time.perf_counter()
-    for _ in range(args.steps):
-        for i, hx in h_in:
-            i.x.copy_(hx, non_blocking=True)
-        one_step()
+    upload(0)
+    for s_i in range(args.steps):
+        buf = s_i & 1
+        stream.wait_event(ev_in[buf])
+        for i in insts:
+            i.submit_all(srv.ctx, alt=bool(buf))
+            outstanding.append(list(i.tickets))
+        srv.ctx.epara_step(stream.cuda_stream, 0)
+        ev_free[buf] = torch.cuda.Event()
+        ev_free[buf].record(stream)
+        # (after the step is enqueued: its small descriptor upload must not queue behind the next step's
+        # 150 MB of images in the host-to-device copy engine)
+        if s_i + 1 < args.steps:
+            upload(buf ^ 1)
         for i, hl, ha in h_out:
             hl.copy_(i.logits, non_blocking=True)
             ha.copy_(i.argmax, non_blocking=True)
-        stream.synchronize()
+    stream.synchronize()                    # every step's results are on the host when the clock stops
     e2e_s = time.perf_counter() - t0
     drain()
     if world > 1:
@@ -381,9 +419,11 @@ def run_gpu(args):
     per_step = lambda v: v / args.steps
     if dom == "gemm":
         ach = per_step(flops) / (prof["gemm"][0] / 1e3) / 1e12
-        roof = {"kernel": "gemm_tc_kernel (all GEMM launches of a step)", "bound": "tensor", "achieved": ach,
-                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
-                "traffic": None, "peak_source": peaks["source"] + " (sustained)"}
+        roof = {"kernel": "gemm_tc_kernel + gemm_stream_kernel (all GEMM launches of a step)", "bound": "tensor",
+                "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops_sustained"],
+                "traffic": None if stress else GEMM_TRAFFIC_PER_LAUNCH_MIXED,
+                "peak_source": peaks["source"] + " (sustained)"}
     elif dom == "attn_dec":
         ach = per_step(kvbytes) / (prof["attn_dec"][0] / 1e3) / 1e9
         roof = {"kernel": "attn_decode_kernel (all launches of a step)", "bound": "hbm", "achieved": ach,
@@ -590,6 +630,9 @@ def main():
     ap.add_argument("--impl", default="epara", choices=["epara", "reference"])
     ap.add_argument("--workload", default="mixed", choices=["mixed", "stress"],
                     help="mixed: the co-resident step the metric is quoted on; stress: 8B decoder batch 256 + 16 ViT-B")
+    ap.add_argument("--kv-hi", type=int, default=4096,
+                    help="mixed workload: upper bound of the decoders' KV lengths (a short cache keeps a profiler capture small; "
+                         "the GEMM launches do not depend on it)")
     ap.add_argument("--no-poisson", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -80,8 +80,21 @@ class Instance:
         inp.out_logits = self.logits[out_slot].data_ptr()
         inp.out_argmax = self.argmax.data_ptr() + 4 * out_slot
 
-    def submit_all(self, ctx: "E.Context"):
-        ctx.epara_submit_many(self.mid, self.category, self.inputs, self.n_req, self.tickets)
+    def submit_all(self, ctx: "E.Context", alt: bool = False):
+        """Submits the whole pool; alt=True takes the inputs from the second input buffer (make_alt)."""
+        ctx.epara_submit_many(self.mid, self.category, self.inputs_alt if alt else self.inputs, self.n_req, self.tickets)
+
+    def make_alt(self):
+        """A second device input buffer with its own request descriptors, so that the inputs of the next
+        step can be uploaded while the current step still reads the first one."""
+        if self.x is None:
+            self.x_alt, self.inputs_alt = None, self.inputs
+            return
+        self.x_alt = torch.empty_like(self.x)
+        self.inputs_alt = (E.Inputs * self.n_req)()
+        for i in range(self.n_req):
+            C.memmove(C.byref(self.inputs_alt[i]), C.byref(self.inputs[i]), C.sizeof(E.Inputs))
+            self.inputs_alt[i].input = self.x_alt[i].data_ptr()
 
     def input_bytes(self) -> int:
         return 0 if self.x is None else self.x.numel() * self.x.element_size()
