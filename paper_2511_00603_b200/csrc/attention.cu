@@ -612,15 +612,20 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
         mma_bf16_16816(sc[2 * np + 1], qa[ks], r[2], r[3]);
       }
     }
-    // scale, mask, online softmax (rows gq and gq+8 of the warp tile)
+    // online softmax (rows gq and gq+8 of the warp tile).  The running maximum is kept in units of the raw
+    // scores (the scale is positive), so that scaling and subtracting the maximum are one FMA per score;
+    // only the ragged last block of keys needs masking.
+    if (kb + 64 > T) {
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+        const int key = kb + n * 8 + 2 * tq;
+        if (key >= T) { sc[n][0] = -INFINITY; sc[n][2] = -INFINITY; }
+        if (key + 1 >= T) { sc[n][1] = -INFINITY; sc[n][3] = -INFINITY; }
+      }
+    }
     float mx_lo = m_lo, mx_hi = m_hi;
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
-      const int key = kb + n * 8 + 2 * tq;
-      sc[n][0] = (key < T) ? sc[n][0] * scale : -INFINITY;
-      sc[n][1] = (key + 1 < T) ? sc[n][1] * scale : -INFINITY;
-      sc[n][2] = (key < T) ? sc[n][2] * scale : -INFINITY;
-      sc[n][3] = (key + 1 < T) ? sc[n][3] * scale : -INFINITY;
       mx_lo = fmaxf(mx_lo, fmaxf(sc[n][0], sc[n][1]));
       mx_hi = fmaxf(mx_hi, fmaxf(sc[n][2], sc[n][3]));
     }
@@ -628,8 +633,9 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
     mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-    const float a_lo = exp2f(m_lo - mx_lo), a_hi = exp2f(m_hi - mx_hi);
+    const float a_lo = exp2f((m_lo - mx_lo) * scale), a_hi = exp2f((m_hi - mx_hi) * scale);
     m_lo = mx_lo; m_hi = mx_hi;
+    const float nm_lo = -m_lo * scale, nm_hi = -m_hi * scale;
     l_lo *= a_lo; l_hi *= a_hi;
 #pragma unroll
     for (int n = 0; n < 8; ++n) { o[n][0] *= a_lo; o[n][1] *= a_lo; o[n][2] *= a_hi; o[n][3] *= a_hi; }
@@ -637,8 +643,8 @@ __global__ void __launch_bounds__(ENC_ROWS * 2, 2) attn_encoder_kernel(const Att
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
       if ((n >> 1) >= np_lim) continue;      // all keys of the group are masked: never read below
-      const float p0 = exp2f(sc[n][0] - m_lo), p1 = exp2f(sc[n][1] - m_lo);
-      const float p2 = exp2f(sc[n][2] - m_hi), p3 = exp2f(sc[n][3] - m_hi);
+      const float p0 = exp2f(fmaf(sc[n][0], scale, nm_lo)), p1 = exp2f(fmaf(sc[n][1], scale, nm_lo));
+      const float p2 = exp2f(fmaf(sc[n][2], scale, nm_hi)), p3 = exp2f(fmaf(sc[n][3], scale, nm_hi));
       l_lo += p0 + p1;
       l_hi += p2 + p3;
       pa[n >> 1][(n & 1) * 2 + 0] = pack2(p0, p1);

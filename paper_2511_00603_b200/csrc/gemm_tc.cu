@@ -686,6 +686,9 @@ void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int
   if (rows_cap <= 0) { *bn = 128; *ksplit = 1; return; }
   if (rows_cap > 256) {                       // dense: tensor-bound; a 128 x 256 MMA runs at about twice the
     *bn = (N > 128) ? 256 : 128;              // efficiency of a 128 x 128 one, which outweighs padded columns
+    // fp32-residual outputs leave in 16-column boxes, so their tiles may be 192 wide (48 columns per
+    // epilogue warp): N = 384 then fills two tiles exactly instead of wasting a quarter of two 256-wide ones
+    if ((epi & EPI_RESID_F32) && N % 192 == 0 && padded(192) < padded(256)) *bn = 192;
     *ksplit = 1;
     return;
   }
