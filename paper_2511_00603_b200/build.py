@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libepara.so")
-SOURCES = ["epara_api.cu", "kernels_misc.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_stream.cu", "attention.cu"]
+SOURCES = ["epara_api.cu", "kernels_misc.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_stream.cu", "attention.cu", "attention_tc.cu"]
 
 
 def _stale() -> bool:

@@ -1,0 +1,392 @@
+// Encoder (bidirectional) attention on the sm_100a tensor cores, head dimension 64, up to 224 tokens.
+//
+// One persistent CTA per SM walks over (image, head) items.  Per item, with T tokens, KP = T rounded
+// up to 16 key columns and one or two tiles of 128 query rows:
+//   warp 0 (one lane)  TMA producer: the Q tiles (128 x 64), the K tile and the V tile (KP x 64) of the
+//                      item straight out of the qkv activation matrix [rows, 3d] (128-byte swizzle);
+//   warp 1 (one lane)  MMA issuer: S_m = Q_m K^T (tcgen05.mma M 128, N KP, K 64) into TMEM for both
+//                      query tiles, later O_m = P_m V (M 128, N 64, K KP) into a third TMEM region;
+//   warps 2..9         256 workers; thread = (query row, half).  First they transpose V (tokens x 64) into
+//                      V^T (64 x tokens, K-major swizzled: the B operand of P V), zeroing tokens >= T.
+//                      Softmax: two passes over the thread's half of the row of S in TMEM (reading TMEM is
+//                      cheap): maximum (the halves meet in shared memory), then p = exp2((s - max) * scale)
+//                      with the row sum in fp32; P goes to shared memory as bf16 in the K-major
+//                      128-byte-swizzled layout the MMA reads as its A operand.  Key columns >= T are masked
+//                      by selection.  Last they read their half of O from TMEM, divide by the row sum and
+//                      store bf16 (rows >= T are not stored).
+// Rows of the Q / K / V tiles past the image's T tokens belong to the next image or lie past the matrix
+// (TMA fills those with zeros); they only ever reach masked columns, zeroed V^T columns or rows that
+// are not stored.  Every mbarrier wait is bounded: when one runs out the kernel records a code in
+// *status, all roles leave their loops, TMEM is freed and the kernel returns.
+#include "common.cuh"
+#include "kernels.h"
+#include "tcgen05.cuh"
+
+namespace epara {
+
+namespace {
+
+using namespace tc;
+
+constexpr int ET_THREADS = 320;                       // 10 warps
+constexpr int ET_Q_BYTES = 128 * 128;                 // one query tile: 128 rows of 128 bytes
+constexpr int ET_KV_BYTES = ENC_TC_MAX_T * 128;       // K or V tile at the largest KP (224 rows)
+constexpr int ET_VT_BLOCK = 64 * 128;                 // V^T: one 64-key block = 64 rows (dims) of 128 bytes
+constexpr int ET_P_BLOCK = 128 * 128;                 // P: one 64-key block = 128 rows of 128 bytes
+constexpr int ET_OFF_Q = 0;
+constexpr int ET_OFF_K = 2 * ET_Q_BYTES;
+constexpr int ET_OFF_V = ET_OFF_K + ET_KV_BYTES;
+constexpr int ET_OFF_VT = ET_OFF_V + ET_KV_BYTES;
+constexpr int ET_OFF_P = ET_OFF_VT + 4 * ET_VT_BLOCK;
+constexpr int ET_OFF_L = ET_OFF_P + 4 * ET_P_BLOCK;   // partial row sums [2 tiles][2 halves][128] fp32, then partial maxima
+constexpr int ET_OFF_BAR = ET_OFF_L + 4096;
+constexpr size_t ET_SMEM = 1024 + ET_OFF_BAR + 256;
+static_assert(ET_OFF_V % 1024 == 0 && ET_OFF_VT % 1024 == 0 && ET_OFF_P % 1024 == 0, "swizzle atoms are 1024 bytes");
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+constexpr int ET_S_COL0 = 0, ET_S_COL1 = 224, ET_O_COL = 448;   // TMEM columns: S_0, S_1, O (64)
+
+enum { B_FULL_QK = 0, B_FULL_V, B_QK_FREE, B_V_FREE, B_VT_READY, B_S_FULL0, B_S_FULL1, B_S_EMPTY0, B_S_EMPTY1,
+       B_P_READY0, B_P_READY1, B_O_FULL0, B_O_FULL1, B_O_EMPTY, B_MX0, B_MX1, B_COUNT };
+
+struct ItemRef {
+  const AttnEncGroup* g;
+  int b, h;
+};
+__device__ __forceinline__ ItemRef find_item(const AttnEncGroup* groups, int n_groups, int item) {
+  int gi = 0;
+  for (int i = 1; i < n_groups; ++i) if (item >= groups[i].blk_start) gi = i;
+  ItemRef r;
+  r.g = groups + gi;
+  const int local = item - r.g->blk_start;
+  r.b = local / r.g->H;
+  r.h = local - r.b * r.g->H;
+  return r;
+}
+
+__global__ void __launch_bounds__(ET_THREADS, 1)
+attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status) {
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t bars = base + ET_OFF_BAR;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + ET_OFF_BAR + 8 * B_COUNT);
+  static_assert(8 * B_COUNT + 16 <= 256, "barrier area");
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* sm_l = reinterpret_cast<float*>(base_ptr + ET_OFF_L);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B_FULL_QK), 1); mbar_init(bar(B_FULL_V), 1); mbar_init(bar(B_QK_FREE), 1);
+    mbar_init(bar(B_V_FREE), 256); mbar_init(bar(B_VT_READY), 256);
+    mbar_init(bar(B_S_FULL0), 1); mbar_init(bar(B_S_FULL1), 1);
+    mbar_init(bar(B_S_EMPTY0), 256); mbar_init(bar(B_S_EMPTY1), 256);
+    mbar_init(bar(B_P_READY0), 256); mbar_init(bar(B_P_READY1), 256);
+    mbar_init(bar(B_O_FULL0), 1); mbar_init(bar(B_O_FULL1), 1); mbar_init(bar(B_O_EMPTY), 256);
+    mbar_init(bar(B_MX0), 256); mbar_init(bar(B_MX1), 256);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                  // the qkv matrix comes from the kernel before this one
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      const AttnEncGroup* g_prev = nullptr;
+      uint32_t it = 0;
+      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++it) {
+        const ItemRef r = find_item(groups, n_groups, item);
+        const AttnEncGroup* g = r.g;
+        if (g != g_prev) { tensormap_acquire(&g->tmQ); tensormap_acquire(&g->tmKV); g_prev = g; }
+        const int T = g->T, KP = g->KP, d = g->H * 64, n_mt = (T + 127) >> 7;
+        const int row0 = r.b * T;
+        // Q and K: free once both S = Q K^T of the previous item are complete
+        if (!mbar_wait<false>(bar(B_QK_FREE), (it & 1u) ^ 1u, abort_flag)) { ok = false; atomicExch(status, 11); break; }
+        mbar_expect_tx(bar(B_FULL_QK), (uint32_t)(n_mt * ET_Q_BYTES + KP * 128));
+        for (int m = 0; m < n_mt; ++m)
+          tma_load_2d(base + ET_OFF_Q + m * ET_Q_BYTES, &g->tmQ, r.h * 64, row0 + m * 128, bar(B_FULL_QK));
+        tma_load_2d(base + ET_OFF_K, &g->tmKV, d + r.h * 64, row0, bar(B_FULL_QK));
+        // V: free once the transposing warps have read the previous one
+        if (!mbar_wait<false>(bar(B_V_FREE), (it & 1u) ^ 1u, abort_flag)) { ok = false; atomicExch(status, 12); break; }
+        mbar_expect_tx(bar(B_FULL_V), (uint32_t)(KP * 128));
+        tma_load_2d(base + ET_OFF_V, &g->tmKV, 2 * d + r.h * 64, row0, bar(B_FULL_V));
+      }
+      if (!ok) *abort_flag = 1;
+      // copies in flight when a wait gave up: the consumers have left, so nothing reads them; let them land
+      if (!ok) {
+        volatile int never = 0;
+        mbar_wait<false>(bar(B_FULL_QK), (it & 1u), &never);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    // Order of issue per item: P_0 V, then Q_0 K^T of the NEXT item, then P_1 V, then Q_1 K^T of the next
+    // item -- so that the scores of the next item are waiting in TMEM when the softmax warps get there.
+    // Barriers of the first query tile complete once per item, those of the second once per item with two
+    // tiles, O_EMPTY once per tile: each has its own use counter (items of different models mix).
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t n_o = 0;
+      uint32_t cnt_s[2] = {0, 0};               // S = Q K^T issued so far, per tile index
+      uint32_t cnt_pv[2] = {0, 0};              // P V issued so far, per tile index
+      uint32_t cnt_qk = 0;                      // items whose Q / K have been consumed
+      // Q_m K^T of an item (its Q and K must have landed: caller waited FULL_QK)
+      auto issue_s = [&](const AttnEncGroup* g, int m) -> bool {
+        if (!mbar_wait<false>(bar(B_S_EMPTY0 + m), (cnt_s[m] & 1u) ^ 1u, abort_flag)) { atomicExch(status, 14); return false; }
+        tc_fence_after();
+        const uint32_t idesc_s = make_idesc(g->KP);
+        const uint64_t dq = make_smem_desc(base + ET_OFF_Q + m * ET_Q_BYTES), dk = make_smem_desc(base + ET_OFF_K);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(m ? ET_S_COL1 : ET_S_COL0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_f16(d_tmem, dq + (uint64_t)(k * 2), dk + (uint64_t)(k * 2), idesc_s, k > 0 ? 1u : 0u);
+        mma_commit(bar(B_S_FULL0 + m));
+        ++cnt_s[m];
+        return true;
+      };
+      auto wait_qk = [&]() -> bool {
+        if (!mbar_wait<false>(bar(B_FULL_QK), cnt_qk & 1u, abort_flag)) { atomicExch(status, 13); return false; }
+        tc_fence_after();
+        ++cnt_qk;
+        return true;
+      };
+      uint32_t it = 0;
+      const AttnEncGroup* g_next = nullptr;
+      if ((int)blockIdx.x < total_items) {
+        g_next = find_item(groups, n_groups, blockIdx.x).g;
+        const int n_mt = (g_next->T + 127) >> 7;
+        ok = wait_qk();
+        for (int m = 0; m < n_mt && ok; ++m) ok = issue_s(g_next, m);
+        if (ok) mma_commit(bar(B_QK_FREE));     // arrives when every MMA issued so far is complete
+      }
+      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++it) {
+        const AttnEncGroup* g = g_next;
+        const int KP = g->KP, n_mt = (g->T + 127) >> 7;
+        const bool has_next = item + (int)gridDim.x < total_items;
+        int n_mt_next = 0;
+        if (has_next) {
+          g_next = find_item(groups, n_groups, item + gridDim.x).g;
+          n_mt_next = (g_next->T + 127) >> 7;
+        }
+        if (!mbar_wait<false>(bar(B_VT_READY), it & 1u, abort_flag)) { ok = false; atomicExch(status, 15); break; }
+        for (int m = 0; m < n_mt && ok; ++m) {
+          if (!mbar_wait<false>(bar(B_P_READY0 + m), cnt_pv[m] & 1u, abort_flag)) { ok = false; atomicExch(status, 16); break; }
+          // O must have been read out by the warps that store the previous tile
+          if (!mbar_wait<false>(bar(B_O_EMPTY), (n_o & 1u) ^ 1u, abort_flag)) { ok = false; atomicExch(status, 17); break; }
+          ++n_o;
+          tc_fence_after();
+          const uint32_t idesc_o = make_idesc(64);
+          const uint32_t d_tmem = tmem_base + (uint32_t)ET_O_COL;
+          const int ksteps = KP >> 4;
+          for (int k = 0; k < ksteps; ++k) {
+            const uint64_t dp = make_smem_desc(base + ET_OFF_P + (k >> 2) * ET_P_BLOCK) + (uint64_t)((k & 3) * 2);
+            const uint64_t dv = make_smem_desc(base + ET_OFF_VT + (k >> 2) * ET_VT_BLOCK) + (uint64_t)((k & 3) * 2);
+            mma_f16(d_tmem, dp, dv, idesc_o, k > 0 ? 1u : 0u);
+          }
+          mma_commit(bar(B_O_FULL0 + m));
+          ++cnt_pv[m];
+          // scores of the next item: tile 0 after this item's first P V, the rest after its last
+          if (has_next) {
+            if (m == 0) {
+              ok = wait_qk() && issue_s(g_next, 0);
+              if (ok && n_mt_next == 1) mma_commit(bar(B_QK_FREE));
+            }
+            if (ok && m == n_mt - 1 && n_mt_next == 2) {
+              ok = issue_s(g_next, 1);
+              if (ok) mma_commit(bar(B_QK_FREE));
+            }
+          }
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else {
+    // ------------------------------------------------------------------ workers (warps 2..9, 256 threads)
+    // Thread (quarter, lane, half): query row quarter*32 + lane of the current tile, and one half of the
+    // key columns for the softmax / one half of the 64 output dims for the store.
+    const int quarter = warp & 3, row = quarter * 32 + lane, half = (warp - 2) >> 2;
+    const int wtid = threadIdx.x - 64;                      // 0..255
+    const float scale = 1.4426950408889634f * 0.125f;       // log2(e) / sqrt(64)
+    float* sm_mx = sm_l + 512;                              // [2 tiles][2 halves][128] partial row maxima
+    bool ok = true;
+    uint32_t it = 0;
+    uint32_t cnt_m[2] = {0, 0};                             // tiles processed so far, per tile index
+    int prev_last = -1;                                     // last tile index of the previous item
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++it) {
+      const ItemRef r = find_item(groups, n_groups, item);
+      const AttnEncGroup* g = r.g;
+      const int T = g->T, KP = g->KP, d = g->H * 64, n_mt = (T + 127) >> 7;
+      // ---- V (tokens x 64, swizzled by the TMA) -> V^T (64 x tokens, K-major swizzled), tokens >= T zeroed.
+      // V tile: token t, 16-byte piece dc (dims 8 dc .. 8 dc + 7) sits at t * 128 + ((dc ^ (t & 7)) << 4).
+      // V^T: dim dd, token t sits in block t / 64 at dd/8 * 1024 + dd%8 * 128 + (((t%64)/8 ^ dd%8) << 4) + t%8 * 2.
+      // (the previous item's last P V, which read V^T, is complete: these threads waited for its O)
+      if (!mbar_wait<false>(bar(B_FULL_V), it & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 20); break; }
+      {
+        const unsigned char* vsm = base_ptr + ET_OFF_V;
+        unsigned char* vt = base_ptr + ET_OFF_VT;
+        const int t = wtid;                                 // one token per thread (KP <= 224 < 256), all 8 dim pieces
+        if (t < KP) {
+          unsigned char* blk0 = vt + (t >> 6) * ET_VT_BLOCK + (t & 7) * 2;
+          const int tc8 = (t & 63) >> 3;
+#pragma unroll
+          for (int dc = 0; dc < 8; ++dc) {
+            uint4 u = *reinterpret_cast<const uint4*>(vsm + t * 128 + ((dc ^ (t & 7)) << 4));
+            if (t >= T) u = make_uint4(0u, 0u, 0u, 0u);     // tokens past the image must not reach P V
+            const unsigned short* e = reinterpret_cast<const unsigned short*>(&u);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)                     // dim dd = 8 dc + j: dd / 8 = dc, dd % 8 = j
+              *reinterpret_cast<unsigned short*>(blk0 + dc * 1024 + j * 128 + ((tc8 ^ j) << 4)) = e[j];
+          }
+        }
+        fence_async_smem();
+        mbar_arrive(bar(B_VT_READY));
+        mbar_arrive(bar(B_V_FREE));
+      }
+      // ---- softmax of the item's tiles: this thread's half of the key columns
+      const int c_split = ((KP >> 1) + 15) & ~15;
+      const int c_lo = half ? c_split : 0, c_hi = half ? KP : c_split;
+      for (int m = 0; m < n_mt && ok; ++m) {
+        if (!mbar_wait<false>(bar(B_S_FULL0 + m), cnt_m[m] & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 18); break; }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(m ? ET_S_COL1 : ET_S_COL0);
+        // up to 64 columns per TMEM round trip (the loads of a round are in flight together)
+        auto load64 = [&](int c0, uint32_t* v) -> int {
+          const int n = min(64, c_hi - c0);
+          if (n >= 32) tmem_ld32_nowait(taddr + (uint32_t)c0, v);
+          else tmem_ld16_nowait(taddr + (uint32_t)c0, v);
+          if (n == 64) tmem_ld32_nowait(taddr + (uint32_t)(c0 + 32), v + 32);
+          else if (n == 48) tmem_ld16_nowait(taddr + (uint32_t)(c0 + 32), v + 32);
+          tmem_ld_wait();
+          tmem_regs_ready16(v); tmem_regs_ready16(v + 16); tmem_regs_ready16(v + 32); tmem_regs_ready16(v + 48);
+          return n;
+        };
+        // a block of 16 loaded columns that reaches past the image: those columns become -inf (uniform branch)
+        auto mask16 = [&](int c, uint32_t* v) {
+          if (c + 16 > T) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) if (c + j >= T) v[j] = 0xff800000u;
+          }
+        };
+        // pass 1: row maximum (four independent chains)
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
+          uint32_t v[64];
+          const int n = load64(c0, v);
+#pragma unroll
+          for (int b16 = 0; b16 < 4; ++b16) {
+            if (b16 * 16 >= n) break;
+            mask16(c0 + b16 * 16, v + b16 * 16);
+#pragma unroll
+            for (int j = b16 * 16; j < b16 * 16 + 16; j += 4) {
+              mx0 = fmaxf(mx0, __uint_as_float(v[j])); mx1 = fmaxf(mx1, __uint_as_float(v[j + 1]));
+              mx2 = fmaxf(mx2, __uint_as_float(v[j + 2])); mx3 = fmaxf(mx3, __uint_as_float(v[j + 3]));
+            }
+          }
+        }
+        sm_mx[(m * 2 + half) * 128 + row] = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        // the two halves of a row meet here (an mbarrier, so that the wait is bounded like all others)
+        mbar_arrive(bar(B_MX0 + m));
+        if (!mbar_wait<false>(bar(B_MX0 + m), cnt_m[m] & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 22); break; }
+        const float mx = fmaxf(sm_mx[(m * 2) * 128 + row], sm_mx[(m * 2 + 1) * 128 + row]);
+        const float nms = -mx * scale;
+        // P may be overwritten once the P V of the tile before this one is complete
+        if (m > 0 || prev_last >= 0) {
+          const int pm = m > 0 ? 0 : prev_last;
+          if (!mbar_wait<false>(bar(B_O_FULL0 + pm), (cnt_m[pm] - 1u) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 19); break; }
+        }
+        // pass 2: p = exp2(s * scale - max * scale), row sum, bf16 P in the swizzled K-major layout
+        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+        unsigned char* prow = base_ptr + ET_OFF_P + (row >> 3) * 1024 + (row & 7) * 128;
+        const int sw = row & 7;
+        for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
+          uint32_t v[64];
+          const int n = load64(c0, v);
+#pragma unroll
+          for (int b16 = 0; b16 < 4; ++b16) {
+            if (b16 * 16 >= n) break;
+            mask16(c0 + b16 * 16, v + b16 * 16);
+#pragma unroll
+            for (int i = 2 * b16; i < 2 * b16 + 2; ++i) {   // 16-byte pieces of 8 keys; piece index kc, block kc / 8
+              const float p0 = ex2_approx(fmaf(__uint_as_float(v[8 * i]), scale, nms));
+              const float p1 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 1]), scale, nms));
+              const float p2 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 2]), scale, nms));
+              const float p3 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 3]), scale, nms));
+              const float p4 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 4]), scale, nms));
+              const float p5 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 5]), scale, nms));
+              const float p6 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 6]), scale, nms));
+              const float p7 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 7]), scale, nms));
+              l0 += p0 + p4; l1 += p1 + p5; l2 += p2 + p6; l3 += p3 + p7;
+              const int kc = (c0 >> 3) + i;
+              *reinterpret_cast<uint4*>(prow + (kc >> 3) * ET_P_BLOCK + (((kc & 7) ^ sw) << 4)) =
+                  make_uint4(pack2(p0, p1), pack2(p2, p3), pack2(p4, p5), pack2(p6, p7));
+            }
+          }
+        }
+        // this thread's reads of S_m are over: the next item's Q K^T may overwrite it
+        tc_fence_before();
+        mbar_arrive(bar(B_S_EMPTY0 + m));
+        sm_l[(m * 2 + half) * 128 + row] = (l0 + l1) + (l2 + l3);
+        fence_async_smem();                      // P must be visible to the tensor core's reads
+        mbar_arrive(bar(B_P_READY0 + m));
+        ++cnt_m[m];
+      }
+      // ---- outputs: this thread's half of the 64 dims of its row, for each tile
+      for (int m = 0; m < n_mt && ok; ++m) {
+        if (!mbar_wait<false>(bar(B_O_FULL0 + m), (cnt_m[m] - 1u) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 21); break; }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ET_O_COL + half * 32);
+        uint32_t o[32];
+        tmem_ld32(taddr, o);
+        tc_fence_before();
+        mbar_arrive(bar(B_O_EMPTY));                        // O may be overwritten by the next P V
+        const int q = m * 128 + row;
+        if (q < T) {
+          // (both halves' sums were published before P_READY, which the P V -- and so O_FULL -- waited for)
+          const float inv = 1.0f / (sm_l[(m * 2) * 128 + row] + sm_l[(m * 2 + 1) * 128 + row]);
+          uint4* dst = reinterpret_cast<uint4*>(g->out + ((size_t)r.b * T + q) * d + (size_t)r.h * 64 + half * 32);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            dst[k] = make_uint4(pack2(__uint_as_float(o[8 * k]) * inv, __uint_as_float(o[8 * k + 1]) * inv),
+                                pack2(__uint_as_float(o[8 * k + 2]) * inv, __uint_as_float(o[8 * k + 3]) * inv),
+                                pack2(__uint_as_float(o[8 * k + 4]) * inv, __uint_as_float(o[8 * k + 5]) * inv),
+                                pack2(__uint_as_float(o[8 * k + 6]) * inv, __uint_as_float(o[8 * k + 7]) * inv));
+        }
+      }
+      prev_last = n_mt - 1;
+    }
+    if (!ok) *abort_flag = 1;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_attn_encoder_tc(const AttnEncGroup* groups, int n_groups, int total_items, int* status, int sm_count,
+                                   cudaStream_t st) {
+  if (n_groups == 0 || total_items == 0) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(attn_encoder_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ET_SMEM);
+  if (e != cudaSuccess) return e;
+  const int grid = total_items < sm_count ? total_items : sm_count;
+  return launch_pdl(attn_encoder_tc_kernel, dim3(grid), dim3(ET_THREADS), ET_SMEM, st, groups, n_groups, total_items, status);
+}
+
+}  // namespace epara

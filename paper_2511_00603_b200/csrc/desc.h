@@ -109,13 +109,17 @@ struct AttnDecGroup {
                          // length may leave without the dependency wait); 0: an earlier kernel writes it
 };
 
-struct AttnEncGroup {
+struct alignas(64) AttnEncGroup {
+  CUtensorMap tmQ;       // tensor-core kernel: qkv [rows, 3d] bf16, box 64 columns x 128 rows, 128-byte swizzle
+  CUtensorMap tmKV;      // same matrix, box 64 columns x KP rows
   const bf16* qkv;       // [B*T, 3d]: q | k | v, head h at column h*hd within each
   bf16* out;             // [B*T, d]
   int B, T, H, hd;
-  int blk_start;         // first block of this group
-  int q_blocks;          // query blocks per (image, head)
-  int pad0, pad1;
+  int blk_start;         // first block (item) of this group
+  int q_blocks;          // query blocks per (image, head); 1 for the tensor-core kernel
+  int tc;                // 1: runs in the tensor-core kernel (hd 64, T <= ENC_TC_MAX_T), fixed when the model is placed
+  int KP;                // T rounded up to a multiple of 16
+  int pad[8];
 };
 
 struct AssembleGroup {   // z[b, 0] = cls + pos[0]; z[b, 1+p] = E[b*np + p] + pos[1+p]
@@ -138,7 +142,7 @@ struct OutputGroup {     // copy logits rows to the requests' buffers and take t
 namespace epara {
 static_assert(sizeof(GemmGroup) % 64 == 0, "GemmGroup holds 64-byte aligned TMA maps");
 static_assert(sizeof(NormGroup) % 8 == 0 && sizeof(GatherGroup) % 8 == 0 && sizeof(RopeGroup) % 8 == 0 &&
-              sizeof(AttnDecGroup) % 8 == 0 && sizeof(AttnEncGroup) % 8 == 0 && sizeof(AssembleGroup) % 8 == 0 &&
+              sizeof(AttnDecGroup) % 8 == 0 && sizeof(AttnEncGroup) % 64 == 0 && sizeof(AssembleGroup) % 8 == 0 &&
               sizeof(OutputGroup) % 8 == 0 && sizeof(ReqDesc) % 16 == 0 && sizeof(AttnReq) % 16 == 0,
               "descriptor sizes");
 }  // namespace epara

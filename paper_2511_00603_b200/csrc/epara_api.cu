@@ -339,6 +339,12 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
       memset(&at, 0, sizeof(at));
       at.kind = EPARA_K_ATTN_ENC; at.rows_per_req = T;
       at.aenc.qkv = qkv; at.aenc.out = a; at.aenc.T = T; at.aenc.H = d.n_heads; at.aenc.hd = d.head_dim;
+      at.aenc.KP = round_up(T, 16);
+      at.aenc.tc = (d.head_dim == 64 && T <= ENC_TC_MAX_T && bl.gemm_impl == EPARA_GEMM_TCGEN05) ? 1 : 0;
+      if (at.aenc.tc && bl.c) {
+        if (!make_tmap(&at.aenc.tmQ, qkv, Mcap, 3 * dm, 3 * dm, 128)) return EPARA_E_CUDA;
+        if (!make_tmap(&at.aenc.tmKV, qkv, Mcap, 3 * dm, 3 * dm, at.aenc.KP)) return EPARA_E_CUDA;
+      }
       m->ops.push_back(at);
       if (!add_gemm(bl, m, a, dm, Mcap, w[4], dm, dm, z, dm, w[5], EPI_RESID_F32, T)) return EPARA_E_CUDA;
       add_norm(m, z, dm, h, w[6], w[7], dm, NORM_LN, 1e-6f, T);
@@ -752,8 +758,9 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       if (who.empty()) continue;
       more = true;
       // GEMM groups go out in up to two launches: tensor-core tiles (pass 0) and the weight-streaming
-      // kernel for groups that never exceed 16 rows (pass 1)
-      const int n_pass = (kind == EPARA_K_GEMM) ? 2 : 1;
+      // kernel for groups that never exceed 16 rows (pass 1); encoder attention likewise: the tcgen05
+      // kernel (pass 0) and the mma.sync kernel for shapes it does not take (pass 1)
+      const int n_pass = (kind == EPARA_K_GEMM || kind == EPARA_K_ATTN_ENC) ? 2 : 1;
       for (int pass = 0; pass < n_pass; ++pass) {
       Launch L;
       memset(&L, 0, sizeof(L));
@@ -854,10 +861,12 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           }
           case EPARA_K_ATTN_ENC: {
             AttnEncGroup g = op.aenc;
-            g.B = a->B; g.q_blocks = attn_encoder_q_blocks(g.T); g.blk_start = total;
+            if ((g.tc != 0) != (pass == 0)) break;             // the other pass takes it
+            g.B = a->B; g.q_blocks = g.tc ? 1 : attn_encoder_q_blocks(g.T); g.blk_start = total;
             total += a->B * g.H * g.q_blocks;
             mx = std::max(mx, g.T);
-            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
+            ++n_put;
+            if (put(&g, sizeof(g), 64) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_OUTPUT: {
@@ -871,7 +880,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
         if (pass == n_pass - 1) a->cursor++;
       }
       L.p0 = total; L.p1 = mx;
-      if (kind == EPARA_K_GEMM) {
+      if (kind == EPARA_K_GEMM || kind == EPARA_K_ATTN_ENC) {
         L.n_groups = n_put;
         if (n_put == 0) continue;
       }
@@ -921,7 +930,10 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
         err = launch_attn_decode((const AttnDecGroup*)gp, L.n_groups, L.p0, L.p1 & 0xffff, L.p1 >> 16, L.p2, L.p3 >> 8,
                                  L.p3 & 255, attn_decode_fused(L.p0, L.p1 & 0xffff, L.p2, c->sm_count) ? 1 : 0, st);
         break;
-      case EPARA_K_ATTN_ENC: err = launch_attn_encoder((const AttnEncGroup*)gp, L.n_groups, L.p0, L.p1, st); break;
+      case EPARA_K_ATTN_ENC:
+        if (L.p2 == 0) err = launch_attn_encoder_tc((const AttnEncGroup*)gp, L.n_groups, L.p0, c->dev_status, c->sm_count, st);
+        else err = launch_attn_encoder((const AttnEncGroup*)gp, L.n_groups, L.p0, L.p1, st);
+        break;
       case EPARA_K_OUTPUT: launch_output((const OutputGroup*)gp, L.n_groups, L.p1, st); break;
     }
     if (prof) cudaEventRecord(slot.prof[2 * li + 1], st);

@@ -44,7 +44,13 @@ cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int tot
 void launch_attn_fill_reqs(AttnReq* reqs, const int32_t* kv_lens, const int32_t* tables, int stride, int B,
                            cudaStream_t st);
 
-// Encoder (bidirectional) attention, one block per (image, head, query block).
+// Encoder attention on tcgen05 for groups with AttnEncGroup::tc (hd 64, T <= ENC_TC_MAX_T): persistent,
+// one item per (image, head); total_items = sum of B * H.  `status` as for the GEMM.
+constexpr int ENC_TC_MAX_T = 224;
+cudaError_t launch_attn_encoder_tc(const AttnEncGroup* groups, int n_groups, int total_items, int* status, int sm_count,
+                                   cudaStream_t st);
+
+// Encoder (bidirectional) attention on mma.sync, one block per (image, head, query block).
 cudaError_t launch_attn_encoder(const AttnEncGroup* groups, int n_groups, int total_blocks, int max_T,
                                 cudaStream_t st);
 int attn_encoder_q_blocks(int T);
