@@ -6,9 +6,9 @@
 //                      item straight out of the qkv activation matrix [rows, 3d] (128-byte swizzle);
 //   warp 1 (one lane)  MMA issuer: S_m = Q_m K^T (tcgen05.mma M 128, N KP, K 64) into TMEM for both
 //                      query tiles, later O_m = P_m V (M 128, N 64, K KP) into a third TMEM region;
-//   warps 2..9         256 workers; thread = (query row, half).  First they transpose V (tokens x 64) into
-//                      V^T (64 x tokens, K-major swizzled: the B operand of P V), zeroing tokens >= T.
-//                      Softmax: two passes over the thread's half of the row of S in TMEM (reading TMEM is
+//   warps 2..9         256 workers; thread = (query row, half).  V is consumed by the MMA as the TMA wrote it
+//                      (tokens x 64 is the MN-major form of the B operand); the workers only zero its rows
+//                      >= T.  Softmax: two passes over the thread's half of the row of S in TMEM (reading TMEM is
 //                      cheap): maximum (the halves meet in shared memory), then p = exp2((s - max) * scale)
 //                      with the row sum in fp32; P goes to shared memory as bf16 in the K-major
 //                      128-byte-swizzled layout the MMA reads as its A operand.  Key columns >= T are masked
@@ -31,17 +31,15 @@ using namespace tc;
 constexpr int ET_THREADS = 320;                       // 10 warps
 constexpr int ET_Q_BYTES = 128 * 128;                 // one query tile: 128 rows of 128 bytes
 constexpr int ET_KV_BYTES = ENC_TC_MAX_T * 128;       // K or V tile at the largest KP (224 rows)
-constexpr int ET_VT_BLOCK = 64 * 128;                 // V^T: one 64-key block = 64 rows (dims) of 128 bytes
 constexpr int ET_P_BLOCK = 128 * 128;                 // P: one 64-key block = 128 rows of 128 bytes
 constexpr int ET_OFF_Q = 0;
 constexpr int ET_OFF_K = 2 * ET_Q_BYTES;
 constexpr int ET_OFF_V = ET_OFF_K + ET_KV_BYTES;
-constexpr int ET_OFF_VT = ET_OFF_V + ET_KV_BYTES;
-constexpr int ET_OFF_P = ET_OFF_VT + 4 * ET_VT_BLOCK;
+constexpr int ET_OFF_P = ET_OFF_V + ET_KV_BYTES;
 constexpr int ET_OFF_L = ET_OFF_P + 4 * ET_P_BLOCK;   // partial row sums [2 tiles][2 halves][128] fp32, then partial maxima
 constexpr int ET_OFF_BAR = ET_OFF_L + 4096;
 constexpr size_t ET_SMEM = 1024 + ET_OFF_BAR + 256;
-static_assert(ET_OFF_V % 1024 == 0 && ET_OFF_VT % 1024 == 0 && ET_OFF_P % 1024 == 0, "swizzle atoms are 1024 bytes");
+static_assert(ET_OFF_V % 1024 == 0 && ET_OFF_P % 1024 == 0, "swizzle atoms are 1024 bytes");
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -52,6 +50,19 @@ constexpr int ET_S_COL0 = 0, ET_S_COL1 = 224, ET_O_COL = 448;   // TMEM columns:
 
 enum { B_FULL_QK = 0, B_FULL_V, B_QK_FREE, B_V_FREE, B_VT_READY, B_S_FULL0, B_S_FULL1, B_S_EMPTY0, B_S_EMPTY1,
        B_P_READY0, B_P_READY1, B_O_FULL0, B_O_FULL1, B_O_EMPTY, B_MX0, B_MX1, B_COUNT };
+
+// V tile as the B operand of P V: tokens (the K dimension of the MMA) x 64 dims (N), dims contiguous =
+// MN-major.  Rows of 128 bytes, 128-byte swizzle, 8-token groups 1024 bytes apart; N = 64 is a single
+// 128-byte row, so the only stride in play is the one between 8-token groups (given in both offset fields).
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(1024 >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
 
 struct ItemRef {
   const AttnEncGroup* g;
@@ -84,7 +95,7 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
     mbar_init(bar(B_FULL_QK), 1); mbar_init(bar(B_FULL_V), 1); mbar_init(bar(B_QK_FREE), 1);
-    mbar_init(bar(B_V_FREE), 256); mbar_init(bar(B_VT_READY), 256);
+    mbar_init(bar(B_V_FREE), 1); mbar_init(bar(B_VT_READY), 256);
     mbar_init(bar(B_S_FULL0), 1); mbar_init(bar(B_S_FULL1), 1);
     mbar_init(bar(B_S_EMPTY0), 256); mbar_init(bar(B_S_EMPTY1), 256);
     mbar_init(bar(B_P_READY0), 256); mbar_init(bar(B_P_READY1), 256);
@@ -121,7 +132,7 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
         for (int m = 0; m < n_mt; ++m)
           tma_load_2d(base + ET_OFF_Q + m * ET_Q_BYTES, &g->tmQ, r.h * 64, row0 + m * 128, bar(B_FULL_QK));
         tma_load_2d(base + ET_OFF_K, &g->tmKV, d + r.h * 64, row0, bar(B_FULL_QK));
-        // V: free once the transposing warps have read the previous one
+        // V: free once the last P V of the previous item is complete
         if (!mbar_wait<false>(bar(B_V_FREE), (it & 1u) ^ 1u, abort_flag)) { ok = false; atomicExch(status, 12); break; }
         mbar_expect_tx(bar(B_FULL_V), (uint32_t)(KP * 128));
         tma_load_2d(base + ET_OFF_V, &g->tmKV, 2 * d + r.h * 64, row0, bar(B_FULL_V));
@@ -189,15 +200,16 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
           if (!mbar_wait<false>(bar(B_O_EMPTY), (n_o & 1u) ^ 1u, abort_flag)) { ok = false; atomicExch(status, 17); break; }
           ++n_o;
           tc_fence_after();
-          const uint32_t idesc_o = make_idesc(64);
+          const uint32_t idesc_o = make_idesc(64) | (1u << 16);     // B operand MN-major
           const uint32_t d_tmem = tmem_base + (uint32_t)ET_O_COL;
           const int ksteps = KP >> 4;
           for (int k = 0; k < ksteps; ++k) {
             const uint64_t dp = make_smem_desc(base + ET_OFF_P + (k >> 2) * ET_P_BLOCK) + (uint64_t)((k & 3) * 2);
-            const uint64_t dv = make_smem_desc(base + ET_OFF_VT + (k >> 2) * ET_VT_BLOCK) + (uint64_t)((k & 3) * 2);
+            const uint64_t dv = make_smem_desc_mn(base + ET_OFF_V + k * 2048);   // 16 tokens = two 8-token groups
             mma_f16(d_tmem, dp, dv, idesc_o, k > 0 ? 1u : 0u);
           }
           mma_commit(bar(B_O_FULL0 + m));
+          if (m == n_mt - 1) mma_commit(bar(B_V_FREE));     // V may be overwritten once this P V is complete
           ++cnt_pv[m];
           // scores of the next item: tile 0 after this item's first P V, the rest after its last
           if (has_next) {
@@ -230,32 +242,13 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
       const ItemRef r = find_item(groups, n_groups, item);
       const AttnEncGroup* g = r.g;
       const int T = g->T, KP = g->KP, d = g->H * 64, n_mt = (T + 127) >> 7;
-      // ---- V (tokens x 64, swizzled by the TMA) -> V^T (64 x tokens, K-major swizzled), tokens >= T zeroed.
-      // V tile: token t, 16-byte piece dc (dims 8 dc .. 8 dc + 7) sits at t * 128 + ((dc ^ (t & 7)) << 4).
-      // V^T: dim dd, token t sits in block t / 64 at dd/8 * 1024 + dd%8 * 128 + (((t%64)/8 ^ dd%8) << 4) + t%8 * 2.
-      // (the previous item's last P V, which read V^T, is complete: these threads waited for its O)
+      // ---- V is consumed by the tensor core as the TMA wrote it.  Its rows T .. KP-1 are another image's
+      // tokens or stale memory; they meet P columns that are exactly zero, but 0 x NaN is NaN: zero them.
       if (!mbar_wait<false>(bar(B_FULL_V), it & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 20); break; }
-      {
-        const unsigned char* vsm = base_ptr + ET_OFF_V;
-        unsigned char* vt = base_ptr + ET_OFF_VT;
-        const int t = wtid;                                 // one token per thread (KP <= 224 < 256), all 8 dim pieces
-        if (t < KP) {
-          unsigned char* blk0 = vt + (t >> 6) * ET_VT_BLOCK + (t & 7) * 2;
-          const int tc8 = (t & 63) >> 3;
-#pragma unroll
-          for (int dc = 0; dc < 8; ++dc) {
-            uint4 u = *reinterpret_cast<const uint4*>(vsm + t * 128 + ((dc ^ (t & 7)) << 4));
-            if (t >= T) u = make_uint4(0u, 0u, 0u, 0u);     // tokens past the image must not reach P V
-            const unsigned short* e = reinterpret_cast<const unsigned short*>(&u);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)                     // dim dd = 8 dc + j: dd / 8 = dc, dd % 8 = j
-              *reinterpret_cast<unsigned short*>(blk0 + dc * 1024 + j * 128 + ((tc8 ^ j) << 4)) = e[j];
-          }
-        }
-        fence_async_smem();
-        mbar_arrive(bar(B_VT_READY));
-        mbar_arrive(bar(B_V_FREE));
-      }
+      if (wtid < (KP - T) * 8)
+        *reinterpret_cast<uint4*>(base_ptr + ET_OFF_V + (T + (wtid >> 3)) * 128 + (wtid & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+      fence_async_smem();
+      mbar_arrive(bar(B_VT_READY));
       // ---- softmax of the item's tiles: this thread's half of the key columns
       const int c_split = ((KP >> 1) + 15) & ~15;
       const int c_lo = half ? c_split : 0, c_hi = half ? KP : c_split;
