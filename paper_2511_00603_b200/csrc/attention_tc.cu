@@ -256,38 +256,33 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
         if (!mbar_wait<false>(bar(B_S_FULL0 + m), cnt_m[m] & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 18); break; }
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(m ? ET_S_COL1 : ET_S_COL0);
-        // up to 64 columns per TMEM round trip (the loads of a round are in flight together)
-        auto load64 = [&](int c0, uint32_t* v) -> int {
-          const int n = min(64, c_hi - c0);
-          if (n >= 32) tmem_ld32_nowait(taddr + (uint32_t)c0, v);
-          else tmem_ld16_nowait(taddr + (uint32_t)c0, v);
-          if (n == 64) tmem_ld32_nowait(taddr + (uint32_t)(c0 + 32), v + 32);
-          else if (n == 48) tmem_ld16_nowait(taddr + (uint32_t)(c0 + 32), v + 32);
-          tmem_ld_wait();
-          tmem_regs_ready16(v); tmem_regs_ready16(v + 16); tmem_regs_ready16(v + 32); tmem_regs_ready16(v + 48);
-          return n;
-        };
-        // a block of 16 loaded columns that reaches past the image: those columns become -inf (uniform branch)
-        auto mask16 = [&](int c, uint32_t* v) {
+        // The thread's half of the row (at most 112 columns) is read from TMEM once, all loads in flight
+        // together, and stays in registers for both the maximum and the exponentials.
+        const int n16 = (c_hi - c_lo) >> 4;                 // 16-column blocks of this half: 0..7
+        uint32_t v[112];
+#pragma unroll
+        for (int b16 = 0; b16 < 7; ++b16)
+          if (b16 < n16) tmem_ld16_nowait(taddr + (uint32_t)(c_lo + 16 * b16), v + 16 * b16);
+        tmem_ld_wait();
+#pragma unroll
+        for (int b16 = 0; b16 < 7; ++b16) tmem_regs_ready16(v + 16 * b16);
+        // this thread's reads of S_m are over: the next item's Q K^T may overwrite it
+        tc_fence_before();
+        mbar_arrive(bar(B_S_EMPTY0 + m));
+        // row maximum (four independent chains); columns past the image become -inf (uniform branch per block)
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+        for (int b16 = 0; b16 < 7; ++b16) {
+          if (b16 >= n16) break;
+          const int c = c_lo + 16 * b16;
           if (c + 16 > T) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) if (c + j >= T) v[j] = 0xff800000u;
+            for (int j = 0; j < 16; ++j) if (c + j >= T) v[16 * b16 + j] = 0xff800000u;
           }
-        };
-        // pass 1: row maximum (four independent chains)
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-        for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
-          uint32_t v[64];
-          const int n = load64(c0, v);
 #pragma unroll
-          for (int b16 = 0; b16 < 4; ++b16) {
-            if (b16 * 16 >= n) break;
-            mask16(c0 + b16 * 16, v + b16 * 16);
-#pragma unroll
-            for (int j = b16 * 16; j < b16 * 16 + 16; j += 4) {
-              mx0 = fmaxf(mx0, __uint_as_float(v[j])); mx1 = fmaxf(mx1, __uint_as_float(v[j + 1]));
-              mx2 = fmaxf(mx2, __uint_as_float(v[j + 2])); mx3 = fmaxf(mx3, __uint_as_float(v[j + 3]));
-            }
+          for (int j = 16 * b16; j < 16 * b16 + 16; j += 4) {
+            mx0 = fmaxf(mx0, __uint_as_float(v[j])); mx1 = fmaxf(mx1, __uint_as_float(v[j + 1]));
+            mx2 = fmaxf(mx2, __uint_as_float(v[j + 2])); mx3 = fmaxf(mx3, __uint_as_float(v[j + 3]));
           }
         }
         sm_mx[(m * 2 + half) * 128 + row] = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
@@ -301,37 +296,26 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
           const int pm = m > 0 ? 0 : prev_last;
           if (!mbar_wait<false>(bar(B_O_FULL0 + pm), (cnt_m[pm] - 1u) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 19); break; }
         }
-        // pass 2: p = exp2(s * scale - max * scale), row sum, bf16 P in the swizzled K-major layout
+        // p = exp2(s * scale - max * scale), row sum, bf16 P in the swizzled K-major layout
         float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
         unsigned char* prow = base_ptr + ET_OFF_P + (row >> 3) * 1024 + (row & 7) * 128;
         const int sw = row & 7;
-        for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
-          uint32_t v[64];
-          const int n = load64(c0, v);
 #pragma unroll
-          for (int b16 = 0; b16 < 4; ++b16) {
-            if (b16 * 16 >= n) break;
-            mask16(c0 + b16 * 16, v + b16 * 16);
-#pragma unroll
-            for (int i = 2 * b16; i < 2 * b16 + 2; ++i) {   // 16-byte pieces of 8 keys; piece index kc, block kc / 8
-              const float p0 = ex2_approx(fmaf(__uint_as_float(v[8 * i]), scale, nms));
-              const float p1 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 1]), scale, nms));
-              const float p2 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 2]), scale, nms));
-              const float p3 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 3]), scale, nms));
-              const float p4 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 4]), scale, nms));
-              const float p5 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 5]), scale, nms));
-              const float p6 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 6]), scale, nms));
-              const float p7 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 7]), scale, nms));
-              l0 += p0 + p4; l1 += p1 + p5; l2 += p2 + p6; l3 += p3 + p7;
-              const int kc = (c0 >> 3) + i;
-              *reinterpret_cast<uint4*>(prow + (kc >> 3) * ET_P_BLOCK + (((kc & 7) ^ sw) << 4)) =
-                  make_uint4(pack2(p0, p1), pack2(p2, p3), pack2(p4, p5), pack2(p6, p7));
-            }
-          }
+        for (int i = 0; i < 14; ++i) {                      // 16-byte pieces of 8 keys; piece index kc, block kc / 8
+          if (i >= 2 * n16) break;
+          const float p0 = ex2_approx(fmaf(__uint_as_float(v[8 * i]), scale, nms));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 1]), scale, nms));
+          const float p2 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 2]), scale, nms));
+          const float p3 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 3]), scale, nms));
+          const float p4 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 4]), scale, nms));
+          const float p5 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 5]), scale, nms));
+          const float p6 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 6]), scale, nms));
+          const float p7 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 7]), scale, nms));
+          l0 += p0 + p4; l1 += p1 + p5; l2 += p2 + p6; l3 += p3 + p7;
+          const int kc = (c_lo >> 3) + i;
+          *reinterpret_cast<uint4*>(prow + (kc >> 3) * ET_P_BLOCK + (((kc & 7) ^ sw) << 4)) =
+              make_uint4(pack2(p0, p1), pack2(p2, p3), pack2(p4, p5), pack2(p6, p7));
         }
-        // this thread's reads of S_m are over: the next item's Q K^T may overwrite it
-        tc_fence_before();
-        mbar_arrive(bar(B_S_EMPTY0 + m));
         sm_l[(m * 2 + half) * 128 + row] = (l0 + l1) + (l2 + l3);
         fence_async_smem();                      // P must be visible to the tensor core's reads
         mbar_arrive(bar(B_P_READY0 + m));
@@ -341,9 +325,9 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
       for (int m = 0; m < n_mt && ok; ++m) {
         if (!mbar_wait<false>(bar(B_O_FULL0 + m), (cnt_m[m] - 1u) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 21); break; }
         tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ET_O_COL + half * 32);
+        const uint32_t oaddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ET_O_COL + half * 32);
         uint32_t o[32];
-        tmem_ld32(taddr, o);
+        tmem_ld32(oaddr, o);
         tc_fence_before();
         mbar_arrive(bar(B_O_EMPTY));                        // O may be overwritten by the next P V
         const int q = m * 128 + row;
