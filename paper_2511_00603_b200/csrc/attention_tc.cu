@@ -46,10 +46,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
-constexpr int ET_S_COL0 = 0, ET_S_COL1 = 224, ET_O_COL = 448;   // TMEM columns: S_0, S_1, O (64)
+// TMEM columns: S_0 and S_1.  O_m = P_m V is written over the first 64 columns of S_m, which the softmax
+// has read out by then; the next item's S_m waits until O_m has been read out in turn.
+constexpr int ET_S_COL0 = 0, ET_S_COL1 = 256;
 
-enum { B_FULL_QK = 0, B_FULL_V, B_QK_FREE, B_V_FREE, B_VT_READY, B_S_FULL0, B_S_FULL1, B_S_EMPTY0, B_S_EMPTY1,
-       B_P_READY0, B_P_READY1, B_O_FULL0, B_O_FULL1, B_O_EMPTY, B_MX0, B_MX1, B_COUNT };
+enum { B_FULL_QK = 0, B_FULL_V, B_QK_FREE, B_V_FREE, B_VT_READY, B_S_FULL0, B_S_FULL1,
+       B_P_READY0, B_P_READY1, B_O_FULL0, B_O_FULL1, B_O_EMPTY0, B_O_EMPTY1, B_MX0, B_MX1, B_COUNT };
 
 // V tile as the B operand of P V: tokens (the K dimension of the MMA) x 64 dims (N), dims contiguous =
 // MN-major.  Rows of 128 bytes, 128-byte swizzle, 8-token groups 1024 bytes apart; N = 64 is a single
@@ -97,9 +99,9 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
     mbar_init(bar(B_FULL_QK), 1); mbar_init(bar(B_FULL_V), 1); mbar_init(bar(B_QK_FREE), 1);
     mbar_init(bar(B_V_FREE), 1); mbar_init(bar(B_VT_READY), 256);
     mbar_init(bar(B_S_FULL0), 1); mbar_init(bar(B_S_FULL1), 1);
-    mbar_init(bar(B_S_EMPTY0), 256); mbar_init(bar(B_S_EMPTY1), 256);
     mbar_init(bar(B_P_READY0), 256); mbar_init(bar(B_P_READY1), 256);
-    mbar_init(bar(B_O_FULL0), 1); mbar_init(bar(B_O_FULL1), 1); mbar_init(bar(B_O_EMPTY), 256);
+    mbar_init(bar(B_O_FULL0), 1); mbar_init(bar(B_O_FULL1), 1);
+    mbar_init(bar(B_O_EMPTY0), 256); mbar_init(bar(B_O_EMPTY1), 256);
     mbar_init(bar(B_MX0), 256); mbar_init(bar(B_MX1), 256);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -146,19 +148,20 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    // Order of issue per item: P_0 V, then Q_0 K^T of the NEXT item, then P_1 V, then Q_1 K^T of the next
-    // item -- so that the scores of the next item are waiting in TMEM when the softmax warps get there.
+    // Order of issue per item: P_0 V, P_1 V, then Q_0 K^T and Q_1 K^T of the NEXT item, each as soon as
+    // the workers have read O_0 / O_1 out of the TMEM region it overwrites -- the scores of the next item
+    // are waiting in TMEM when the softmax warps get there.
     // Barriers of the first query tile complete once per item, those of the second once per item with two
-    // tiles, O_EMPTY once per tile: each has its own use counter (items of different models mix).
+    // tiles: each has its own use counter (items of different models mix).
     if (lane == 0) {
       bool ok = true;
-      uint32_t n_o = 0;
       uint32_t cnt_s[2] = {0, 0};               // S = Q K^T issued so far, per tile index
       uint32_t cnt_pv[2] = {0, 0};              // P V issued so far, per tile index
       uint32_t cnt_qk = 0;                      // items whose Q / K have been consumed
       // Q_m K^T of an item (its Q and K must have landed: caller waited FULL_QK)
       auto issue_s = [&](const AttnEncGroup* g, int m) -> bool {
-        if (!mbar_wait<false>(bar(B_S_EMPTY0 + m), (cnt_s[m] & 1u) ^ 1u, abort_flag)) { atomicExch(status, 14); return false; }
+        // the region still holds O_m of the previous item with this tile until the workers have read it
+        if (!mbar_wait<false>(bar(B_O_EMPTY0 + m), (cnt_s[m] & 1u) ^ 1u, abort_flag)) { atomicExch(status, 14); return false; }
         tc_fence_after();
         const uint32_t idesc_s = make_idesc(g->KP);
         const uint64_t dq = make_smem_desc(base + ET_OFF_Q + m * ET_Q_BYTES), dk = make_smem_desc(base + ET_OFF_K);
@@ -196,12 +199,9 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
         if (!mbar_wait<false>(bar(B_VT_READY), it & 1u, abort_flag)) { ok = false; atomicExch(status, 15); break; }
         for (int m = 0; m < n_mt && ok; ++m) {
           if (!mbar_wait<false>(bar(B_P_READY0 + m), cnt_pv[m] & 1u, abort_flag)) { ok = false; atomicExch(status, 16); break; }
-          // O must have been read out by the warps that store the previous tile
-          if (!mbar_wait<false>(bar(B_O_EMPTY), (n_o & 1u) ^ 1u, abort_flag)) { ok = false; atomicExch(status, 17); break; }
-          ++n_o;
-          tc_fence_after();
+          tc_fence_after();                     // (P_READY also says that every worker has read S_m out)
           const uint32_t idesc_o = make_idesc(64) | (1u << 16);     // B operand MN-major
-          const uint32_t d_tmem = tmem_base + (uint32_t)ET_O_COL;
+          const uint32_t d_tmem = tmem_base + (uint32_t)(m ? ET_S_COL1 : ET_S_COL0);
           const int ksteps = KP >> 4;
           for (int k = 0; k < ksteps; ++k) {
             const uint64_t dp = make_smem_desc(base + ET_OFF_P + (k >> 2) * ET_P_BLOCK) + (uint64_t)((k & 3) * 2);
@@ -211,17 +211,12 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
           mma_commit(bar(B_O_FULL0 + m));
           if (m == n_mt - 1) mma_commit(bar(B_V_FREE));     // V may be overwritten once this P V is complete
           ++cnt_pv[m];
-          // scores of the next item: tile 0 after this item's first P V, the rest after its last
-          if (has_next) {
-            if (m == 0) {
-              ok = wait_qk() && issue_s(g_next, 0);
-              if (ok && n_mt_next == 1) mma_commit(bar(B_QK_FREE));
-            }
-            if (ok && m == n_mt - 1 && n_mt_next == 2) {
-              ok = issue_s(g_next, 1);
-              if (ok) mma_commit(bar(B_QK_FREE));
-            }
-          }
+        }
+        // scores of the next item
+        if (ok && has_next) {
+          ok = wait_qk();
+          for (int m = 0; m < n_mt_next && ok; ++m) ok = issue_s(g_next, m);
+          if (ok) mma_commit(bar(B_QK_FREE));
         }
       }
       if (!ok) *abort_flag = 1;
@@ -266,9 +261,7 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
         tmem_ld_wait();
 #pragma unroll
         for (int b16 = 0; b16 < 7; ++b16) tmem_regs_ready16(v + 16 * b16);
-        // this thread's reads of S_m are over: the next item's Q K^T may overwrite it
-        tc_fence_before();
-        mbar_arrive(bar(B_S_EMPTY0 + m));
+        tc_fence_before();                                  // (this thread's reads of S_m are over; P_READY tells the MMA warp)
         // row maximum (four independent chains); columns past the image become -inf (uniform branch per block)
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
@@ -325,11 +318,11 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
       for (int m = 0; m < n_mt && ok; ++m) {
         if (!mbar_wait<false>(bar(B_O_FULL0 + m), (cnt_m[m] - 1u) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 21); break; }
         tc_fence_after();
-        const uint32_t oaddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ET_O_COL + half * 32);
+        const uint32_t oaddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((m ? ET_S_COL1 : ET_S_COL0) + half * 32);
         uint32_t o[32];
         tmem_ld32(oaddr, o);
         tc_fence_before();
-        mbar_arrive(bar(B_O_EMPTY));                        // O may be overwritten by the next P V
+        mbar_arrive(bar(B_O_EMPTY0 + m));                   // the next item's S_m may overwrite the region
         const int q = m * 128 + row;
         if (q < T) {
           // (both halves' sums were published before P_READY, which the P V -- and so O_FULL -- waited for)
