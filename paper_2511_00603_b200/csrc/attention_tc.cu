@@ -6,13 +6,13 @@
 //                      item straight out of the qkv activation matrix [rows, 3d] (128-byte swizzle);
 //   warp 1 (one lane)  MMA issuer: S_m = Q_m K^T (tcgen05.mma M 128, N KP, K 64) into TMEM for both
 //                      query tiles, later O_m = P_m V (M 128, N 64, K KP) into a third TMEM region;
-//   warps 2..9         256 workers; thread = (query row, half).  V is consumed by the MMA as the TMA wrote it
+//   warps 2..13        384 workers; thread = (query row, part of the key columns).  V is consumed by the MMA as the TMA wrote it
 //                      (tokens x 64 is the MN-major form of the B operand); the workers only zero its rows
-//                      >= T.  Softmax: two passes over the thread's half of the row of S in TMEM (reading TMEM is
-//                      cheap): maximum (the halves meet in shared memory), then p = exp2((s - max) * scale)
+//                      >= T.  Softmax: the thread reads its part of the row of S from TMEM once and keeps it in
+//                      registers: maximum (the parts meet in shared memory), then p = exp2((s - max) * scale)
 //                      with the row sum in fp32; P goes to shared memory as bf16 in the K-major
 //                      128-byte-swizzled layout the MMA reads as its A operand.  Key columns >= T are masked
-//                      by selection.  Last they read their half of O from TMEM, divide by the row sum and
+//                      by selection.  Last two of the three parts read half of O each from TMEM, divide by the row sum and
 //                      store bf16 (rows >= T are not stored).
 // Rows of the Q / K / V tiles past the image's T tokens belong to the next image or lie past the matrix
 // (TMA fills those with zeros); they only ever reach masked columns, zeroed V^T columns or rows that
@@ -28,7 +28,11 @@ namespace {
 
 using namespace tc;
 
-constexpr int ET_THREADS = 320;                       // 10 warps
+constexpr int ET_NS = 3;                              // worker threads per query row: each takes a part of the key columns
+constexpr int ET_WORKERS = 128 * ET_NS;
+constexpr int ET_THREADS = 64 + ET_WORKERS;
+constexpr int ET_NB = (ENC_TC_MAX_T / 16 + ET_NS - 1) / ET_NS;   // 16-column blocks per thread at most (5)
+constexpr int ET_OUT_PARTS = 2;                       // parts that store output: 32 of the 64 dims each
 constexpr int ET_Q_BYTES = 128 * 128;                 // one query tile: 128 rows of 128 bytes
 constexpr int ET_KV_BYTES = ENC_TC_MAX_T * 128;       // K or V tile at the largest KP (224 rows)
 constexpr int ET_P_BLOCK = 128 * 128;                 // P: one 64-key block = 128 rows of 128 bytes
@@ -36,8 +40,9 @@ constexpr int ET_OFF_Q = 0;
 constexpr int ET_OFF_K = 2 * ET_Q_BYTES;
 constexpr int ET_OFF_V = ET_OFF_K + ET_KV_BYTES;
 constexpr int ET_OFF_P = ET_OFF_V + ET_KV_BYTES;
-constexpr int ET_OFF_L = ET_OFF_P + 4 * ET_P_BLOCK;   // partial row sums [2 tiles][2 halves][128] fp32, then partial maxima
-constexpr int ET_OFF_BAR = ET_OFF_L + 4096;
+constexpr int ET_OFF_L = ET_OFF_P + 4 * ET_P_BLOCK;   // partial row sums [2 tiles][parts][128] fp32, then partial maxima (4 KB each at most)
+constexpr int ET_OFF_BAR = ET_OFF_L + 8192;
+static_assert(2 * 2 * ET_NS * 128 * 4 <= 8192, "row sums and maxima");
 constexpr size_t ET_SMEM = 1024 + ET_OFF_BAR + 256;
 static_assert(ET_OFF_V % 1024 == 0 && ET_OFF_P % 1024 == 0, "swizzle atoms are 1024 bytes");
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -50,7 +55,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // has read out by then; the next item's S_m waits until O_m has been read out in turn.
 constexpr int ET_S_COL0 = 0, ET_S_COL1 = 256;
 
-enum { B_FULL_QK = 0, B_FULL_V, B_QK_FREE, B_V_FREE, B_VT_READY, B_S_FULL0, B_S_FULL1,
+enum { B_FULL_QK = 0, B_FULL_V, B_QK_FREE, B_V_FREE, B_S_FULL0, B_S_FULL1,
        B_P_READY0, B_P_READY1, B_O_FULL0, B_O_FULL1, B_O_EMPTY0, B_O_EMPTY1, B_MX0, B_MX1, B_COUNT };
 
 // V tile as the B operand of P V: tokens (the K dimension of the MMA) x 64 dims (N), dims contiguous =
@@ -97,12 +102,12 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
     mbar_init(bar(B_FULL_QK), 1); mbar_init(bar(B_FULL_V), 1); mbar_init(bar(B_QK_FREE), 1);
-    mbar_init(bar(B_V_FREE), 1); mbar_init(bar(B_VT_READY), 256);
+    mbar_init(bar(B_V_FREE), 1);
     mbar_init(bar(B_S_FULL0), 1); mbar_init(bar(B_S_FULL1), 1);
-    mbar_init(bar(B_P_READY0), 256); mbar_init(bar(B_P_READY1), 256);
+    mbar_init(bar(B_P_READY0), ET_WORKERS); mbar_init(bar(B_P_READY1), ET_WORKERS);
     mbar_init(bar(B_O_FULL0), 1); mbar_init(bar(B_O_FULL1), 1);
-    mbar_init(bar(B_O_EMPTY0), 256); mbar_init(bar(B_O_EMPTY1), 256);
-    mbar_init(bar(B_MX0), 256); mbar_init(bar(B_MX1), 256);
+    mbar_init(bar(B_O_EMPTY0), ET_WORKERS); mbar_init(bar(B_O_EMPTY1), ET_WORKERS);
+    mbar_init(bar(B_MX0), ET_WORKERS); mbar_init(bar(B_MX1), ET_WORKERS);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -196,7 +201,6 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
           g_next = find_item(groups, n_groups, item + gridDim.x).g;
           n_mt_next = (g_next->T + 127) >> 7;
         }
-        if (!mbar_wait<false>(bar(B_VT_READY), it & 1u, abort_flag)) { ok = false; atomicExch(status, 15); break; }
         for (int m = 0; m < n_mt && ok; ++m) {
           if (!mbar_wait<false>(bar(B_P_READY0 + m), cnt_pv[m] & 1u, abort_flag)) { ok = false; atomicExch(status, 16); break; }
           tc_fence_after();                     // (P_READY also says that every worker has read S_m out)
@@ -222,13 +226,13 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
       if (!ok) *abort_flag = 1;
     }
   } else {
-    // ------------------------------------------------------------------ workers (warps 2..9, 256 threads)
-    // Thread (quarter, lane, half): query row quarter*32 + lane of the current tile, and one half of the
-    // key columns for the softmax / one half of the 64 output dims for the store.
-    const int quarter = warp & 3, row = quarter * 32 + lane, half = (warp - 2) >> 2;
-    const int wtid = threadIdx.x - 64;                      // 0..255
+    // ------------------------------------------------------------------ workers (warps 2.., ET_WORKERS threads)
+    // Thread (quarter, lane, part): query row quarter*32 + lane of the current tile, and one part of the
+    // key columns for the softmax; parts 0 and 1 also store one half of the 64 output dims.
+    const int quarter = warp & 3, row = quarter * 32 + lane, part = (warp - 2) >> 2;
+    const int wtid = threadIdx.x - 64;
     const float scale = 1.4426950408889634f * 0.125f;       // log2(e) / sqrt(64)
-    float* sm_mx = sm_l + 512;                              // [2 tiles][2 halves][128] partial row maxima
+    float* sm_mx = sm_l + 2 * ET_NS * 128;                  // [2 tiles][parts][128] partial row maxima
     bool ok = true;
     uint32_t it = 0;
     uint32_t cnt_m[2] = {0, 0};                             // tiles processed so far, per tile index
@@ -237,35 +241,30 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
       const ItemRef r = find_item(groups, n_groups, item);
       const AttnEncGroup* g = r.g;
       const int T = g->T, KP = g->KP, d = g->H * 64, n_mt = (T + 127) >> 7;
-      // ---- V is consumed by the tensor core as the TMA wrote it.  Its rows T .. KP-1 are another image's
-      // tokens or stale memory; they meet P columns that are exactly zero, but 0 x NaN is NaN: zero them.
-      if (!mbar_wait<false>(bar(B_FULL_V), it & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 20); break; }
-      if (wtid < (KP - T) * 8)
-        *reinterpret_cast<uint4*>(base_ptr + ET_OFF_V + (T + (wtid >> 3)) * 128 + (wtid & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
-      fence_async_smem();
-      mbar_arrive(bar(B_VT_READY));
       // ---- softmax of the item's tiles: this thread's half of the key columns
-      const int c_split = ((KP >> 1) + 15) & ~15;
-      const int c_lo = half ? c_split : 0, c_hi = half ? KP : c_split;
+      // the KP / 16 blocks of 16 columns are dealt to the parts as evenly as possible
+      const int nb = KP >> 4, nb_lo = nb / ET_NS, nb_rem = nb % ET_NS;
+      const int b_lo = part * nb_lo + min(part, nb_rem);
+      const int c_lo = b_lo * 16, c_hi = c_lo + (nb_lo + (part < nb_rem ? 1 : 0)) * 16;
       for (int m = 0; m < n_mt && ok; ++m) {
         if (!mbar_wait<false>(bar(B_S_FULL0 + m), cnt_m[m] & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 18); break; }
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(m ? ET_S_COL1 : ET_S_COL0);
         // The thread's half of the row (at most 112 columns) is read from TMEM once, all loads in flight
         // together, and stays in registers for both the maximum and the exponentials.
-        const int n16 = (c_hi - c_lo) >> 4;                 // 16-column blocks of this half: 0..7
-        uint32_t v[112];
+        const int n16 = (c_hi - c_lo) >> 4;                 // 16-column blocks of this part: 0..ET_NB
+        uint32_t v[16 * ET_NB];
 #pragma unroll
-        for (int b16 = 0; b16 < 7; ++b16)
+        for (int b16 = 0; b16 < ET_NB; ++b16)
           if (b16 < n16) tmem_ld16_nowait(taddr + (uint32_t)(c_lo + 16 * b16), v + 16 * b16);
         tmem_ld_wait();
 #pragma unroll
-        for (int b16 = 0; b16 < 7; ++b16) tmem_regs_ready16(v + 16 * b16);
+        for (int b16 = 0; b16 < ET_NB; ++b16) tmem_regs_ready16(v + 16 * b16);
         tc_fence_before();                                  // (this thread's reads of S_m are over; P_READY tells the MMA warp)
         // row maximum (four independent chains); columns past the image become -inf (uniform branch per block)
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-        for (int b16 = 0; b16 < 7; ++b16) {
+        for (int b16 = 0; b16 < ET_NB; ++b16) {
           if (b16 >= n16) break;
           const int c = c_lo + 16 * b16;
           if (c + 16 > T) {
@@ -278,11 +277,13 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
             mx2 = fmaxf(mx2, __uint_as_float(v[j + 2])); mx3 = fmaxf(mx3, __uint_as_float(v[j + 3]));
           }
         }
-        sm_mx[(m * 2 + half) * 128 + row] = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        sm_mx[(m * ET_NS + part) * 128 + row] = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         // the two halves of a row meet here (an mbarrier, so that the wait is bounded like all others)
         mbar_arrive(bar(B_MX0 + m));
         if (!mbar_wait<false>(bar(B_MX0 + m), cnt_m[m] & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 22); break; }
-        const float mx = fmaxf(sm_mx[(m * 2) * 128 + row], sm_mx[(m * 2 + 1) * 128 + row]);
+        float mx = sm_mx[(m * ET_NS) * 128 + row];
+#pragma unroll
+        for (int p2 = 1; p2 < ET_NS; ++p2) mx = fmaxf(mx, sm_mx[(m * ET_NS + p2) * 128 + row]);
         const float nms = -mx * scale;
         // P may be overwritten once the P V of the tile before this one is complete
         if (m > 0 || prev_last >= 0) {
@@ -294,7 +295,7 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
         unsigned char* prow = base_ptr + ET_OFF_P + (row >> 3) * 1024 + (row & 7) * 128;
         const int sw = row & 7;
 #pragma unroll
-        for (int i = 0; i < 14; ++i) {                      // 16-byte pieces of 8 keys; piece index kc, block kc / 8
+        for (int i = 0; i < 2 * ET_NB; ++i) {               // 16-byte pieces of 8 keys; piece index kc, block kc / 8
           if (i >= 2 * n16) break;
           const float p0 = ex2_approx(fmaf(__uint_as_float(v[8 * i]), scale, nms));
           const float p1 = ex2_approx(fmaf(__uint_as_float(v[8 * i + 1]), scale, nms));
@@ -309,25 +310,39 @@ attn_encoder_tc_kernel(const AttnEncGroup* __restrict__ groups, int n_groups, in
           *reinterpret_cast<uint4*>(prow + (kc >> 3) * ET_P_BLOCK + (((kc & 7) ^ sw) << 4)) =
               make_uint4(pack2(p0, p1), pack2(p2, p3), pack2(p4, p5), pack2(p6, p7));
         }
-        sm_l[(m * 2 + half) * 128 + row] = (l0 + l1) + (l2 + l3);
-        fence_async_smem();                      // P must be visible to the tensor core's reads
+        sm_l[(m * ET_NS + part) * 128 + row] = (l0 + l1) + (l2 + l3);
+        if (m == 0) {
+          // V is consumed by the tensor core as the TMA wrote it.  Its rows T .. KP-1 are another image's tokens
+          // or stale memory; they meet P columns that are exactly zero, but 0 x NaN is NaN: zero them before the
+          // first tile's P is reported (every P V of the item is issued after that report).  Waiting for V
+          // only here leaves its load, which starts when the previous item's last P V is done, a whole
+          // softmax to arrive.
+          if (!mbar_wait<false>(bar(B_FULL_V), it & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 20); break; }
+          if (wtid < (KP - T) * 8)
+            *reinterpret_cast<uint4*>(base_ptr + ET_OFF_V + (T + (wtid >> 3)) * 128 + (wtid & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_async_smem();                      // P (and the zeroed V rows) must be visible to the tensor core's reads
         mbar_arrive(bar(B_P_READY0 + m));
         ++cnt_m[m];
       }
-      // ---- outputs: this thread's half of the 64 dims of its row, for each tile
+      // ---- outputs: parts 0 and 1 read one half of the 64 dims of their row, for each tile
       for (int m = 0; m < n_mt && ok; ++m) {
         if (!mbar_wait<false>(bar(B_O_FULL0 + m), (cnt_m[m] - 1u) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 21); break; }
+        if (part >= ET_OUT_PARTS) { mbar_arrive(bar(B_O_EMPTY0 + m)); continue; }
         tc_fence_after();
-        const uint32_t oaddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((m ? ET_S_COL1 : ET_S_COL0) + half * 32);
+        const uint32_t oaddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((m ? ET_S_COL1 : ET_S_COL0) + part * 32);
         uint32_t o[32];
         tmem_ld32(oaddr, o);
         tc_fence_before();
         mbar_arrive(bar(B_O_EMPTY0 + m));                   // the next item's S_m may overwrite the region
         const int q = m * 128 + row;
         if (q < T) {
-          // (both halves' sums were published before P_READY, which the P V -- and so O_FULL -- waited for)
-          const float inv = 1.0f / (sm_l[(m * 2) * 128 + row] + sm_l[(m * 2 + 1) * 128 + row]);
-          uint4* dst = reinterpret_cast<uint4*>(g->out + ((size_t)r.b * T + q) * d + (size_t)r.h * 64 + half * 32);
+          // (all parts' sums were published before P_READY, which the P V -- and so O_FULL -- waited for)
+          float l = sm_l[(m * ET_NS) * 128 + row];
+#pragma unroll
+          for (int p2 = 1; p2 < ET_NS; ++p2) l += sm_l[(m * ET_NS + p2) * 128 + row];
+          const float inv = 1.0f / l;
+          uint4* dst = reinterpret_cast<uint4*>(g->out + ((size_t)r.b * T + q) * d + (size_t)r.h * 64 + part * 32);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             dst[k] = make_uint4(pack2(__uint_as_float(o[8 * k]) * inv, __uint_as_float(o[8 * k + 1]) * inv),
