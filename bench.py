@@ -24,9 +24,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # DRAM bytes (read + write) per GEMM launch of the mixed step, from one ncu pass over the 130 GEMM launches
-# of a step (65 tensor-core + 65 weight-streaming: 16.10 + 8.77 GB and 2.08 + 0.0005 GB; see
+# of a step (65 tensor-core + 65 weight-streaming: 16.15 + 8.83 GB and 2.08 + 0.0007 GB; see
 # profiles/gemm_kernels_mixed_step_dram_traffic.md).  Set to None when the GEMM kernels change.
-GEMM_TRAFFIC_PER_LAUNCH_MIXED = (16104832768 + 8773382144 + 2083244288 + 522240) / 130
+GEMM_TRAFFIC_PER_LAUNCH_MIXED = (16145210880 + 8828690176 + 2083236096 + 654848) / 130
 
 METRIC = "mixed-category requests/s"
 UNIT = "requests/s"
