@@ -103,6 +103,23 @@ def test_small_vit_with_biases(mods, impl):
     srv.close()
 
 
+@pytest.mark.parametrize("img,patch,T", [(128, 16, 65), (176, 16, 122), (192, 16, 145), (208, 16, 170), (240, 16, 226)])
+def test_vit_token_counts_around_the_attention_tiles(mods, img, patch, T):
+    """Encoder attention at token counts on both sides of its tile edges: one 128-row query tile
+    only partly filled (65, 122), a second tile with 17 and 42 rows (145, 170), key counts that are
+    not multiples of 16, and 226 tokens, which is past the single-tile kernel's range and takes the
+    flash-loop kernel.  Head size 64, three images so that the items do not fill the grid evenly."""
+    E, server = mods
+    srv = server.Server(workspace_bytes=256 << 20)
+    p = synth.make_vit(d=128, n_layers=1, n_heads=2, mlp=256, n_cls=10, seed=60 + T, device=DEV, img=img, patch=patch,
+                       std=0.1, perturb=0.2)
+    assert p["T"] == T
+    imgs = synth.make_images(3, seed=61 + T, device=DEV, img=img)
+    m = srv.add_model(p, max_batch=4)
+    _vit_check(srv, E, p, imgs, m, E.CAT_FS)
+    srv.close()
+
+
 def test_config2_vit_b16_batch_2(mods):
     """ViT-B/16 shape (197 tokens, d 768, 12 layers, 12 heads, MLP 3072, 1000 classes)."""
     E, server = mods
