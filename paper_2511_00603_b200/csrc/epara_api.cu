@@ -206,15 +206,17 @@ bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap,
   gemm_tc_config(rows_cap, N, K, g.epi, sm_count, &g.bn, &g.ksplit);
   if (max_rows <= GEMM_STREAM_MAX_ROWS && bl.gemm_impl == EPARA_GEMM_TCGEN05) {
     g.stream = 1; g.bn = 16; g.ksplit = 1;
+  } else if (bl.gemm_impl == EPARA_GEMM_TCGEN05 && gemm_tc_pair_eligible(rows_cap, N, K, g.epi, g.bn, g.ksplit)) {
+    g.stream = 2;                              // 256-row tiles on CTA pairs
   }
   if (g.ksplit > 1) {
     const size_t tiles_m = (size_t)((rows_cap + TC_BM - 1) / TC_BM), tiles_n = (size_t)((N + g.bn - 1) / g.bn);
     m->splitk_bytes = std::max(m->splitk_bytes, (size_t)g.ksplit * tiles_m * TC_BM * tiles_n * g.bn * 4);
     m->splitk_tiles = std::max(m->splitk_tiles, tiles_m * tiles_n);
   }
-  if (bl.c && !g.stream) {
+  if (bl.c && g.stream != 1) {
     if (!make_tmap(&g.tmA, A, rows_cap, K, lda, TC_BM)) return false;
-    if (!make_tmap(&g.tmW, W, N, K, K, g.bn)) return false;
+    if (!make_tmap(&g.tmW, W, N, K, K, g.stream == 2 ? g.bn / 2 : g.bn)) return false;   // a pair's CTA loads half of the W rows
     if (!make_tmap_c(&g.tmC, C, rows_cap, N, ldc, g.epi)) return false;
   }
   g.c_rows = (int)rows_cap;
@@ -757,10 +759,11 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
         if (a.cursor < a.m->ops.size() && a.m->ops[a.cursor].kind == kind) who.push_back(&a);
       if (who.empty()) continue;
       more = true;
-      // GEMM groups go out in up to two launches: tensor-core tiles (pass 0) and the weight-streaming
-      // kernel for groups that never exceed 16 rows (pass 1); encoder attention likewise: the tcgen05
-      // kernel (pass 0) and the mma.sync kernel for shapes it does not take (pass 1)
-      const int n_pass = (kind == EPARA_K_GEMM || kind == EPARA_K_ATTN_ENC) ? 2 : 1;
+      // GEMM groups go out in up to three launches: tensor-core tiles (pass 0), the weight-streaming
+      // kernel for groups that never exceed 16 rows (pass 1) and 256-row tiles on CTA pairs for the dense
+      // bf16-output groups (pass 2); encoder attention in two: the tcgen05 kernel (pass 0) and the
+      // mma.sync kernel for shapes it does not take (pass 1)
+      const int n_pass = kind == EPARA_K_GEMM ? 3 : (kind == EPARA_K_ATTN_ENC ? 2 : 1);
       for (int pass = 0; pass < n_pass; ++pass) {
       Launch L;
       memset(&L, 0, sizeof(L));
@@ -831,9 +834,13 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           }
           case EPARA_K_GEMM: {
             GemmGroup g = op.gemm;
-            if ((g.stream != 0) != (pass == 1)) break;         // the other pass takes it
+            if (g.stream != pass) break;                       // another pass takes it
             g.M = rows;
-            if (g.stream) {
+            if (g.stream == 2) {
+              g.tiles_m = (rows + 2 * TC_BM - 1) / (2 * TC_BM); g.tiles_n = (g.N + g.bn - 1) / g.bn;
+              g.tile_start = total;
+              total += g.tiles_m * g.tiles_n;
+            } else if (g.stream) {
               g.tiles_m = 1; g.tiles_n = gemm_stream_tiles(g.N);
               g.tile_start = total;
               total += g.tiles_n;
@@ -922,6 +929,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       case EPARA_K_NORM: launch_norm((const NormGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_GEMM:
         if (L.p2 == 1) err = launch_gemm_stream((const GemmGroup*)gp, L.n_groups, L.p0, L.p1, st);
+        else if (L.p2 == 2) err = launch_gemm_tc_pair((const GemmGroup*)gp, L.n_groups, L.p0, c->dev_status, c->sm_count, st);
         else if (simt) launch_gemm_simt((const GemmGroup*)gp, L.n_groups, L.p0, st);
         else err = launch_gemm_tc((const GemmGroup*)gp, L.n_groups, L.p0, L.p3, c->dev_status, c->sm_count, st);
         break;
@@ -1028,8 +1036,8 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
   if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool simt = impl == EPARA_GEMM_SIMT;
-  std::vector<GemmGroup> gs, gs_stream;      // tensor-core (or CUDA-core) groups; weight-streaming groups (M <= 16)
-  int total = 0, total_stream = 0, max_rows_stream = 0;
+  std::vector<GemmGroup> gs, gs_stream, gs_pair;   // tensor-core (or CUDA-core) groups; weight-streaming groups (M <= 16); CTA-pair groups
+  int total = 0, total_stream = 0, max_rows_stream = 0, total_pair = 0;
   size_t soff = epara_gemm_scratch_bytes(n);
   for (int i = 0; i < n; ++i) {
     const epara_gemm_problem& q = p[i];
@@ -1056,6 +1064,17 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
       continue;
     }
     if (!simt) gemm_tc_config(q.M, q.N, q.K, q.epilogue, 148, &g.bn, &g.ksplit);
+    if (!simt && gemm_tc_pair_eligible(q.M, q.N, q.K, q.epilogue, g.bn, g.ksplit)) {
+      g.stream = 2;
+      g.tiles_m = (q.M + 2 * TC_BM - 1) / (2 * TC_BM); g.tiles_n = (q.N + g.bn - 1) / g.bn;
+      g.tile_start = total_pair;
+      total_pair += g.tiles_m * g.tiles_n;
+      if (!make_tmap(&g.tmA, q.A, q.M, q.K, q.lda, TC_BM)) return EPARA_E_CUDA;
+      if (!make_tmap(&g.tmW, q.W, q.N, q.K, q.ldw, g.bn / 2)) return EPARA_E_CUDA;
+      if (!make_tmap_c(&g.tmC, q.C, q.M, q.N, q.ldc, q.epilogue)) return EPARA_E_CUDA;
+      gs_pair.push_back(g);
+      continue;
+    }
     const int tm = simt ? SIMT_TILE : TC_BM, tn = simt ? SIMT_TILE : g.bn;
     g.tiles_m = (q.M + tm - 1) / tm; g.tiles_n = (q.N + tn - 1) / tn;
     g.tile_start = total;
@@ -1079,6 +1098,7 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
   int* status = (int*)scratch;
   GemmGroup* dev_groups = (GemmGroup*)((unsigned char*)scratch + 256);
   GemmGroup* dev_stream = dev_groups + gs.size();
+  GemmGroup* dev_pair = dev_stream + gs_stream.size();
   if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) return EPARA_E_CUDA;
   // (a copy from pageable host memory is staged before cudaMemcpyAsync returns, so the vectors may go out of scope)
   if (!gs.empty() &&
@@ -1086,6 +1106,9 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
     return EPARA_E_CUDA;
   if (!gs_stream.empty() &&
       cudaMemcpyAsync(dev_stream, gs_stream.data(), gs_stream.size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return EPARA_E_CUDA;
+  if (!gs_pair.empty() &&
+      cudaMemcpyAsync(dev_pair, gs_pair.data(), gs_pair.size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return EPARA_E_CUDA;
   cudaError_t err = cudaSuccess;
   if (simt) {
@@ -1099,6 +1122,8 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
     err = launch_gemm_tc(dev_groups, (int)gs.size(), total, max_bn, status, sm, st);
     if (err == cudaSuccess)
       err = launch_gemm_stream(dev_stream, (int)gs_stream.size(), total_stream, max_rows_stream, st);
+    if (err == cudaSuccess)
+      err = launch_gemm_tc_pair(dev_pair, (int)gs_pair.size(), total_pair, status, sm, st);
   }
   return err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
 }

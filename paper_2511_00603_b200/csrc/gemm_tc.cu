@@ -210,7 +210,8 @@ __device__ __forceinline__ void splitk_reduce(const GView& g, const Item& it, in
 // happens at L2; the SM never reads C).  The hardware clips rows and columns outside the tensor.
 // The accumulator is handed back to the MMA warp as soon as this warp's last chunk has left TMEM.
 // MODE: 0 bf16 output, 1 SwiGLU, 2 fp32 residual.
-template <int MODE>
+// REMOTE: tempty is a shared::cluster address (the accumulator barrier of the pair's leader).
+template <int MODE, bool REMOTE = false>
 __device__ __forceinline__ void epi_direct(const GView& g, const Item& it, uint32_t taddr, unsigned char* wst, int quarter,
                                            int part, int lane, uint2 bias_reg, uint32_t tempty) {
   constexpr int CW = (MODE == 2) ? 16 : 32;                  // accumulator columns per chunk
@@ -222,7 +223,7 @@ __device__ __forceinline__ void epi_direct(const GView& g, const Item& it, uint3
   if (c_begin >= c_end) {                                    // nothing to do for this warp: release at once
     tc_fence_before();
     __syncwarp();
-    if (lane == 0) mbar_arrive(tempty);
+    if (lane == 0) { if (REMOTE) mbar_arrive_cluster(tempty); else mbar_arrive(tempty); }
     return;
   }
 #pragma unroll 1
@@ -238,7 +239,7 @@ __device__ __forceinline__ void epi_direct(const GView& g, const Item& it, uint3
     if (c + CW >= c_end) {                                   // that was this warp's last read of the accumulator
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty);
+      if (lane == 0) { if (REMOTE) mbar_arrive_cluster(tempty); else mbar_arrive(tempty); }
     }
     if (g.epi & EPI_BIAS) {
       // the bias values of this chunk sit in consecutive lanes of bias_reg (zero past N)
@@ -558,6 +559,182 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
   }
 }
 
+// ---------------------------------------------------------------------------------- tile pairs
+// The same pipeline for 256 x bn tiles worked by two CTAs of a cluster (the two SMs of a TPC): each CTA
+// loads its own 128 rows of A and bn / 2 rows of W per k-block (32 KB instead of 48: six ring stages, and
+// a third less traffic from L2 per flop, which is what bounds the one-CTA kernel on all 148 SMs), rank 0
+// issues one M = 256 MMA for both, the accumulator rows of a CTA's half live in its own TMEM and its own
+// epilogue warps write them out.  Barriers: every CTA's loads are counted on rank 0's full barrier;
+// the MMA completion is reported to the empty / accumulator-full barriers of both CTAs; the epilogue
+// warps of both report a drained accumulator to rank 0.  Only bf16 / GELU / SwiGLU outputs with
+// ksplit = 1 take this path; a work item is one 256-row tile, GemmGroup::tiles_m counts 256-row tiles.
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_STAGE_BYTES = RING_BYTES / PAIR_STAGES;     // 32 KB: A 16 KB + at most 128 rows of W
+
+template <class G>
+__device__ __forceinline__ Item decode_item_pair(const G& g, int local, int rank) {
+  Item it;
+  it.split = 0;
+  it.tile = local;
+  it.m0 = (local / g.tiles_n) * (2 * TC_BM) + rank * TC_BM;
+  it.n0 = (local % g.tiles_n) * g.bn;
+  it.kb0 = 0;
+  it.kb1 = (g.K + TC_BK - 1) / TC_BK;
+  return it;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(N_THREADS, 1)
+gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status) {
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  unsigned char* stage_out = base_ptr + RING_BYTES;
+  const uint32_t bars = base + RING_BYTES + STAGE_OUT_BYTES;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * MAX_STAGES + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + RING_BYTES + STAGE_OUT_BYTES + 8 * (2 * MAX_STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < PAIR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                        // the peer's barriers exist before anything is reported to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (one per CTA)
+    if (lane == 0) {
+      pdl_wait();
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const GemmGroup* g_prev = nullptr;
+      GroupCache gc;
+      gc.g = nullptr;
+      for (int item = pair; item < total_items && ok; item += n_pairs) {
+        group_cache(gc, groups, n_groups, item);
+        const GemmGroup* g = gc.g;
+        const Item it = decode_item_pair(*g, item - gc.start, rank);
+        if (g != g_prev) {
+          tensormap_acquire(&g->tmA);
+          tensormap_acquire(&g->tmW);
+          g_prev = g;
+        }
+        const int half = gc.bn >> 1;
+        const uint32_t bytes = 2u * (A_BYTES + (uint32_t)half * TC_BK * 2);     // both CTAs' boxes of a k-block
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 31); break; }
+          if (rank == 0) mbar_expect_tx(full_bar(stage), bytes);
+          const uint32_t sa = base + stage * PAIR_STAGE_BYTES;
+          const uint32_t fb = mapa_shared(full_bar(stage), 0);
+          tma_load_2d_pair(sa, &g->tmA, kb * TC_BK, it.m0, fb);
+          tma_load_2d_pair(sa + A_BYTES, &g->tmW, kb * TC_BK, it.n0 + rank * half, fb);
+          if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (rank 0 only)
+    if (lane == 0 && rank == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      GroupCache gc;
+      gc.g = nullptr;
+      for (int item = pair; item < total_items && ok; item += n_pairs) {
+        group_cache(gc, groups, n_groups, item);
+        const uint32_t idesc = make_idesc_pair(gc.bn);
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 32); break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
+        for (int kb = 0; kb < gc.kblocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; atomicExch(status, 33); break; }
+          tc_fence_after();
+          const uint32_t sa = base + stage * PAIR_STAGE_BYTES;
+          const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + A_BYTES);
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k)
+            mma_f16_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          mma_commit_pair(empty_bar(stage));
+          if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        mma_commit_pair(tfull_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..17 of both CTAs)
+    pdl_wait();
+    const int ew = warp - 2;
+    const int quarter = warp & 3;
+    const int part = ew >> 2;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    GView g;
+    int g_end = -1;
+    g.tile_start = 0;
+    for (int item = pair; item < total_items && ok; item += n_pairs) {
+      if (item >= g_end || item < g.tile_start) {
+        g = load_view(groups + find_group_tc(groups, n_groups, item));
+        g_end = g.tile_start + g.tiles_m * g.tiles_n;
+        if (lane == 0) tensormap_acquire(g.tmC);
+      }
+      const Item it = decode_item_pair(g, item - g.tile_start, rank);
+      uint2 bias_reg = make_uint2(0u, 0u);
+      if (g.epi & EPI_BIAS) {
+        const int nb = it.n0 + part * (g.bn >> 2) + lane * 4;
+        if (lane * 4 >= (g.bn >> 2)) {
+          // beyond this warp's columns
+        } else if (nb + 4 <= g.N) {
+          bias_reg = __ldg(reinterpret_cast<const uint2*>(g.bias + nb));
+        } else {
+          unsigned short e[4] = {0, 0, 0, 0};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) if (nb + j < g.N) e[j] = __bfloat16_as_ushort(g.bias[nb + j]);
+          bias_reg = make_uint2((uint32_t)e[0] | ((uint32_t)e[1] << 16), (uint32_t)e[2] | ((uint32_t)e[3] << 16));
+        }
+      }
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 34); break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * ACC_COLS);
+      unsigned char* wst = stage_out + ew * 2048;
+      const uint32_t te = mapa_shared(tempty_bar(acc), 0);
+      if (g.epi & EPI_SWIGLU) epi_direct<1, true>(g, it, taddr, wst, quarter, part, lane, bias_reg, te);
+      else epi_direct<0, true>(g, it, taddr, wst, quarter, part, lane, bias_reg, te);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (lane == 0) bulk_wait_done0();
+    if (!ok) *abort_flag = 1;
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                        // neither CTA leaves while the other may still read its operands or signal it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+  }
+}
+
 }  // namespace
 
 // Tile width and k-split of a GEMM whose row capacity is rows_cap (fixed when the model is placed,
@@ -602,6 +779,22 @@ cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_item
   const int stage_bytes = RING_BYTES / stages;
   return launch_pdl(gemm_tc_kernel, dim3(grid), dim3(N_THREADS), SMEM_BYTES, st, groups, n_groups, total_items, status,
                     stages, stage_bytes);
+}
+
+// A GEMM takes the tile-pair kernel when it is dense (more than 256 rows at capacity), its tiles are 256
+// wide and its output is bf16 (plain, GELU or SwiGLU); decided from the same placement-time quantities
+// as the tile width, never from the batch.
+bool gemm_tc_pair_eligible(long long rows_cap, int N, int K, int epi, int bn, int ksplit) {
+  return rows_cap > 256 && bn == 256 && ksplit == 1 && !(epi & EPI_RESID_F32) && N >= 256;
+}
+
+cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
+                                cudaStream_t st) {
+  if (n_groups == 0 || total_items == 0) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int pairs = total_items < sm_count / 2 ? total_items : sm_count / 2;
+  return launch_pdl(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(N_THREADS), SMEM_BYTES, st, groups, n_groups, total_items, status);
 }
 
 }  // namespace epara

@@ -23,6 +23,9 @@ constexpr int TC_BM = 128;
 constexpr int TC_BN_MAX = 256;
 constexpr int TC_BK = 64;
 void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int* bn, int* ksplit);
+bool gemm_tc_pair_eligible(long long rows_cap, int N, int K, int epi, int bn, int ksplit);
+cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
+                                cudaStream_t st);
 cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int max_bn, int* status,
                            int sm_count, cudaStream_t st);   // max_bn: widest tile among the groups
 
