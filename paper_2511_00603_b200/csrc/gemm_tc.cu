@@ -566,8 +566,8 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
 // issues one M = 256 MMA for both, the accumulator rows of a CTA's half live in its own TMEM and its own
 // epilogue warps write them out.  Barriers: every CTA's loads are counted on rank 0's full barrier;
 // the MMA completion is reported to the empty / accumulator-full barriers of both CTAs; the epilogue
-// warps of both report a drained accumulator to rank 0.  Only bf16 / GELU / SwiGLU outputs with
-// ksplit = 1 take this path; a work item is one 256-row tile, GemmGroup::tiles_m counts 256-row tiles.
+// warps of both report a drained accumulator to rank 0.  Only groups with ksplit = 1 and tiles of 192
+// or 256 columns take this path; a work item is one 256-row tile, GemmGroup::tiles_m counts 256-row tiles.
 constexpr int PAIR_STAGES = 6;
 constexpr int PAIR_STAGE_BYTES = RING_BYTES / PAIR_STAGES;     // 32 KB: A 16 KB + at most 128 rows of W
 
@@ -618,6 +618,21 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
+    if (lane != 0) {
+      // L2 prefetch of the fp32 residual tiles this CTA will add to (see the one-CTA kernel)
+      pdl_wait();
+      for (int item = pair; item < total_items; item += n_pairs) {
+        const GemmGroup& g = groups[find_group_tc(groups, n_groups, item)];
+        if (!(g.epi & EPI_RESID_F32)) continue;
+        const Item it = decode_item_pair(g, item - g.tile_start, rank);
+        const int ncols = min(g.bn, g.N - it.n0);
+        for (int r = lane - 1; r < TC_BM && it.m0 + r < g.M; r += 31) {
+          const float* rowp = reinterpret_cast<const float*>(g.C) + (size_t)(it.m0 + r) * g.ldc + it.n0;
+          for (int c = 0; c < ncols; c += 32)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + c));
+        }
+      }
+    }
     // ------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
       pdl_wait();
@@ -719,7 +734,8 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * ACC_COLS);
       unsigned char* wst = stage_out + ew * 2048;
       const uint32_t te = mapa_shared(tempty_bar(acc), 0);
-      if (g.epi & EPI_SWIGLU) epi_direct<1, true>(g, it, taddr, wst, quarter, part, lane, bias_reg, te);
+      if (g.epi & EPI_RESID_F32) epi_direct<2, true>(g, it, taddr, wst, quarter, part, lane, bias_reg, te);
+      else if (g.epi & EPI_SWIGLU) epi_direct<1, true>(g, it, taddr, wst, quarter, part, lane, bias_reg, te);
       else epi_direct<0, true>(g, it, taddr, wst, quarter, part, lane, bias_reg, te);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
@@ -781,11 +797,10 @@ cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_item
                     stages, stage_bytes);
 }
 
-// A GEMM takes the tile-pair kernel when it is dense (more than 256 rows at capacity), its tiles are 256
-// wide and its output is bf16 (plain, GELU or SwiGLU); decided from the same placement-time quantities
-// as the tile width, never from the batch.
+// A GEMM takes the tile-pair kernel when it is dense (more than 256 rows at capacity) and its tiles are
+// 192 or 256 wide; decided from the same placement-time quantities as the tile width, never from the batch.
 bool gemm_tc_pair_eligible(long long rows_cap, int N, int K, int epi, int bn, int ksplit) {
-  return rows_cap > 256 && bn == 256 && ksplit == 1 && !(epi & EPI_RESID_F32) && N >= 256;
+  return rows_cap > 256 && (bn == 256 || bn == 192) && ksplit == 1 && N >= bn;
 }
 
 cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
