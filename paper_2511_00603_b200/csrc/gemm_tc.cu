@@ -564,7 +564,8 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
 // loads its own 128 rows of A and bn / 2 rows of W per k-block (32 KB instead of 48: six ring stages, and
 // a third less traffic from L2 per flop, which is what bounds the one-CTA kernel on all 148 SMs), rank 0
 // issues one M = 256 MMA for both, the accumulator rows of a CTA's half live in its own TMEM and its own
-// epilogue warps write them out.  Barriers: every CTA's loads are counted on rank 0's full barrier;
+// epilogue warps write them out.  Warp 0 loads A, warp 18 loads W, warp 1 of rank 0 issues the MMAs, warps
+// 2..17 are the epilogue.  Barriers: every CTA's loads are counted on rank 0's full barrier;
 // the MMA completion is reported to the empty / accumulator-full barriers of both CTAs; the epilogue
 // warps of both report a drained accumulator to rank 0.  Only groups with ksplit = 1 and tiles of 192
 // or 256 columns take this path; a work item is one 256-row tile, GemmGroup::tiles_m counts 256-row tiles.
@@ -583,7 +584,10 @@ __device__ __forceinline__ Item decode_item_pair(const G& g, int local, int rank
   return it;
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(N_THREADS, 1)
+constexpr int PAIR_W_WARP = 2 + EPI_WARPS;                     // the warp after the epilogue warps loads W
+constexpr int PAIR_THREADS = N_THREADS + 32;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
 gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status) {
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -633,7 +637,9 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
         }
       }
     }
-    // ------------------------------------------------------------ TMA producer (one per CTA)
+    // ------------------------------------------------------------ TMA producer of A (one per CTA)
+    // One thread issues a TMA load in some 150 cycles; with both operands on one thread a k-block costs it
+    // more than the 512 cycles its MMAs take once tiles are short.  So the two operands have a thread each.
     if (lane == 0) {
       pdl_wait();
       int stage = 0;
@@ -646,20 +652,39 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
         group_cache(gc, groups, n_groups, item);
         const GemmGroup* g = gc.g;
         const Item it = decode_item_pair(*g, item - gc.start, rank);
-        if (g != g_prev) {
-          tensormap_acquire(&g->tmA);
-          tensormap_acquire(&g->tmW);
-          g_prev = g;
-        }
-        const int half = gc.bn >> 1;
-        const uint32_t bytes = 2u * (A_BYTES + (uint32_t)half * TC_BK * 2);     // both CTAs' boxes of a k-block
+        if (g != g_prev) { tensormap_acquire(&g->tmA); g_prev = g; }
+        const uint32_t bytes = 2u * (A_BYTES + (uint32_t)(gc.bn >> 1) * TC_BK * 2);   // both CTAs' boxes of a k-block
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 31); break; }
           if (rank == 0) mbar_expect_tx(full_bar(stage), bytes);
-          const uint32_t sa = base + stage * PAIR_STAGE_BYTES;
-          const uint32_t fb = mapa_shared(full_bar(stage), 0);
-          tma_load_2d_pair(sa, &g->tmA, kb * TC_BK, it.m0, fb);
-          tma_load_2d_pair(sa + A_BYTES, &g->tmW, kb * TC_BK, it.n0 + rank * half, fb);
+          tma_load_2d_pair(base + stage * PAIR_STAGE_BYTES, &g->tmA, kb * TC_BK, it.m0, mapa_shared(full_bar(stage), 0));
+          if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp == PAIR_W_WARP) {
+    // ------------------------------------------------------------ TMA producer of W (one per CTA)
+    // Weights are never written by a kernel, so this thread does not wait for the earlier kernels of the
+    // stream: the first stages' W boxes are on their way while those still run.  (Bytes that land before
+    // rank 0 has announced them leave the barrier's count negative for a while, which is allowed; the
+    // phase cannot complete before that thread's own arrival.)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const GemmGroup* g_prev = nullptr;
+      GroupCache gc;
+      gc.g = nullptr;
+      for (int item = pair; item < total_items && ok; item += n_pairs) {
+        group_cache(gc, groups, n_groups, item);
+        const GemmGroup* g = gc.g;
+        const Item it = decode_item_pair(*g, item - gc.start, rank);
+        if (g != g_prev) { tensormap_acquire(&g->tmW); g_prev = g; }
+        const int n_half = it.n0 + rank * (gc.bn >> 1);
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 35); break; }
+          tma_load_2d_pair(base + stage * PAIR_STAGE_BYTES + A_BYTES, &g->tmW, kb * TC_BK, n_half, mapa_shared(full_bar(stage), 0));
           if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -809,7 +834,7 @@ cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total
   cudaError_t e = cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int pairs = total_items < sm_count / 2 ? total_items : sm_count / 2;
-  return launch_pdl(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(N_THREADS), SMEM_BYTES, st, groups, n_groups, total_items, status);
+  return launch_pdl(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(PAIR_THREADS), SMEM_BYTES, st, groups, n_groups, total_items, status);
 }
 
 }  // namespace epara
