@@ -567,8 +567,8 @@ gemm_tc_kernel(const GemmGroup* __restrict__ groups, int n_groups, int total_ite
 // epilogue warps write them out.  Warp 0 loads A, warp 18 loads W, warp 1 of rank 0 issues the MMAs, warps
 // 2..17 are the epilogue.  Barriers: every CTA's loads are counted on rank 0's full barrier;
 // the MMA completion is reported to the empty / accumulator-full barriers of both CTAs; the epilogue
-// warps of both report a drained accumulator to rank 0.  Only groups with ksplit = 1 and tiles of 192
-// or 256 columns take this path; a work item is one 256-row tile, GemmGroup::tiles_m counts 256-row tiles.
+// warps of both report a drained accumulator to rank 0.  Only groups with ksplit = 1 take this path; a
+// work item is one 256-row tile, GemmGroup::tiles_m counts 256-row tiles.
 constexpr int PAIR_STAGES = 6;
 constexpr int PAIR_STAGE_BYTES = RING_BYTES / PAIR_STAGES;     // 32 KB: A 16 KB + at most 128 rows of W
 
@@ -822,10 +822,13 @@ cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_item
                     stages, stage_bytes);
 }
 
-// A GEMM takes the tile-pair kernel when it is dense (more than 256 rows at capacity) and its tiles are
-// 192 or 256 wide; decided from the same placement-time quantities as the tile width, never from the batch.
+// A GEMM takes the tile-pair kernel when it has more than one 128-row tile at capacity and is not split
+// along K; decided from the same placement-time quantities as the tile width, never from the batch.
+// Weight-streaming groups (129..256 rows) gain too: the pair reads every W box from HBM once, each CTA
+// half of it, where two one-CTA row tiles each load all of it.
 bool gemm_tc_pair_eligible(long long rows_cap, int N, int K, int epi, int bn, int ksplit) {
-  return rows_cap > 256 && (bn == 256 || bn == 192) && ksplit == 1 && N >= bn;
+  (void)N; (void)K; (void)epi;
+  return rows_cap > TC_BM && ksplit == 1 && (bn == 128 || bn == 192 || bn == 256);
 }
 
 cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,

@@ -113,10 +113,11 @@ def test_grouped_gemm_tile_pairs(E):
     """Dense bf16-output problems (more than 256 rows, 256-wide tiles) run as 256-row tiles on CTA pairs:
     ragged last pair (one CTA with no valid row), N tails inside the first and the second half of the W
     rows, SwiGLU, one k-block, a long K beyond the six-stage ring, more pairs than SM pairs, fp32-residual
-    outputs with 192- and 256-wide tiles."""
+    outputs with 192- and 256-wide tiles, 128-wide tiles of problems with 129 to 256 rows, N below one tile."""
     cases = [(1000, 1152, 384, ("bias",)), (513, 2048, 256, ("swiglu",)), (700, 264, 1536, ("bias", "gelu")),
              (257, 392, 64, ()), (20000, 512, 128, ("bias",)), (384, 256, 4096, ("gelu", "bias")),
-             (900, 384, 384, ("bias", "resid")), (515, 768, 1536, ("resid",)), (1300, 576, 192, ("bias", "resid"))]
+             (900, 384, 384, ("bias", "resid")), (515, 768, 1536, ("resid",)), (1300, 576, 192, ("bias", "resid")),
+             (200, 512, 512, ("bias", "gelu")), (256, 2048, 2048, ("resid",)), (129, 10, 512, ("bias",))]
     probs, refs = _run_gemm(E, E.GEMM_TCGEN05, cases, seed=9)
     for p, ref, case in zip(probs, refs, cases):
         assert_close(p["C"][:ref.shape[0], :ref.shape[1]], ref, what=f"pair gemm {case}")
