@@ -24,9 +24,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # DRAM bytes (read + write) per GEMM launch of the mixed step, from one ncu pass over the 130 GEMM launches
-# of a step (65 tensor-core + 65 weight-streaming: 16.15 + 8.83 GB and 2.08 + 0.0007 GB; see
+# of a step (65 tile-pair + 65 weight-streaming: 15.92 + 8.54 GB and 2.08 + 0.0008 GB; see
 # profiles/gemm_kernels_mixed_step_dram_traffic.md).  Set to None when the GEMM kernels change.
-GEMM_TRAFFIC_PER_LAUNCH_MIXED = (16145210880 + 8828690176 + 2083236096 + 654848) / 130
+GEMM_TRAFFIC_PER_LAUNCH_MIXED = (15922343680 + 8536922368 + 2083273216 + 750592) / 130
 
 PROFILE_EVERY = 5     # one step in five of the timed region carries per-launch events
 
@@ -424,7 +424,7 @@ def run_gpu(args):
     per_step = lambda v: v / args.steps
     if dom == "gemm":
         ach = per_step(flops) / (prof["gemm"][0] / 1e3) / 1e12
-        roof = {"kernel": "gemm_tc_kernel + gemm_stream_kernel (all GEMM launches of a step)", "bound": "tensor",
+        roof = {"kernel": "gemm_tc_pair_kernel + gemm_tc_kernel + gemm_stream_kernel (all GEMM launches of a step)", "bound": "tensor",
                 "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": ach / peaks["bf16_tflops_sustained"],
                 "traffic": None if stress else GEMM_TRAFFIC_PER_LAUNCH_MIXED,
