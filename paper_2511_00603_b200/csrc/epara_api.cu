@@ -813,8 +813,9 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
         switch (kind) {
           case EPARA_K_GATHER: {
             GatherGroup g = op.gather;
-            g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B; g.blocks = rows;
-            mx = std::max(mx, rows);
+            g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
+            g.blocks = g.kind == GATHER_PATCH ? (rows + GATHER_PATCH_ROWS - 1) / GATHER_PATCH_ROWS : rows;
+            mx = std::max(mx, g.blocks);
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }

@@ -5,6 +5,7 @@
 
 namespace epara {
 
+constexpr int GATHER_PATCH_ROWS = 8;   // patch rows per block of the patch gather
 void launch_gather(const GatherGroup* groups, int n_groups, int max_blocks, cudaStream_t st);
 int norm_blocks(int M, int d);
 void launch_norm(const NormGroup* groups, int n_groups, int max_blocks, cudaStream_t st);

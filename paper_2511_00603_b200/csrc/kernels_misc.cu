@@ -8,6 +8,8 @@
 namespace epara {
 
 // ------------------------------------------------------------------ gather
+// Row and embedding gathers take one block per row (a handful of rows per step); the patch gather takes
+// GATHER_PATCH_ROWS patch rows per block, so that a thread has several 16-byte loads in flight.
 __global__ void __launch_bounds__(128) gather_kernel(const GatherGroup* __restrict__ groups) {
   const GatherGroup g = groups[blockIdx.y];
   if ((int)blockIdx.x >= g.blocks) return;      // (descriptors are not written by kernels: no wait needed to leave)
@@ -31,16 +33,19 @@ __global__ void __launch_bounds__(128) gather_kernel(const GatherGroup* __restri
     }
   } else {  // GATHER_PATCH: row (b*np + i*gw + j), column c*p*p + u*p + v  <-  img[b][c][p*i+u][p*j+v]
     const int p = g.patch, gw = g.img / p, np = gw * gw;
-    const int b = blockIdx.x / np, pi = blockIdx.x % np;
-    const int i = pi / gw, j = pi % gw;
-    const bf16* img = reinterpret_cast<const bf16*>(g.reqs[b].input);
-    bf16* dst = reinterpret_cast<bf16*>(g.out) + (size_t)blockIdx.x * g.width;
-    const int vec_per_row = p / 8;
-    for (int e = threadIdx.x; e < g.width / 8; e += blockDim.x) {
+    const int vec_per_row = p / 8, vecs = g.width / 8;
+    const int row0 = blockIdx.x * GATHER_PATCH_ROWS;
+    const int nrows = min(GATHER_PATCH_ROWS, g.B * np - row0);
+#pragma unroll 4
+    for (int idx = threadIdx.x; idx < nrows * vecs; idx += blockDim.x) {
+      const int row = row0 + idx / vecs, e = idx % vecs;
+      const int b = row / np, pi = row % np;
+      const int i = pi / gw, j = pi % gw;
       const int cu = e / vec_per_row, v8 = e % vec_per_row;   // cu = c*p + u
       const int c = cu / p, u = cu % p;
+      const bf16* img = reinterpret_cast<const bf16*>(g.reqs[b].input);
       const bf16* s = img + ((size_t)c * g.img + (size_t)(p * i + u)) * g.img + p * j + v8 * 8;
-      reinterpret_cast<uint4*>(dst)[e] = *reinterpret_cast<const uint4*>(s);
+      reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(g.out) + (size_t)row * g.width)[e] = *reinterpret_cast<const uint4*>(s);
     }
   }
 }
@@ -266,28 +271,31 @@ void launch_rope_append(const RopeGroup* groups, int n_groups, int max_B, cudaSt
 }
 
 // ------------------------------------------------------------------ ViT token assembly
-__global__ void __launch_bounds__(128) assemble_kernel(const AssembleGroup* __restrict__ groups) {
+constexpr int ASSEMBLE_ROWS = 8;           // token rows per block
+__global__ void __launch_bounds__(256) assemble_kernel(const AssembleGroup* __restrict__ groups) {
   const AssembleGroup g = groups[blockIdx.y];
-  const int row = blockIdx.x;
-  if (row >= g.B * g.T) return;
+  const int row0 = blockIdx.x * ASSEMBLE_ROWS;
+  if (row0 >= g.B * g.T) return;
   pdl_launch_dependents();
   pdl_wait();
-  const int b = row / g.T, t = row % g.T;
-  const bf16* src = (t == 0) ? g.cls : g.E + ((size_t)b * (g.T - 1) + (t - 1)) * g.d;
-  const bf16* pos = g.pos + (size_t)t * g.d;
-  float* z = g.z + (size_t)row * g.d;
-  for (int i = threadIdx.x; i < g.d / 8; i += blockDim.x) {
+  const int nrows = min(ASSEMBLE_ROWS, g.B * g.T - row0), vecs = g.d / 8;
+#pragma unroll 2
+  for (int idx = threadIdx.x; idx < nrows * vecs; idx += blockDim.x) {
+    const int row = row0 + idx / vecs, i = idx % vecs;
+    const int b = row / g.T, t = row % g.T;
+    const bf16* src = (t == 0) ? g.cls : g.E + ((size_t)b * (g.T - 1) + (t - 1)) * g.d;
     float a[8], p[8];
     unpack8(reinterpret_cast<const uint4*>(src)[i], a);
-    unpack8(reinterpret_cast<const uint4*>(pos)[i], p);
-    reinterpret_cast<float4*>(z)[2 * i] = make_float4(a[0] + p[0], a[1] + p[1], a[2] + p[2], a[3] + p[3]);
-    reinterpret_cast<float4*>(z)[2 * i + 1] = make_float4(a[4] + p[4], a[5] + p[5], a[6] + p[6], a[7] + p[7]);
+    unpack8(reinterpret_cast<const uint4*>(g.pos + (size_t)t * g.d)[i], p);
+    float4* z = reinterpret_cast<float4*>(g.z + (size_t)row * g.d);
+    z[2 * i] = make_float4(a[0] + p[0], a[1] + p[1], a[2] + p[2], a[3] + p[3]);
+    z[2 * i + 1] = make_float4(a[4] + p[4], a[5] + p[5], a[6] + p[6], a[7] + p[7]);
   }
 }
 
 void launch_assemble(const AssembleGroup* groups, int n_groups, int max_rows, cudaStream_t st) {
   if (n_groups == 0 || max_rows == 0) return;
-  launch_pdl(assemble_kernel, dim3(max_rows, n_groups), dim3(128), 0, st, groups);
+  launch_pdl(assemble_kernel, dim3((max_rows + ASSEMBLE_ROWS - 1) / ASSEMBLE_ROWS, n_groups), dim3(256), 0, st, groups);
 }
 
 // ------------------------------------------------------------------ output scatter + argmax
