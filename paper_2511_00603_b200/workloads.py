@@ -80,21 +80,34 @@ class Instance:
         inp.out_logits = self.logits[out_slot].data_ptr()
         inp.out_argmax = self.argmax.data_ptr() + 4 * out_slot
 
-    def submit_all(self, ctx: "E.Context", alt: bool = False):
-        """Submits the whole pool; alt=True takes the inputs from the second input buffer (make_alt)."""
-        ctx.epara_submit_many(self.mid, self.category, self.inputs_alt if alt else self.inputs, self.n_req, self.tickets)
+    def submit_all(self, ctx: "E.Context", alt: bool = False, buf: int = -1):
+        """Submits the whole pool; buf = k takes the inputs from the k-th input buffer (make_bufs); alt=True
+        is buffer 1."""
+        k = buf if buf >= 0 else (1 if alt else 0)
+        ctx.epara_submit_many(self.mid, self.category, self.inputs_bufs[k] if k else self.inputs, self.n_req, self.tickets)
+
+    def make_bufs(self, n: int):
+        """n device input buffers (the first is self.x), each with its own request descriptors, so that the
+        inputs of later steps can be uploaded while earlier steps still read theirs."""
+        self.x_bufs, self.inputs_bufs = [self.x], [self.inputs]
+        for _ in range(1, n):
+            if self.x is None:
+                self.x_bufs.append(None)
+                self.inputs_bufs.append(self.inputs)
+                continue
+            xb = torch.empty_like(self.x)
+            ib = (E.Inputs * self.n_req)()
+            for i in range(self.n_req):
+                C.memmove(C.byref(ib[i]), C.byref(self.inputs[i]), C.sizeof(E.Inputs))
+                ib[i].input = xb[i].data_ptr()
+            self.x_bufs.append(xb)
+            self.inputs_bufs.append(ib)
+        self.x_alt = self.x_bufs[1] if n > 1 else None
+        self.inputs_alt = self.inputs_bufs[1] if n > 1 else self.inputs
 
     def make_alt(self):
-        """A second device input buffer with its own request descriptors, so that the inputs of the next
-        step can be uploaded while the current step still reads the first one."""
-        if self.x is None:
-            self.x_alt, self.inputs_alt = None, self.inputs
-            return
-        self.x_alt = torch.empty_like(self.x)
-        self.inputs_alt = (E.Inputs * self.n_req)()
-        for i in range(self.n_req):
-            C.memmove(C.byref(self.inputs_alt[i]), C.byref(self.inputs[i]), C.sizeof(E.Inputs))
-            self.inputs_alt[i].input = self.x_alt[i].data_ptr()
+        """Two input buffers (see make_bufs)."""
+        self.make_bufs(2)
 
     def input_bytes(self) -> int:
         return 0 if self.x is None else self.x.numel() * self.x.element_size()
