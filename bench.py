@@ -377,7 +377,9 @@ def run_gpu(args):
     copy_stream = torch.cuda.Stream(dev)
     ev_in = [torch.cuda.Event() for _ in range(E2E_BUFS)]
     ev_free = [None] * E2E_BUFS
+    ev_out = [None] * E2E_BUFS
     step_done = []
+    out_stream = torch.cuda.Stream(dev)
 
     def upload(buf):
         with torch.cuda.stream(copy_stream):
@@ -400,6 +402,8 @@ def run_gpu(args):
         if s_i >= 2:
             step_done[s_i - 2].synchronize()     # the host stays at most two steps ahead of the device
         stream.wait_event(ev_in[buf])
+        if ev_out[buf] is not None:
+            stream.wait_event(ev_out[buf])       # the results last written to this buffer set have been read back
         for i in insts:
             i.submit_all(srv.ctx, buf=buf)
             outstanding.append(list(i.tickets))
@@ -411,10 +415,17 @@ def run_gpu(args):
         # 150 MB of images in the host-to-device copy engine)
         if s_i + 1 < args.steps:
             upload((s_i + 1) % E2E_BUFS)
-        for i, hl, ha in h_out:
-            hl.copy_(i.logits, non_blocking=True)
-            ha.copy_(i.argmax, non_blocking=True)
-    stream.synchronize()                    # every step's results are on the host when the clock stops
+        # results of this step -> pinned host memory on a stream of its own, out of the step's own output
+        # buffers (one set per input buffer), so that the next step does not wait for the read-back
+        with torch.cuda.stream(out_stream):
+            out_stream.wait_event(ev_free[buf])
+            for i, hl, ha in h_out:
+                hl.copy_(i.logits_bufs[buf], non_blocking=True)
+                ha.copy_(i.argmax_bufs[buf], non_blocking=True)
+            ev_out[buf] = torch.cuda.Event()
+            ev_out[buf].record(out_stream)
+    stream.synchronize()
+    out_stream.synchronize()                # every step's results are on the host when the clock stops
     e2e_s = time.perf_counter() - t0
     drain()
     if world > 1:

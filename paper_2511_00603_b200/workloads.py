@@ -87,21 +87,26 @@ class Instance:
         ctx.epara_submit_many(self.mid, self.category, self.inputs_bufs[k] if k else self.inputs, self.n_req, self.tickets)
 
     def make_bufs(self, n: int):
-        """n device input buffers (the first is self.x), each with its own request descriptors, so that the
-        inputs of later steps can be uploaded while earlier steps still read theirs."""
+        """n buffer sets (set 0 is self.x / self.logits / self.argmax), each with its own request
+        descriptors: device inputs, so that the inputs of later steps can be uploaded while earlier steps
+        still read theirs, and device outputs, so that a step's results can be read back while the next
+        step runs."""
         self.x_bufs, self.inputs_bufs = [self.x], [self.inputs]
+        self.logits_bufs, self.argmax_bufs = [self.logits], [self.argmax]
         for _ in range(1, n):
-            if self.x is None:
-                self.x_bufs.append(None)
-                self.inputs_bufs.append(self.inputs)
-                continue
-            xb = torch.empty_like(self.x)
+            xb = None if self.x is None else torch.empty_like(self.x)
+            lb, ab = torch.zeros_like(self.logits), torch.full_like(self.argmax, -1)
             ib = (E.Inputs * self.n_req)()
             for i in range(self.n_req):
                 C.memmove(C.byref(ib[i]), C.byref(self.inputs[i]), C.sizeof(E.Inputs))
-                ib[i].input = xb[i].data_ptr()
+                if xb is not None:
+                    ib[i].input = xb[i].data_ptr()
+                ib[i].out_logits = lb[i].data_ptr()
+                ib[i].out_argmax = ab.data_ptr() + 4 * i
             self.x_bufs.append(xb)
             self.inputs_bufs.append(ib)
+            self.logits_bufs.append(lb)
+            self.argmax_bufs.append(ab)
         self.x_alt = self.x_bufs[1] if n > 1 else None
         self.inputs_alt = self.inputs_bufs[1] if n > 1 else self.inputs
 
