@@ -49,7 +49,8 @@ struct alignas(64) GemmGroup {
   int* counters;   // [tiles_m * tiles_n], zero between launches
   int c_rows;      // row extent of tmC (rows at and beyond it are never written)
   int stream;      // 1: at most 16 rows ever, runs in the weight-streaming kernel (16 W rows per block,
-                   // tiles_n = ceil(N / 16), no TMA maps); 0: tensor-core tiles
+                   // tiles_n = ceil(N / 16), no TMA maps); 0: one-CTA tensor-core tiles; 2: 256-row tiles on
+                   // CTA pairs (tiles_m counts 256-row tiles and tmW's box holds bn / 2 rows)
   int pad1, pad2;
 };
 

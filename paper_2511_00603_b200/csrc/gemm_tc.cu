@@ -19,6 +19,10 @@
 // The K reduction of an output element is the same sequence whatever else is in the launch.
 // Every mbarrier wait is bounded: when a wait runs out the kernel records a code in *status, all
 // roles leave their loops, TMEM is freed and the kernel returns.
+//
+// Two kernels share this pipeline and its epilogue: gemm_tc_kernel (one CTA per 128-row tile; groups of
+// 17 to 128 rows and the split-k groups) and gemm_tc_pair_kernel further down (two CTAs of a cluster per
+// 256-row tile, tcgen05 cta_group::2; every other group of more than 128 rows).
 #include "common.cuh"
 #include "kernels.h"
 #include "tcgen05.cuh"
