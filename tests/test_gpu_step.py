@@ -211,6 +211,39 @@ def test_config5_8b_layer_shapes_shallow_strict(mods):
     _decoder_case(E, server, p, B=3, lo=512, hi=8192, seed=41, n_check=2)
 
 
+def test_instance_buffer_sets_give_the_same_answers(mods):
+    """The end-to-end loop of the benchmark rotates buffer sets (device inputs, outputs and request
+    descriptors per set): a step fed from set 2 gives bit-identical results, in that set's own output
+    buffers, to a step fed from set 0, and leaves the other sets' outputs alone."""
+    E, server = mods
+    from paper_2511_00603_b200 import workloads as W
+    srv = server.Server(workspace_bytes=256 << 20)
+    pm = synth.make_mlp([256, 384, 72], seed=70, device=DEV, perturb=0.3, std=0.1)
+    pv = synth.make_vit(d=128, n_layers=1, n_heads=2, mlp=256, n_cls=10, seed=71, device=DEV, img=64, std=0.1)
+    insts = [W.Instance(srv, pm, E.CAT_FS, 9, seed=72), W.Instance(srv, pv, E.CAT_LS, 3, seed=73)]
+    stream = torch.cuda.current_stream().cuda_stream
+    for i in insts:
+        i.make_bufs(3)
+        i.submit_all(srv.ctx)
+    srv.ctx.epara_step(stream, 0)
+    torch.cuda.synchronize()
+    for i in insts:
+        for t in i.tickets:
+            assert srv.ctx.epara_collect(t)[0] == E.OK
+        assert (i.argmax >= 0).all() and (i.argmax_bufs[2] == -1).all()
+        i.x_bufs[2].copy_(i.x)
+        i.x.zero_()                                   # set 0's inputs are not what the next step may read
+        i.submit_all(srv.ctx, buf=2)
+    srv.ctx.epara_step(stream, 0)
+    torch.cuda.synchronize()
+    for i in insts:
+        for t in i.tickets:
+            assert srv.ctx.epara_collect(t)[0] == E.OK
+        assert torch.equal(i.logits_bufs[2], i.logits) and torch.equal(i.argmax_bufs[2], i.argmax)
+        assert (i.argmax_bufs[1] == -1).all()
+    srv.close()
+
+
 def test_mixed_bench_workload_sampled_parity(mods):
     """The benchmark's own configuration (8 co-resident instances, full batches, one step): sampled
     requests of every instance against the oracle, plus properties that hold for all of them."""
