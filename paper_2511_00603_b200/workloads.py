@@ -80,11 +80,10 @@ class Instance:
         inp.out_logits = self.logits[out_slot].data_ptr()
         inp.out_argmax = self.argmax.data_ptr() + 4 * out_slot
 
-    def submit_all(self, ctx: "E.Context", alt: bool = False, buf: int = -1):
-        """Submits the whole pool; buf = k takes the inputs from the k-th input buffer (make_bufs); alt=True
-        is buffer 1."""
-        k = buf if buf >= 0 else (1 if alt else 0)
-        ctx.epara_submit_many(self.mid, self.category, self.inputs_bufs[k] if k else self.inputs, self.n_req, self.tickets)
+    def submit_all(self, ctx: "E.Context", buf: int = 0):
+        """Submits the whole pool; buf = k takes inputs, outputs and descriptors from buffer set k (make_bufs)."""
+        ctx.epara_submit_many(self.mid, self.category, self.inputs_bufs[buf] if buf else self.inputs, self.n_req,
+                              self.tickets)
 
     def make_bufs(self, n: int):
         """n buffer sets (set 0 is self.x / self.logits / self.argmax), each with its own request
@@ -107,12 +106,6 @@ class Instance:
             self.inputs_bufs.append(ib)
             self.logits_bufs.append(lb)
             self.argmax_bufs.append(ab)
-        self.x_alt = self.x_bufs[1] if n > 1 else None
-        self.inputs_alt = self.inputs_bufs[1] if n > 1 else self.inputs
-
-    def make_alt(self):
-        """Two input buffers (see make_bufs)."""
-        self.make_bufs(2)
 
     def input_bytes(self) -> int:
         return 0 if self.x is None else self.x.numel() * self.x.element_size()
