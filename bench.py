@@ -23,10 +23,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) per GEMM launch of the mixed step, from one ncu pass over the 130 GEMM launches
-# of a step (65 tile-pair + 65 weight-streaming: 15.92 + 8.54 GB and 2.08 + 0.0008 GB; see
-# profiles/gemm_kernels_mixed_step_dram_traffic.md).  Set to None when the GEMM kernels change.
-GEMM_TRAFFIC_PER_LAUNCH_MIXED = (15922343680 + 8536922368 + 2083273216 + 750592) / 130
+# DRAM bytes (read + write) per tensor-core GEMM launch of the mixed step, from one ncu pass over the GEMM
+# launches of a step (65 tile-pair launches: 15.92 GB read + 8.54 GB written; the 65 weight-streaming
+# launches moved 2.08 GB).  Not measured by this run: the profile it comes from is named beside it in the
+# JSON line.  Set to None when the GEMM kernels change.
+GEMM_TC_TRAFFIC_PER_LAUNCH_MIXED = (15922343680 + 8536922368) / 65
+GEMM_TRAFFIC_SOURCE = "profiles/gemm_kernels_mixed_step_dram_traffic.md (one ncu pass, dram__bytes_read.sum + dram__bytes_write.sum)"
 
 E2E_BUFS = 4          # device input buffers per instance in the end-to-end loop
 PROFILE_EVERY = 5     # one step in five of the timed region carries per-launch events
@@ -149,43 +151,65 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------ CPU oracle leg
 class OracleSampler:
-    """Times the oracle, as it stands, on a bounded sample of the mixed workload: 8 MLP-A requests,
-    1 ViT-S image, 1 decoder request (1B shape, KV length 2112 = the mean of U[128,4096]).  The models
-    are generated once; every sample() draws fresh inputs and returns seconds per request per family."""
+    """Times the oracle, as it stands, on bounded samples of the mixed step.  Only the configuration numbers and
+    the seeded generators are imported: nothing here loads the CUDA library.  The models (MLP-A, ViT-S/16, 1B
+    decoder) are generated once.  The step's decoder requests have the KV lengths of the benchmark's own
+    seeded draw (4 + 256 requests, ~U[128, 4096]); decoder samples walk through them in the order shortest,
+    longest, then evenly spaced ranks, so that a run of 8 or more samples spans the whole range."""
 
     def __init__(self, seed: int = 3):
-        from paper_2511_00603_b200 import synth, workloads as W
-        self.synth, self.seed = synth, seed
+        from paper_2511_00603_b200 import configs, synth
+        self.synth, self.configs, self.seed = synth, configs, seed
         self.cores = os.cpu_count() or 1
-        self.mlp = synth.bits_view(synth.make_mlp(W.MLP_A, seed=seed))
-        self.vit = synth.bits_view(synth.make_vit(seed=seed + 2, **W.VIT_S))
-        self.dec = synth.bits_view(synth.make_decoder(seed=seed + 4, **W.DEC_1B))
-        self.n = 0
+        self.mlp = synth.bits_view(synth.make_mlp(configs.MLP_A, seed=seed))
+        self.vit = synth.bits_view(synth.make_vit(seed=seed + 2, **configs.VIT_S))
+        self.dec = synth.bits_view(synth.make_decoder(seed=seed + 4, **configs.DEC_1B))
+        lens = []
+        for k, n in ((6, configs.MIXED_LS_BATCH), (7, configs.MIXED_FS_BATCH)):      # the two decoder instances of the step
+            lens += list(synth.make_decode_batch(n, configs.MIXED_KV_LO, configs.MIXED_KV_HI, configs.DEC_1B["vocab"],
+                                                 seed * 1000 + k)[1])
+        self.lens = sorted(int(v) for v in lens)
+        n = len(self.lens)
+        ranks = [0, n - 1] + [round((j + 0.5) * n / 6) for j in range(6)]
+        self.len_cycle = [self.lens[min(n - 1, r)] for r in ranks]
+        self.n_mlp = self.n_vit = self.n_dec = 0
 
-    def sample(self):
+    def time_mlp(self, n: int) -> float:
         from oracle import epara_oracle as O
-        synth, s = self.synth, self.seed + 100 * self.n
-        self.n += 1
-        t = {}
-        x = synth.make_mlp_inputs(8, 512, seed=s + 1)
+        x = self.synth.make_mlp_inputs(n, self.configs.MLP_A[0], seed=self.seed + 1000 + self.n_mlp)
+        self.n_mlp += n
+        xb = [self.synth.to_bits(x[i]) for i in range(n)]
         t0 = time.perf_counter()
-        for i in range(8):
-            O.mlp_forward(synth.to_bits(x[i]), self.mlp["W"], self.mlp["b"])
-        t["mlp"] = (time.perf_counter() - t0) / 8
-        img = synth.to_bits(synth.make_images(1, seed=s + 3)[0])
-        t0 = time.perf_counter()
-        O.vit_forward(img, self.vit)
-        t["vit"] = time.perf_counter() - t0
-        toks, lens, tables, npages = synth.make_decode_batch(1, 2112, 2112, 32000, seed=s + 5)
-        pool = synth.to_bits(synth.make_kv_pool(16, npages, 8, 64, seed=s + 6))
-        t0 = time.perf_counter()
-        O.decoder_step(int(toks[0]), int(lens[0]), tables[0], lambda l, pg: pool[l, pg], self.dec)
-        t["decoder"] = time.perf_counter() - t0
-        return t
+        for i in range(n):
+            O.mlp_forward(xb[i], self.mlp["W"], self.mlp["b"])
+        return time.perf_counter() - t0
 
+    def time_vit(self, n: int) -> float:
+        from oracle import epara_oracle as O
+        imgs = self.synth.make_images(n, seed=self.seed + 2000 + self.n_vit)
+        self.n_vit += n
+        ib = [self.synth.to_bits(imgs[i]) for i in range(n)]
+        t0 = time.perf_counter()
+        for i in range(n):
+            O.vit_forward(ib[i], self.vit)
+        return time.perf_counter() - t0
 
-def mixed_counts(ls=4, fs=256):
-    return {"mlp": ls + 2 * fs, "vit": ls + 2 * fs, "decoder": ls + fs}
+    def time_decoder(self, n: int):
+        """n decoder requests at the next n lengths of the cycle; returns (seconds, the lengths)."""
+        from oracle import epara_oracle as O
+        cfg = self.configs.DEC_1B
+        total, used = 0.0, []
+        for _ in range(n):
+            L = self.len_cycle[self.n_dec % len(self.len_cycle)]
+            toks, lens, tables, npages = self.synth.make_decode_batch(1, L, L, cfg["vocab"], seed=self.seed + 3000 + self.n_dec)
+            pool = self.synth.to_bits(self.synth.make_kv_pool(cfg["n_layers"], npages, cfg["n_kv_heads"], cfg["head_dim"],
+                                                              seed=self.seed + 4000 + self.n_dec))
+            self.n_dec += 1
+            t0 = time.perf_counter()
+            O.decoder_step(int(toks[0]), L, tables[0], lambda l, pg: pool[l, pg], self.dec)
+            total += time.perf_counter() - t0
+            used.append(L)
+        return total, used
 
 
 def oracle_rps(t, counts):
@@ -194,28 +218,57 @@ def oracle_rps(t, counts):
 
 
 def run_reference(args):
+    """The oracle on the host cores.  Each step times a bounded sample of the mixed step -- 32 MLP-A requests,
+    1 ViT-S/16 image, 1 decoder request -- and the step's time is the per-family seconds per request times the
+    family's request count; the decoder samples walk over the step's own KV lengths (shortest and longest
+    first)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    counts = mixed_counts()
-    vals = []
     smp = OracleSampler()
-    cores = smp.cores
+    counts = smp.configs.mixed_counts()
+    acc = {"mlp": [0.0, 0], "vit": [0.0, 0], "decoder": [0.0, 0]}
+    dec_lens = []
     for i in range(args.warmup + args.steps):
-        t = smp.sample()
+        t_m, t_v = smp.time_mlp(32), smp.time_vit(1)
+        t_d, used = smp.time_decoder(1)
         if i >= args.warmup:
-            vals.append(oracle_rps(t, counts))
-    rps = sum(v[0] for v in vals) / len(vals)
-    step_s = sum(v[1] for v in vals) / len(vals)
-    sample = ("per step: 8 MLP-A + 1 ViT-S image + 1 decoder request (1B, KV 2112) timed, step time extrapolated "
-              "to the 1292-request mixed step by per-family counts")
+            for k, t, n in (("mlp", t_m, 32), ("vit", t_v, 1), ("decoder", t_d, 1)):
+                acc[k][0] += t
+                acc[k][1] += n
+            dec_lens += used
+    per_req = {k: acc[k][0] / max(acc[k][1], 1) for k in acc}
+    rps, step_s = oracle_rps(per_req, counts)
+    sample = (f"timed over {args.steps} steps: {acc['mlp'][1]} MLP-A requests, {acc['vit'][1]} ViT-S/16 images, "
+              f"{acc['decoder'][1]} 1B-decoder requests at KV lengths {dec_lens} (taken from the step's own lengths: shortest, "
+              f"longest, then evenly spaced ranks); a step's time = seconds per request of each family x the family's "
+              f"count in the {sum(counts.values())}-request mixed step ({counts}): extrapolated, the full step was never run")
     line = {"impl": "reference", "metric": METRIC, "value": rps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD},
-            "cpu_baseline": {"value": rps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": rps, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": sample,
+                             "seconds_per_request": per_req},
             "e2e": {"value": rps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
     return 0
+
+
+def cpu_baseline_leg():
+    """The oracle timed beside the GPU run: every MLP-A request of a step (516), 16 ViT-S/16 images and 8 decoder
+    requests (the step's shortest and longest KV length and six evenly spaced ranks)."""
+    smp = OracleSampler()
+    counts = smp.configs.mixed_counts()
+    t_m = smp.time_mlp(counts["mlp"])
+    t_v = smp.time_vit(16)
+    t_d, used = smp.time_decoder(8)
+    per_req = {"mlp": t_m / counts["mlp"], "vit": t_v / 16, "decoder": t_d / 8}
+    rps, step_s = oracle_rps(per_req, counts)
+    return {"value": rps, "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+            "sample": (f"timed: all {counts['mlp']} MLP-A requests of a step ({t_m:.2f} s), 16 of its {counts['vit']} ViT-S/16 "
+                       f"images ({t_v:.2f} s), 8 of its {counts['decoder']} decoder requests at KV lengths {used} ({t_d:.2f} s); "
+                       f"ViT and decoder families extrapolated by their counts to the {sum(counts.values())}-request step "
+                       f"({step_s:.0f} s)"),
+            "seconds_per_request": per_req}
 
 
 # ------------------------------------------------------------------------------ GPU leg
@@ -490,18 +543,30 @@ def run_gpu(args):
         return 0
 
     # ---- roofline of the dominant kernel ----
-    dom = max(prof, key=lambda k: prof[k][0])
+    # The GEMM launches of a step are two kinds of work: tensor-core launches (tile pairs and one-CTA tiles),
+    # judged against the tensor peak, and weight-streaming launches (groups of at most 16 rows), judged against
+    # HBM.  The timed region is a fraction of a second; which bf16 peak applies depends on the clock it ran at,
+    # so both fractions are given beside the sampled clock: the burst peak when the median SM clock stayed
+    # within 10 % of the maximum, the sustained (power-capped) peak otherwise.
     per_step = lambda v: v / args.steps
+    tc_ms, st_ms = prof["gemm"][0], prof["gemm_stream"][0]
+    sflops = sum(i.stream_gemm_flops for i in infos)
+    swbytes = sum(i.stream_weight_bytes for i in infos)
+    near_max = bool(clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] >= 0.9 * clocks["sm_max_mhz"])
+    dom = max(("gemm", "attn_dec", "attn_enc", "norm"), key=lambda k: prof[k][0])
     if dom == "gemm":
-        ach = per_step(flops) / (prof["gemm"][0] / 1e3) / 1e12
-        roof = {"kernel": "gemm_tc_pair_kernel + gemm_tc_kernel + gemm_stream_kernel (all GEMM launches of a step)", "bound": "tensor",
-                "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops_sustained"],
-                "traffic": None if stress else GEMM_TRAFFIC_PER_LAUNCH_MIXED,
-                "peak_source": peaks["source"] + " (sustained)"}
+        ach = per_step(flops - sflops) / (tc_ms / 1e3) / 1e12
+        peak = peaks["bf16_tflops"] if near_max else peaks["bf16_tflops_sustained"]
+        roof = {"kernel": "gemm_tc_pair_kernel + gemm_tc_kernel (the tensor-core GEMM launches of a step)", "bound": "tensor",
+                "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                "frac_of_burst_peak": ach / peaks["bf16_tflops"], "frac_of_sustained_peak": ach / peaks["bf16_tflops_sustained"],
+                "sm_mhz_median": clocks.get("sm_mhz"), "launches_per_step": prof["gemm"][1], "ms_per_step": tc_ms,
+                "traffic": None if (stress or GEMM_TC_TRAFFIC_PER_LAUNCH_MIXED is None) else GEMM_TC_TRAFFIC_PER_LAUNCH_MIXED,
+                "traffic_source": None if stress else GEMM_TRAFFIC_SOURCE,
+                "peak_source": peaks["source"] + (" (burst: median SM clock within 10 % of max)" if near_max else " (sustained)")}
     elif dom == "attn_dec":
         ach = per_step(kvbytes) / (prof["attn_dec"][0] / 1e3) / 1e9
-        roof = {"kernel": "attn_decode_kernel (all launches of a step)", "bound": "hbm", "achieved": ach,
+        roof = {"kernel": "attn_decode_mma_kernel (all launches of a step)", "bound": "hbm", "achieved": ach,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
                 "peak_source": peaks["source"]}
     else:
@@ -509,10 +574,15 @@ def run_gpu(args):
                 "frac": None, "traffic": None, "peak_source": peaks["source"]}
     kernels = {k: {"ms_per_step": prof[k][0], "launches_per_step": prof[k][1]} for k in prof if prof[k][1]}
     if prof["gemm"][1]:
-        kernels["gemm"]["tflops"] = per_step(flops) / (prof["gemm"][0] / 1e3) / 1e12
-        kernels["gemm"]["weight_gbs"] = per_step(wbytes) / (prof["gemm"][0] / 1e3) / 1e9
+        kernels["gemm"]["tflops"] = per_step(flops - sflops) / (tc_ms / 1e3) / 1e12
+        kernels["gemm"]["frac_tensor_burst"] = kernels["gemm"]["tflops"] / peaks["bf16_tflops"]
+        kernels["gemm"]["frac_tensor_sustained"] = kernels["gemm"]["tflops"] / peaks["bf16_tflops_sustained"]
+    if prof["gemm_stream"][1]:
+        kernels["gemm_stream"]["weight_gbs"] = per_step(swbytes) / (st_ms / 1e3) / 1e9
+        kernels["gemm_stream"]["frac_hbm"] = kernels["gemm_stream"]["weight_gbs"] / peaks["hbm_gbs"]
     if prof["attn_dec"][1]:
         kernels["attn_dec"]["kv_gbs"] = per_step(kvbytes) / (prof["attn_dec"][0] / 1e3) / 1e9
+        kernels["attn_dec"]["frac_hbm"] = kernels["attn_dec"]["kv_gbs"] / peaks["hbm_gbs"]
 
     poisson = None
     if not args.no_poisson and not stress:
@@ -520,14 +590,18 @@ def run_gpu(args):
 
     cpu = None
     if not args.no_cpu_baseline and not stress:
-        smp = OracleSampler()
-        t, cores = smp.sample(), smp.cores
-        rps, step_s = oracle_rps(t, mixed_counts())
-        cpu = {"value": rps, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "8 MLP-A + 1 ViT-S image + 1 decoder request (1B, KV 2112) timed once each; step time "
-                         "extrapolated to the 1292-request mixed step by per-family counts",
-               "seconds_per_request": t}
+        cpu = cpu_baseline_leg()
     srv.close()
+    del insts, srv
+    torch.cuda.empty_cache()
+    # whole steps of the single-model configurations, measured after (outside) the timed region
+    cfg_steps = None
+    if not args.no_config_steps and not stress:
+        from paper_2511_00603_b200 import synth
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        cfg_steps = {"vit_b16": [measure_vit_step(torch, E, server, W, synth, peaks, W.VIT_B, b, 10, flush) for b in (1, 8, 64)],
+                     "decoder_1b": [measure_decode_step(torch, E, server, W, synth, peaks, W.DEC_1B, b, 128, 4096, 10, flush)
+                                    for b in (1, 32, 128)]}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
@@ -537,11 +611,61 @@ def run_gpu(args):
             "clocks": clocks, "gpu_launches": launches,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "ms_per_step_unprofiled": ms_plain,
-            "ls_latency": poisson}
+            "ls_latency": poisson, "config_steps": cfg_steps}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+# ------------------------------------------------------------------------------ whole steps of one model
+def _timed_steps(torch, srv, inst, steps, flush):
+    """Median device time of `steps` steps of one instance (L2 flushed before each), then one more step
+    bracketed per launch for the per-kind split."""
+    stream = torch.cuda.current_stream(srv.device)
+    times, info = [], None
+    for i in range(steps + 4):
+        if i == steps + 3:
+            srv.ctx.epara_set_profile(True)
+        flush.zero_()
+        inst.submit_all(srv.ctx)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        info = srv.ctx.epara_step(stream.cuda_stream, 0)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        for t in inst.tickets:
+            srv.ctx.epara_collect(t)
+        if 3 <= i < steps + 3:
+            times.append(e0.elapsed_time(e1))
+    prof = srv.ctx.epara_step_profile()
+    return sorted(times)[len(times) // 2], info, {k: round(v[0], 4) for k, v in prof.items() if v[1]}
+
+
+def measure_vit_step(torch, E, server, W, synth, peaks, cfgm, B, steps, flush):
+    """Whole steps of one ViT at batch B (configs[1]: ViT-B/16 at batch 1 / 8 / 64, each its own step)."""
+    srv = server.Server(device=torch.cuda.current_device(), workspace_bytes=2 << 30)
+    inst = W.Instance(srv, synth.make_vit(seed=1, device=srv.device, **cfgm), E.CAT_FS, B, seed=11)
+    ms, info, kinds = _timed_steps(torch, srv, inst, steps, flush)
+    d, L, T = cfgm["d"], cfgm["n_layers"], 197
+    fl = info.gemm_flops + 4.0 * T * T * d * L * B
+    srv.close()
+    return {"kernel": "vit step", "d": d, "B": B, "ms": ms, "launches": info.launches, "images_per_s": B / (ms / 1e3),
+            "tflops_step": fl / (ms / 1e3) / 1e12, "frac_tensor_burst": fl / (ms / 1e3) / 1e12 / peaks["bf16_tflops"],
+            "frac_tensor_sustained": fl / (ms / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "weight_gbs": info.weight_bytes / (ms / 1e3) / 1e9, "per_kind_ms": kinds}
+
+
+def measure_decode_step(torch, E, server, W, synth, peaks, cfgm, B, lo, hi, steps, flush):
+    """Whole decode steps of one decoder at batch B (configs[2]; the decoder of configs[4]) through the step API."""
+    srv = server.Server(device=torch.cuda.current_device(), workspace_bytes=2 << 30)
+    inst = W.Instance(srv, synth.make_decoder(seed=2, device=srv.device, **cfgm), E.CAT_FS, B, seed=21, kv_lo=lo, kv_hi=hi)
+    ms, info, kinds = _timed_steps(torch, srv, inst, steps, flush)
+    byt = info.weight_bytes + info.kv_bytes
+    srv.close()
+    return {"kernel": "decode step", "d": cfgm["d"], "B": B, "ms": ms, "launches": info.launches,
+            "weight_gb": info.weight_bytes / 1e9, "kv_gb": info.kv_bytes / 1e9, "hbm_gbs": byt / (ms / 1e3) / 1e9,
+            "frac_hbm": byt / (ms / 1e3) / 1e9 / peaks["hbm_gbs"], "tokens_per_s": B / (ms / 1e3), "per_kind_ms": kinds}
 
 
 # ------------------------------------------------------------------------------ single-kernel timings
@@ -627,70 +751,14 @@ def run_micro(args):
         print(json.dumps({"kernel": "attn_decode+combine", "B": B, "Hq": Hq, "Hkv": Hkv, "hd": hd, "tokens": int(lens.sum()),
                           "ms": ms, "kv_gbs": kvb / (ms / 1e3) / 1e9, "frac_hbm": kvb / (ms / 1e3) / 1e9 / peaks["hbm_gbs"]}))
     elif args.micro == "vit_step":
-        # whole steps of one ViT (configs[1]: ViT-B/16 at batch 1 / 8 / 64, each its own frequency-sensitive step)
         from paper_2511_00603_b200 import server, workloads as W
-        cfgm = W.VIT_S if args.case == "vit_s" else W.VIT_B
-        B = args.m or 64
-        srv = server.Server(device=0, workspace_bytes=2 << 30)
-        inst = W.Instance(srv, synth.make_vit(seed=1, device=dev, **cfgm), E.CAT_FS, B, seed=11)
-        times = []
-        for i in range(args.steps + 4):
-            if i == args.steps + 3:
-                srv.ctx.epara_set_profile(True)
-            flush.zero_()
-            inst.submit_all(srv.ctx)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            info = srv.ctx.epara_step(stream.cuda_stream, 0)
-            e1.record(stream)
-            torch.cuda.synchronize()
-            for t in inst.tickets:
-                srv.ctx.epara_collect(t)
-            if 3 <= i < args.steps + 3:
-                times.append(e0.elapsed_time(e1))
-        prof = srv.ctx.epara_step_profile()
-        ms = sorted(times)[len(times) // 2]
-        d, L, T, F = cfgm["d"], cfgm["n_layers"], 197, cfgm["mlp"]
-        attn_flops = 4.0 * T * T * d * L * B
-        print(json.dumps({"kernel": "vit step", "case": args.case or "vit_b", "B": B, "ms": ms, "launches": info.launches,
-                          "images_per_s": B / (ms / 1e3), "gemm_tflop": info.gemm_flops / 1e12,
-                          "tflops_step": (info.gemm_flops + attn_flops) / (ms / 1e3) / 1e12,
-                          "frac_tensor_sustained": (info.gemm_flops + attn_flops) / (ms / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
-                          "per_kind_ms": {k: round(v[0], 4) for k, v in prof.items() if v[1]}}))
-        srv.close()
+        print(json.dumps(measure_vit_step(torch, E, server, W, synth, peaks, W.VIT_S if args.case == "vit_s" else W.VIT_B,
+                                          args.m or 64, args.steps, flush)))
     elif args.micro == "decode_step":
-        # whole decode steps of one decoder (configs[2] / the decoder of configs[4]) through the step API
         from paper_2511_00603_b200 import server, workloads as W
-        cfgm = W.DEC_8B if args.case == "dec_8b" else W.DEC_1B
-        hi = 8192 if args.case == "dec_8b" else 4096
-        lo = 512 if args.case == "dec_8b" else 128
-        B = args.m or 128
-        srv = server.Server(device=0, workspace_bytes=2 << 30)
-        inst = W.Instance(srv, synth.make_decoder(seed=2, device=dev, **cfgm), E.CAT_FS, B, seed=21, kv_lo=lo, kv_hi=hi)
-        times = []
-        for i in range(args.steps + 4):
-            if i == args.steps + 3:
-                srv.ctx.epara_set_profile(True)      # one more step, bracketed per launch, for the per-kind split
-            flush.zero_()
-            inst.submit_all(srv.ctx)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            info = srv.ctx.epara_step(stream.cuda_stream, 0)
-            e1.record(stream)
-            torch.cuda.synchronize()
-            for t in inst.tickets:
-                srv.ctx.epara_collect(t)
-            if 3 <= i < args.steps + 3:
-                times.append(e0.elapsed_time(e1))
-        prof = srv.ctx.epara_step_profile()
-        ms = sorted(times)[len(times) // 2]
-        byt = info.weight_bytes + info.kv_bytes
-        print(json.dumps({"kernel": "decode step", "case": args.case, "B": B, "ms": ms, "launches": info.launches,
-                          "weight_gb": info.weight_bytes / 1e9, "kv_gb": info.kv_bytes / 1e9,
-                          "hbm_gbs": byt / (ms / 1e3) / 1e9, "frac_hbm": byt / (ms / 1e3) / 1e9 / peaks["hbm_gbs"],
-                          "tokens_per_s": B / (ms / 1e3),
-                          "per_kind_ms": {k: round(v[0], 4) for k, v in prof.items() if v[1]}}))
-        srv.close()
+        big = args.case == "dec_8b"
+        print(json.dumps(measure_decode_step(torch, E, server, W, synth, peaks, W.DEC_8B if big else W.DEC_1B, args.m or 128,
+                                             512 if big else 128, 8192 if big else 4096, args.steps, flush)))
     return 0
 
 
@@ -710,6 +778,8 @@ def main():
                          "the GEMM launches do not depend on it)")
     ap.add_argument("--no-poisson", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-config-steps", action="store_true",
+                    help="skip the whole-step timings of ViT-B/16 (batch 1/8/64) and the 1B decoder (batch 1/32/128)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -102,6 +102,10 @@ typedef struct {
   long long kv_pages;
   int max_kv_len;               /* decoder: longest cached length a request may have */
   int max_batch;                /* rows reserved in the workspace (0 -> cap_ls + cap_fs) */
+  void* trace;                  /* device, decoder only, may be NULL: when given, every step copies the model's
+                                   residual stream into it after the embedding and after each layer, fp32
+                                   [n_layers + 1][max_batch][d] (row = the request's place in its batch).  For
+                                   checking the layers one by one; costs n_layers + 1 small copies per step. */
 } epara_model_desc;
 
 /* One request.  Unused fields are ignored for the model's kind. */
@@ -128,22 +132,30 @@ typedef struct {
   double gemm_flops;        /* 2 M N K over all GEMM groups */
   double weight_bytes;      /* bytes of weight matrices the step streams */
   double kv_bytes;          /* bytes of cached K/V the step reads */
-  int device_error;         /* filled by epara_collect when a kernel reported a bounded-wait failure */
+  double stream_gemm_flops;   /* the part of gemm_flops in weight-streaming launches (groups of at most 16 rows) */
+  double stream_weight_bytes; /* the part of weight_bytes in those launches */
 } epara_step_info;
 
 typedef struct {
-  int status;               /* EPARA_OK, EPARA_E_TIMEOUT (dropped), EPARA_E_DEVICE */
+  int status;               /* EPARA_OK, EPARA_E_TIMEOUT (dropped), EPARA_E_DEVICE, EPARA_E_CUDA, EPARA_E_RESOURCE */
   uint64_t step_id;
   void* logits;             /* the request's out_logits */
   int n_out;
   int32_t* argmax;
+  int device_error;         /* with EPARA_E_DEVICE: the code a kernel of the step left in the step's status word.
+                               1..49: a bounded wait ran out (which role gave up); 101: a block table named a page
+                               outside the model's kv_pages at the append; 102: the same at an attention read.
+                               The accesses behind 101 / 102 are skipped, never performed. */
 } epara_output;
 
 /* Kinds of kernels a step launches (index into epara_step_profile arrays). */
 enum {
   EPARA_K_GATHER = 0, EPARA_K_NORM = 1, EPARA_K_GEMM = 2, EPARA_K_ROPE = 3, EPARA_K_ATTN_DEC = 4,
   EPARA_K_ATTN_COMBINE = 5, EPARA_K_ATTN_ENC = 6, EPARA_K_ASSEMBLE = 7, EPARA_K_OUTPUT = 8,
-  EPARA_K_COUNT = 9
+  EPARA_K_GEMM_STREAM = 9,  /* the weight-streaming GEMM launches (groups of at most 16 rows); EPARA_K_GEMM holds
+                               the tensor-core launches */
+  EPARA_K_TRACE = 10,       /* copies into epara_model_desc.trace */
+  EPARA_K_COUNT = 11
 };
 
 /* Creates a context on cfg->device.  Returns INVALID (null/unaligned workspace), CUDA. */
@@ -174,9 +186,14 @@ int epara_submit_many(epara_ctx*, int model_id, int category, const epara_inputs
  * now_ns < 0 uses the host's monotonic clock.  info may be NULL. */
 int epara_step(epara_ctx*, void* cuda_stream, long long now_ns, epara_step_info* info);
 
-/* PENDING until the step that took the ticket has finished on the device (never blocks);
- * then OK with out filled, TIMEOUT if the request was dropped, DEVICE on a device error.
- * INVALID for an unknown (or already collected) ticket.  A ticket still queued is PENDING. */
+/* PENDING until the step that took the ticket has finished on the device (never blocks); then the
+ * request's final answer, also in out->status: OK with out filled; TIMEOUT if the request was dropped at
+ * admission; DEVICE when a kernel of its step reported an error (out->device_error has the code; every
+ * request of that step answers DEVICE, and the step's outputs must not be used); CUDA or RESOURCE when
+ * its step failed on the host after admission (a failed copy or launch, descriptors that did not fit):
+ * such requests are not re-queued.  Every step has a status word of its own, so a device error marks one
+ * step only.  INVALID for an unknown (or already collected) ticket.  A ticket still queued is PENDING.
+ * An answer stays available until it is collected, however many steps run in between. */
 int epara_collect(epara_ctx*, uint64_t ticket, epara_output* out);
 
 /* With cfg.profile = 1: per kernel kind, total milliseconds and launch count of the most
@@ -185,6 +202,9 @@ int epara_step_profile(epara_ctx*, float* ms_per_kind, int* launches_per_kind);
 
 /* Switches the per-launch event bracketing of epara_config.profile on (1) or off (0). */
 int epara_set_profile(epara_ctx*, int on);
+/* Most launches a profiled step may have (default 4096); a profiled step with more answers RESOURCE and
+ * runs nothing, its requests answer RESOURCE at collect. */
+int epara_set_max_profile_launches(epara_ctx*, int n);
 
 int epara_destroy(epara_ctx*);
 const char* epara_strerror(int status);
@@ -222,22 +242,26 @@ enum { EPARA_EPI_BIAS = 1, EPARA_EPI_GELU = 2, EPARA_EPI_SWIGLU = 4, EPARA_EPI_R
 
 /* C_g = epilogue(A_g W_g^T + bias_g) for every problem in one grouped launch.  RESID_F32:
  * C is fp32 and is updated in place, C += A W^T + bias.  `problems` is host memory;
- * `scratch` is device memory, 256-byte aligned, of at least epara_gemm_scratch_bytes_for(problems, n)
+ * `scratch` is device memory, 256-byte aligned, of at least epara_gemm_scratch_bytes_for(device, problems, n)
  * bytes (descriptors, plus fp32 partials for small-M problems that are split along K);
  * epara_gemm_scratch_bytes(n) suffices for EPARA_GEMM_SIMT. */
 int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm_problem* problems, int n,
                        void* scratch, size_t scratch_bytes);
 size_t epara_gemm_scratch_bytes(int n_problems);
-size_t epara_gemm_scratch_bytes_for(const epara_gemm_problem* problems, int n);
+size_t epara_gemm_scratch_bytes_for(int device, const epara_gemm_problem* problems, int n);
 
 /* Split-KV paged decode attention with GQA (one layer).  q: bf16 [B, q_stride] (head h at
- * column h*hd); kv_layer: bf16 [pages][2][Hkv][16][hd]; kv_lens int32 [B] = tokens to attend
- * (cached + appended); tables: int32 [B, table_stride]; out bf16 [B, Hq*hd];
- * scratch: at least epara_decode_attention_scratch_bytes(B, Hq, hd, max_len) bytes (request table,
- * fp32 chunk partials, chunk counters; the call clears the counters itself). */
+ * column h*hd); kv_layer: bf16 [kv_pages][2][Hkv][16][hd]; kv_lens int32 [B] = tokens to attend
+ * (cached + appended; values outside [0, max_len] are clamped, a request of length 0 leaves its output
+ * row unwritten); tables: int32 [B, table_stride]; out bf16 [B, Hq*hd];
+ * scratch: at least epara_decode_attention_scratch_bytes(B, Hq, hd, max_len) bytes (descriptor, request
+ * table, fp32 chunk partials, chunk counters; the call clears what must start at zero itself).
+ * A page id outside [0, kv_pages) is never dereferenced: the page is read as absent and the int32 at byte
+ * EPARA_DECODE_STATUS_OFFSET of `scratch` is set to 102 (it is 0 after a clean call). */
+#define EPARA_DECODE_STATUS_OFFSET 192
 int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
-                           const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out,
-                           int B, int Hq, int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes);
+                           long long kv_pages, const int32_t* kv_lens, const int32_t* tables, int table_stride,
+                           void* out, int B, int Hq, int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes);
 size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len);
 
 /* Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart
@@ -261,13 +285,25 @@ size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len);
  * it; make that first call outside any stream capture.  All calls on a device share the one array,
  * which keeps whatever the previous call left in it: the request table and the partials are written
  * before they are read, and the per-(request, kv head) chunk counters, the one part that must start
- * at zero, are cleared on the stream by every call.  Two calls whose kernels may overlap on the GPU
- * -- different streams without an ordering between them -- race on that array; order them. */
+ * at zero, are cleared on the stream by every call (a small set-up kernel, which also writes the call's
+ * descriptor from its own arguments, so no host buffer has to outlive the call).  Two calls whose kernels
+ * may overlap on the GPU -- different streams without an ordering between them -- race on that array;
+ * order them.  epara_decode_attention_static_status copies the last call's status word back (it waits
+ * for the device): OK and *code = 0 after a clean call, DEVICE and *code = 102 when a block table named
+ * a page outside [0, kv_pages). */
 #define EPARA_STATIC_SCRATCH_BYTES (8u << 20)
 int epara_decode_attention_static(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
-                                  const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out,
-                                  int B, int Hq, int Hkv, int hd, int max_len);
+                                  long long kv_pages, const int32_t* kv_lens, const int32_t* tables, int table_stride,
+                                  void* out, int B, int Hq, int Hkv, int hd, int max_len);
+int epara_decode_attention_static_status(int device, int* code);
 size_t epara_static_scratch_bytes(void);
+
+/* Self-test of the bounded waits (the paper has no counterpart; it exists so that the give-up path of the
+ * kernels' waits can be run without making a real kernel misbehave).  Launches one thread that waits, for
+ * at most limit_ns (<= 1 s), on a barrier nothing ever arrives at, then synchronises the stream.  Expected
+ * answer: EPARA_E_DEVICE with *code = 90 (the wait ran out and the kernel returned by itself).
+ * status_dev: device int32 used as the status word; code: host. */
+int epara_selftest_bounded_wait(int device, void* cuda_stream, unsigned long long limit_ns, int* status_dev, int* code);
 
 #ifdef __cplusplus
 }

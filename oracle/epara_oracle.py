@@ -206,6 +206,48 @@ def gather_kv(fetch_page: Callable[[int, int], np.ndarray], layer: int, table: n
     return K, V
 
 
+def decoder_layer(x: np.ndarray, li: int, kv_len: int, table: np.ndarray,
+                  fetch_page: Callable[[int, int], np.ndarray], p: Dict,
+                  round_bf16: bool = False) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Layer li of a Llama-style decoder for one new token at position kv_len.
+
+    x is the residual stream entering the layer (fp64 [d]).  Pre-norm attention block, then pre-norm
+    SwiGLU block: x += Wo attn(rope(Wq h), [cache; rope(Wk h)], [cache; Wv h]) with h = RMSNorm(x);
+    x += Wd (silu(Wg h) * (Wu h)) with h = RMSNorm(x).  Query head hq reads KV head hq // (Hq / Hkv).
+    Returns (x leaving the layer, the new token's k [Hkv, hd] after rotation, its v [Hkv, hd]).
+    """
+    D = bf16_to_f64
+    Hq, Hkv, hd = int(p["n_q_heads"]), int(p["n_kv_heads"]), int(p["head_dim"])
+    grp = Hq // Hkv
+    L = p["layers"][li]
+    h = _store(rmsnorm(x, D(L["g1"])), round_bf16)
+    q = _store(linear(h, D(L["Wq"])), round_bf16).reshape(Hq, hd)
+    k = _store(linear(h, D(L["Wk"])), round_bf16).reshape(Hkv, hd)
+    v = _store(linear(h, D(L["Wv"])), round_bf16).reshape(Hkv, hd)
+    q = _store(rope(q, kv_len), round_bf16)
+    k = _store(rope(k, kv_len), round_bf16)
+    Kc, Vc = gather_kv(fetch_page, li, table, kv_len)
+    o = np.empty((Hq, hd))
+    for hq in range(Hq):
+        g = hq // grp
+        Kh = k[g][None, :] if Kc is None else np.concatenate([Kc[g], k[g][None, :]], axis=0)
+        Vh = v[g][None, :] if Vc is None else np.concatenate([Vc[g], v[g][None, :]], axis=0)
+        o[hq] = attention(q[hq], Kh, Vh)
+    o = _store(o.reshape(-1), round_bf16)
+    x = x + linear(o, D(L["Wo"]))
+    h = _store(rmsnorm(x, D(L["g2"])), round_bf16)
+    f = _store(silu(linear(h, D(L["Wg"]))) * linear(h, D(L["Wu"])), round_bf16)
+    x = x + linear(f, D(L["Wd"]))
+    return x, k, v
+
+
+def decoder_head(x: np.ndarray, p: Dict, round_bf16: bool = False) -> np.ndarray:
+    """Final RMSNorm and LM head: logits [vocab] of the residual stream x [d]."""
+    D = bf16_to_f64
+    h = _store(rmsnorm(x, D(p["gf"])), round_bf16)
+    return _store(linear(h, D(p["Wlm"])), round_bf16)
+
+
 def decoder_step(token: int, kv_len: int, table: np.ndarray,
                  fetch_page: Callable[[int, int], np.ndarray], p: Dict,
                  round_bf16: bool = False) -> Dict:
@@ -218,37 +260,19 @@ def decoder_step(token: int, kv_len: int, table: np.ndarray,
 
     p: Emb [V, d], layers[l] = {g1, Wq [Hq*hd, d], Wk [Hkv*hd, d], Wv, Wo [d, Hq*hd], g2,
     Wg [F, d], Wu [F, d], Wd [d, F]}, gf, Wlm [V, d] as bf16 bits; ints n_q_heads,
-    n_kv_heads, head_dim.  Returns logits, argmax, and per layer the appended k, v
-    (fp64 [Hkv, hd]) with the (page, slot) they go to.
+    n_kv_heads, head_dim.  Returns logits, argmax, per layer the appended k, v
+    (fp64 [Hkv, hd]) with the (page, slot) they go to, and the residual stream after the
+    embedding and after every layer ("residual", n_layers + 1 vectors).
     """
-    D = bf16_to_f64
-    Hq, Hkv, hd = int(p["n_q_heads"]), int(p["n_kv_heads"]), int(p["head_dim"])
-    grp = Hq // Hkv
-    x = D(p["Emb"][int(token)])
+    x = bf16_to_f64(p["Emb"][int(token)])
     appended = []
-    for li, L in enumerate(p["layers"]):
-        h = _store(rmsnorm(x, D(L["g1"])), round_bf16)
-        q = _store(linear(h, D(L["Wq"])), round_bf16).reshape(Hq, hd)
-        k = _store(linear(h, D(L["Wk"])), round_bf16).reshape(Hkv, hd)
-        v = _store(linear(h, D(L["Wv"])), round_bf16).reshape(Hkv, hd)
-        q = _store(rope(q, kv_len), round_bf16)
-        k = _store(rope(k, kv_len), round_bf16)
-        Kc, Vc = gather_kv(fetch_page, li, table, kv_len)
-        o = np.empty((Hq, hd))
-        for hq in range(Hq):
-            g = hq // grp
-            Kh = k[g][None, :] if Kc is None else np.concatenate([Kc[g], k[g][None, :]], axis=0)
-            Vh = v[g][None, :] if Vc is None else np.concatenate([Vc[g], v[g][None, :]], axis=0)
-            o[hq] = attention(q[hq], Kh, Vh)
-        o = _store(o.reshape(-1), round_bf16)
-        x = x + linear(o, D(L["Wo"]))
-        h = _store(rmsnorm(x, D(L["g2"])), round_bf16)
-        f = _store(silu(linear(h, D(L["Wg"]))) * linear(h, D(L["Wu"])), round_bf16)
-        x = x + linear(f, D(L["Wd"]))
+    residual = [x]
+    for li in range(len(p["layers"])):
+        x, k, v = decoder_layer(x, li, kv_len, table, fetch_page, p, round_bf16)
+        residual.append(x)
         appended.append({"k": k, "v": v, "page": int(table[kv_len // PAGE]), "slot": kv_len % PAGE})
-    h = _store(rmsnorm(x, D(p["gf"])), round_bf16)
-    logits = _store(linear(h, D(p["Wlm"])), round_bf16)
-    return {"logits": logits, "argmax": argmax_lowest(logits), "appended": appended}
+    logits = decoder_head(x, p, round_bf16)
+    return {"logits": logits, "argmax": argmax_lowest(logits), "appended": appended, "residual": residual}
 
 
 # ------------------------------------------------------------ host-side policy

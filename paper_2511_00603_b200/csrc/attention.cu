@@ -157,6 +157,10 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __
   const int page_begin = t_begin / 16, page_end = (t_end + 15) / 16;
   for (int pg = page_begin + warp; pg < page_end; pg += 4) {
     const int page = rq.table[pg];
+    if (page < 0 || page >= g.kv_pages) {          // outside the pool: reported, read as absent
+      if (lane == 0) atomicExch(g.status, ERR_PAGE_ATTEND);
+      continue;
+    }
     const uint4* kt = reinterpret_cast<const uint4*>(g.kv_layer + (((size_t)page * 2 + 0) * g.Hkv + kvh) * 16 * HD);
     const uint4* vt = reinterpret_cast<const uint4*>(g.kv_layer + (((size_t)page * 2 + 1) * g.Hkv + kvh) * 16 * HD);
     uint4 kr[NL], vr[NL];
@@ -301,6 +305,8 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
   const int gq = lane >> 2, tq = lane & 3;
   const int Hkv = g.Hkv;
   const bf16* kv_layer = g.kv_layer;
+  const long long kv_pages = g.kv_pages;
+  uint32_t bad_mask = 0;                    // pages of this warp whose id was outside the pool (warp-uniform)
 
   // ---- issue all copies of this warp's pages (up to 4), one commit group per page
   unsigned char* wsm = dsm + warp * (NSLOT * 2 * TILE);
@@ -311,6 +317,12 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
     const int pg = page_begin + warp + 4 * i;
     if (i < 4 && pg < page_end) {
       const int page = rq.table[pg];
+      if (page < 0 || page >= kv_pages) {            // outside the pool: reported, read as absent
+        if (lane == 0) atomicExch(g.status, ERR_PAGE_ATTEND);
+        bad_mask |= 1u << i;
+        cp_async_commit();
+        return;
+      }
       const unsigned char* kt = reinterpret_cast<const unsigned char*>(kv_layer + (((size_t)page * 2 + 0) * Hkv + kvh) * 16 * HD);
       const unsigned char* vt = reinterpret_cast<const unsigned char*>(kv_layer + (((size_t)page * 2 + 1) * Hkv + kvh) * 16 * HD);
       const uint32_t kd = wsm_u + (i % NSLOT) * 2 * TILE, vd = kd + TILE;
@@ -348,7 +360,7 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
 
   auto process = [&](int i) {
     const int pg = page_begin + warp + 4 * i;
-    if (pg >= page_end) return;
+    if (pg >= page_end || (bad_mask & (1u << i))) return;
     const uint32_t kd = wsm_u + (i % NSLOT) * 2 * TILE, vd = kd + TILE;
     const int tok0 = pg * 16;
     if (tok0 + 16 > t_end) {
@@ -483,15 +495,27 @@ cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int tot
   return cudaErrorInvalidValue;
 }
 
-__global__ void attn_fill_reqs_kernel(AttnReq* reqs, const int32_t* kv_lens, const int32_t* tables, int stride, int B) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b < B) { reqs[b].table = tables + (size_t)b * stride; reqs[b].len = kv_lens[b]; reqs[b].pad = 0; }
+// Set-up kernel of the single-kernel entry points.  It writes the group descriptor (passed by value, so
+// that no host buffer has to outlive the call) to `dst`, clears the status word and the chunk counters,
+// and fills the request table.  The lengths come from caller device memory: they are clamped to
+// [0, max_len], the range the scratch and the tables were sized for, so that no chunk index can leave the
+// partial buffer.  A request of length 0 attends to nothing and its output row is left unwritten.
+__global__ void attn_prepare_kernel(AttnDecGroup g, AttnDecGroup* dst, AttnReq* reqs, const int32_t* kv_lens,
+                                    const int32_t* tables, int stride, int max_len, int n_counters) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0) { *dst = g; *g.status = 0; }
+  if (i < g.B) {
+    reqs[i].table = tables + (size_t)i * stride;
+    reqs[i].len = min(max(kv_lens[i], 0), max_len);
+    reqs[i].pad = 0;
+  }
+  for (int c = i; c < n_counters; c += gridDim.x * blockDim.x) g.counters[c] = 0;
 }
 
-void launch_attn_fill_reqs(AttnReq* reqs, const int32_t* kv_lens, const int32_t* tables, int stride, int B,
-                           cudaStream_t st) {
-  if (B == 0) return;
-  attn_fill_reqs_kernel<<<(B + 127) / 128, 128, 0, st>>>(reqs, kv_lens, tables, stride, B);
+void launch_attn_prepare(const AttnDecGroup& g, AttnDecGroup* dst, AttnReq* reqs, const int32_t* kv_lens,
+                         const int32_t* tables, int stride, int max_len, int n_counters, cudaStream_t st) {
+  if (g.B == 0) return;
+  attn_prepare_kernel<<<(g.B + 127) / 128, 128, 0, st>>>(g, dst, reqs, kv_lens, tables, stride, max_len, n_counters);
 }
 
 // ------------------------------------------------------------------ encoder attention
@@ -707,13 +731,16 @@ constexpr size_t STATIC_SCRATCH_BYTES = EPARA_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
 constexpr int MAX_DEVICES = 64;
 unsigned char* g_static_ptr[MAX_DEVICES] = {nullptr};
+int g_static_sm[MAX_DEVICES] = {0};
 }  // namespace
 
 extern "C" int epara_decode_attention_static(int device, void* cuda_stream, const void* q, int q_stride,
-                                             const void* kv_layer, const int32_t* kv_lens, const int32_t* tables,
-                                             int table_stride, void* out, int B, int Hq, int Hkv, int hd, int max_len) {
+                                             const void* kv_layer, long long kv_pages, const int32_t* kv_lens,
+                                             const int32_t* tables, int table_stride, void* out, int B, int Hq, int Hkv,
+                                             int hd, int max_len) {
   using namespace epara;
-  if (!q || !kv_layer || !kv_lens || !tables || !out || B < 0 || Hkv <= 0 || Hq <= 0 || Hq % Hkv || max_len <= 0 || hd <= 0)
+  if (!q || !kv_layer || !kv_lens || !tables || !out || B < 0 || Hkv <= 0 || Hq <= 0 || Hq % Hkv || max_len <= 0 || hd <= 0 ||
+      kv_pages <= 0)
     return EPARA_E_INVALID;
   if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(kv_layer) & 15) || (q_stride % 8))
     return EPARA_E_INVALID;
@@ -729,6 +756,9 @@ extern "C" int epara_decode_attention_static(int device, void* cuda_stream, cons
     // first call on this device: resolve the device address of the array (this device is current)
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return EPARA_E_CUDA;
+    int sm = 0;
+    if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sm <= 0) return EPARA_E_CUDA;
+    g_static_sm[device] = sm;
     g_static_ptr[device] = static_cast<unsigned char*>(p);
   }
   unsigned char* s = g_static_ptr[device];
@@ -740,16 +770,26 @@ extern "C" int epara_decode_attention_static(int device, void* cuda_stream, cons
   g.partial = reinterpret_cast<float*>(s + 256 + req_bytes);
   g.counters = reinterpret_cast<int*>(s + 256 + req_bytes + part_bytes);
   g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = chunks; g.req_start = 0;
-  // The array keeps the previous call's contents.  The descriptor and the request table are rewritten
-  // here and every partial that is read is written first by this call's kernel; only the chunk
-  // counters must start at zero, so they are cleared on the stream before the kernel.
-  if (cudaMemsetAsync(g.counters, 0, (size_t)B * Hq * sizeof(int), st) != cudaSuccess) return EPARA_E_CUDA;
-  if (cudaMemcpyAsync(s, &g, sizeof(g), cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
-  launch_attn_fill_reqs(reqs, kv_lens, tables, table_stride, B, st);
+  g.status = reinterpret_cast<int*>(s + DEC_STATUS_OFFSET);
+  g.kv_pages = kv_pages;
+  // The array keeps the previous call's contents.  The set-up kernel rewrites the descriptor and the
+  // request table and clears the status word and the chunk counters (the parts that must start at
+  // zero); every partial that is read is written first by this call's attention kernel.
+  launch_attn_prepare(g, reinterpret_cast<AttnDecGroup*>(s), reqs, kv_lens, tables, table_stride, max_len, B * Hq, st);
   cudaError_t e = launch_attn_decode(reinterpret_cast<const AttnDecGroup*>(s), 1, B, Hkv, Hq, chunks, hd, Hq / Hkv,
-                                     attn_decode_fused(B, Hkv, chunks, 148) ? 1 : 0, st);
+                                     attn_decode_fused(B, Hkv, chunks, g_static_sm[device]) ? 1 : 0, st);
   if (e == cudaErrorInvalidValue) return EPARA_E_UNSUPPORTED;
   return e == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
+}
+
+extern "C" int epara_decode_attention_static_status(int device, int* code) {
+  if (!code || device < 0 || device >= MAX_DEVICES) return EPARA_E_INVALID;
+  *code = 0;
+  if (!g_static_ptr[device]) return EPARA_OK;                 // never used on this device
+  if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
+  if (cudaMemcpy(code, g_static_ptr[device] + epara::DEC_STATUS_OFFSET, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return EPARA_E_CUDA;
+  return *code ? EPARA_E_DEVICE : EPARA_OK;
 }
 
 extern "C" size_t epara_static_scratch_bytes(void) { return STATIC_SCRATCH_BYTES; }

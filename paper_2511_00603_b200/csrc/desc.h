@@ -12,6 +12,10 @@ typedef __nv_bfloat16 bf16;
 
 enum : int { EPI_BIAS = 1, EPI_GELU = 2, EPI_SWIGLU = 4, EPI_RESID_F32 = 8 };
 
+// Codes a kernel leaves in the step's device status word (0 = none).  1..49 are bounded waits that ran
+// out (the role that gave up); the others are indices found out of range, whose access was skipped.
+enum : int { ERR_PAGE_APPEND = 101, ERR_PAGE_ATTEND = 102, ERR_SELFTEST_WAIT = 90 };
+
 // Per admitted request (model order, then batch order).
 struct ReqDesc {
   const void* input;     // MLP row / ViT image
@@ -86,6 +90,8 @@ struct RopeGroup {
   bf16* kv_layer;        // [pages][2][Hkv][16][hd]
   const ReqDesc* reqs;
   const float2* cs;      // [max position + 1][hd/2]: (cos, sin) of position * 10000^(-2j/hd)
+  int* status;           // device word: set to ERR_PAGE_APPEND when a block table names a page outside the pool
+  long long kv_pages;    // pages of the pool; a page id outside [0, kv_pages) is reported, its write skipped
   int B, Hq, Hkv, hd;
 };
 
@@ -108,6 +114,8 @@ struct AttnDecGroup {
   int req_start;         // first grid.z index of this group
   int reqs_stable;       // 1: `reqs` was uploaded before the step's first kernel (a block past a request's
                          // length may leave without the dependency wait); 0: an earlier kernel writes it
+  int* status;           // device word: set to ERR_PAGE_ATTEND when a block table names a page outside the pool
+  long long kv_pages;    // pages of the pool; a page id outside [0, kv_pages) is reported and read as absent
 };
 
 struct alignas(64) AttnEncGroup {

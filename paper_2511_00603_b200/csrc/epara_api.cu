@@ -93,6 +93,9 @@ struct Op {
   AssembleGroup asmb;
   OutputGroup outp;
   double weight_bytes;
+  const void* trace_src;   // EPARA_K_TRACE: copy rows * trace_row_bytes from here ...
+  void* trace_dst;         // ... to here
+  size_t trace_row_bytes;
 };
 
 struct Request {
@@ -100,13 +103,17 @@ struct Request {
   epara_inputs in;
 };
 
-enum { T_QUEUED = 0, T_INFLIGHT = 1, T_DROPPED = 2 };
+// T_INFLIGHT: admitted to a step whose slot still holds the step's record.  T_DONE: the final answer is
+// in `result` (a dropped request, a step that failed on the host, or a step whose slot was recycled).
+enum { T_QUEUED = 0, T_INFLIGHT = 1, T_DONE = 2 };
 struct Ticket {
   int state;
   int model;
   uint64_t step;
   void* out_logits;
   int32_t* out_argmax;
+  int result;          // T_DONE: EPARA_OK / EPARA_E_TIMEOUT / EPARA_E_DEVICE / EPARA_E_CUDA / EPARA_E_RESOURCE
+  int device_error;    // T_DONE with EPARA_E_DEVICE: the code the kernel recorded
 };
 
 struct Model {
@@ -122,14 +129,19 @@ struct Model {
   size_t splitk_bytes = 0, splitk_tiles = 0;   // largest split-k partial buffer / tile count of its GEMMs
 };
 
+// The first BLOB_HEADER bytes of a slot's device blob hold the step's status word; the upload of the blob
+// writes zeros there, so every step starts with a clear word of its own.
+constexpr size_t BLOB_HEADER = 64;
 struct Slot {
   unsigned char* host;  // pinned blob
   unsigned char* dev;   // device blob (in the workspace)
-  int* status_host;     // pinned
+  int* status_host;     // pinned copy of the step's status word, valid once `done` has fired
   cudaEvent_t done;
   uint64_t step_id;     // 0 = never used
   bool busy;
   bool profiled;        // the step in this slot was bracketed with events
+  int launch_status;    // EPARA_OK, or what a failed launch of the step maps to
+  std::vector<uint64_t> tickets;   // requests admitted to the step in this slot
   std::vector<cudaEvent_t> prof;   // 2 per launch when profiling
   std::vector<int> prof_kind;
 };
@@ -139,6 +151,9 @@ struct Launch {
   size_t off;
   int n_groups;
   int p0, p1, p2, p3;
+  const void* src;   // EPARA_K_TRACE
+  void* dst;
+  size_t bytes;
 };
 
 }  // namespace
@@ -148,12 +163,12 @@ struct epara_ctx {
   int sm_count;
   unsigned char* ws;
   size_t ws_bytes, ws_used;
-  int* dev_status;
   std::vector<Model*> models;
   std::unordered_map<uint64_t, Ticket> tickets;
   uint64_t next_ticket, next_step;
   Slot slots[N_SLOTS];
   uint64_t last_step_slot;
+  int max_profile_launches;
 };
 
 namespace {
@@ -171,9 +186,17 @@ size_t carve_size(size_t& used, size_t bytes) {
   return off;
 }
 
-struct Buf {
-  void* p;
-};
+// SM count of a device (cached; 148 on a B200).  Tile widths of the weight-streaming GEMMs depend on it.
+int device_sm_count(int device) {
+  static int cache[64] = {0};
+  if (device < 0 || device >= 64) return 148;
+  if (cache[device] == 0) {
+    int sm = 0;
+    if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sm <= 0) return 148;
+    cache[device] = sm;
+  }
+  return cache[device];
+}
 
 // Builds the op list of a model.  With c == nullptr only counts workspace bytes (in *need).
 // Buffers are requested through `get`, which either carves or counts.
@@ -399,6 +422,16 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
   g.kind = EPARA_K_GATHER; g.rows_per_req = 1;
   g.gather.kind = GATHER_EMB; g.gather.out = x; g.gather.emb = (const bf16*)t[0]; g.gather.width = dm; g.gather.ld = dm;
   m->ops.push_back(g);
+  // debug trace: the residual stream after the embedding and after every layer, [n_layers + 1][max_batch][d] fp32
+  auto add_trace = [&](int index) {
+    if (!d.trace) return;
+    Op tr;
+    memset(&tr, 0, sizeof(tr));
+    tr.kind = EPARA_K_TRACE; tr.rows_per_req = 1;
+    tr.trace_src = x; tr.trace_dst = (float*)d.trace + (size_t)index * B * dm; tr.trace_row_bytes = (size_t)dm * 4;
+    m->ops.push_back(tr);
+  };
+  add_trace(0);
   const size_t layer_elems = (size_t)d.kv_pages * 2 * Hkv * 16 * hd;
   for (int l = 0; l < d.n_layers; ++l) {
     const void* const* w = t + 1 + 6 * l;
@@ -409,7 +442,7 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
     memset(&r, 0, sizeof(r));
     r.kind = EPARA_K_ROPE; r.rows_per_req = 1;
     r.rope.qkv = qkv; r.rope.kv_layer = kv_layer; r.rope.cs = rope_cs;
-    r.rope.Hq = Hq; r.rope.Hkv = Hkv; r.rope.hd = hd;
+    r.rope.Hq = Hq; r.rope.Hkv = Hkv; r.rope.hd = hd; r.rope.kv_pages = d.kv_pages;
     m->ops.push_back(r);
     Op at;
     memset(&at, 0, sizeof(at));
@@ -417,12 +450,13 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
     at.adec.q = qkv; at.adec.q_stride = nq; at.adec.kv_layer = kv_layer; at.adec.out = a; at.adec.partial = partial;
     at.adec.counters = chunk_counters;
     at.adec.Hq = Hq; at.adec.Hkv = Hkv; at.adec.hd = hd; at.adec.max_chunks = m->max_chunks;
-    at.adec.reqs_stable = 1;
+    at.adec.reqs_stable = 1; at.adec.kv_pages = d.kv_pages;
     m->ops.push_back(at);
     if (!add_gemm(bl, m, a, Hq * hd, Bcap, w[2], dm, Hq * hd, x, dm, nullptr, EPI_RESID_F32, 1)) return EPARA_E_CUDA;
     add_norm(m, x, dm, h, w[3], nullptr, dm, NORM_RMS, 1e-5f, 1);
     if (!add_gemm(bl, m, h, dm, Bcap, w[4], 2 * F, dm, f, F, nullptr, EPI_SWIGLU, 1)) return EPARA_E_CUDA;
     if (!add_gemm(bl, m, f, F, Bcap, w[5], dm, F, x, dm, nullptr, EPI_RESID_F32, 1)) return EPARA_E_CUDA;
+    add_trace(l + 1);
   }
   const void* const* w = t + 1 + 6 * d.n_layers;
   add_norm(m, x, dm, h, w[0], nullptr, dm, NORM_RMS, 1e-5f, 1);
@@ -486,6 +520,33 @@ void admit_impl(int n, const uint64_t* tickets, const long long* deadline, const
   (void)tickets;
 }
 
+// Gives every request of the step recorded in `slot` its final answer (the step has finished on the
+// device, or never ran) and forgets the step, so that the slot can take another one.
+void finalize_slot(epara_ctx* c, Slot& slot) {
+  const int code = *slot.status_host;
+  for (uint64_t tk : slot.tickets) {
+    auto it = c->tickets.find(tk);
+    if (it == c->tickets.end() || it->second.state != T_INFLIGHT || it->second.step != slot.step_id) continue;
+    Ticket& t = it->second;
+    t.state = T_DONE;
+    t.device_error = code;
+    t.result = code != 0 ? EPARA_E_DEVICE : slot.launch_status;
+  }
+  slot.tickets.clear();
+  slot.busy = false;
+}
+
+// A step that fails on the host after admission: its requests answer `result`, nothing stays in flight.
+void fail_tickets(epara_ctx* c, const std::vector<uint64_t>& tks, int result) {
+  for (uint64_t tk : tks) {
+    auto it = c->tickets.find(tk);
+    if (it == c->tickets.end()) continue;
+    it->second.state = T_DONE;
+    it->second.result = result;
+    it->second.device_error = 0;
+  }
+}
+
 }  // namespace
 
 // =============================================================================== C ABI
@@ -536,7 +597,7 @@ size_t epara_model_workspace_bytes(const epara_config* cfg, const epara_model_de
   m.tensors.assign(d->tensors, d->tensors + d->n_tensors);
   if (d->kind == EPARA_MODEL_MLP) m.dims.assign(d->mlp_dims, d->mlp_dims + d->n_layers + 1);
   m.max_batch = effective_max_batch(*cfg, *d);
-  Builder bl{nullptr, 0, false, 148, cfg->gemm_impl};
+  Builder bl{nullptr, 0, false, device_sm_count(cfg->device), cfg->gemm_impl};
   build_model(bl, &m, *cfg);
   finish_model(bl, &m);
   return bl.need + 256;
@@ -545,7 +606,7 @@ size_t epara_model_workspace_bytes(const epara_config* cfg, const epara_model_de
 int epara_init(const epara_config* cfg, epara_ctx** out) {
   if (!cfg || !out) return EPARA_E_INVALID;
   if (!cfg->workspace || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255)) return EPARA_E_INVALID;
-  const size_t fixed = N_SLOTS * BLOB_BYTES + 256;
+  const size_t fixed = N_SLOTS * (BLOB_BYTES + 256);
   if (cfg->workspace_bytes < fixed) return EPARA_E_RESOURCE;
   if (cudaSetDevice(cfg->device) != cudaSuccess) return EPARA_E_CUDA;
   epara_ctx* c = new (std::nothrow) epara_ctx();
@@ -560,17 +621,17 @@ int epara_init(const epara_config* cfg, epara_ctx** out) {
   c->next_ticket = 1;
   c->next_step = 1;
   c->last_step_slot = 0;
+  c->max_profile_launches = MAX_PROFILE_LAUNCHES;
   int sm = 0;
   if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) { delete c; return EPARA_E_CUDA; }
   c->sm_count = sm;
-  c->dev_status = (int*)carve(c, 256);
-  if (cudaMemset(c->dev_status, 0, 256) != cudaSuccess) { delete c; return EPARA_E_CUDA; }
   for (int i = 0; i < N_SLOTS; ++i) {
     Slot& s = c->slots[i];
     s.dev = (unsigned char*)carve(c, BLOB_BYTES);
     s.step_id = 0;
     s.busy = false;
     s.profiled = false;
+    s.launch_status = EPARA_OK;
     if (cudaMallocHost((void**)&s.host, BLOB_BYTES) != cudaSuccess ||
         cudaMallocHost((void**)&s.status_host, 64) != cudaSuccess ||
         cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) != cudaSuccess) {
@@ -649,6 +710,7 @@ int epara_submit(epara_ctx* c, int model_id, int category, const epara_inputs* i
   m->q[category].push_back(r);
   Ticket t;
   t.state = T_QUEUED; t.model = model_id; t.step = 0; t.out_logits = in->out_logits; t.out_argmax = in->out_argmax;
+  t.result = EPARA_OK; t.device_error = 0;
   c->tickets[r.ticket] = t;
   *ticket = r.ticket;
   return EPARA_OK;
@@ -698,7 +760,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       admit_impl(n, tk.data(), dl.data(), sid.data(), now_ns, cap, (cat == EPARA_CAT_FS_LT1) ? c->cfg.mf_max : 0, adm, drp);
       std::vector<char> gone(n, 0);
       for (int i : adm) { a.reqs.push_back(q[i]); gone[i] = 1; c->tickets[q[i].ticket].state = T_INFLIGHT; c->tickets[q[i].ticket].step = step_id; }
-      for (int i : drp) { gone[i] = 1; c->tickets[q[i].ticket].state = T_DROPPED; }
+      for (int i : drp) { gone[i] = 1; Ticket& t = c->tickets[q[i].ticket]; t.state = T_DONE; t.result = EPARA_E_TIMEOUT; }
       std::deque<Request> rest;
       for (int i = 0; i < n; ++i) if (!gone[i]) rest.push_back(q[i]);
       q.swap(rest);
@@ -714,12 +776,23 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
   }
 
   // ---- blob slot ----
+  std::vector<uint64_t> admitted_tickets;
+  for (Active& a : act)
+    for (Request& r : a.reqs) admitted_tickets.push_back(r.ticket);
   Slot& slot = c->slots[step_id % N_SLOTS];
   if (slot.busy) {
-    if (cudaEventSynchronize(slot.done) != cudaSuccess) return EPARA_E_CUDA;
-    slot.busy = false;
+    // the step that used this slot N_SLOTS steps ago: wait for it and give its requests their answers
+    if (cudaEventSynchronize(slot.done) != cudaSuccess) {
+      fail_tickets(c, admitted_tickets, EPARA_E_CUDA);
+      if (info) *info = inf;
+      return EPARA_E_CUDA;
+    }
   }
-  size_t off = 0;
+  if (!slot.tickets.empty()) finalize_slot(c, slot);
+  slot.busy = false;
+  memset(slot.host, 0, BLOB_HEADER);         // the step's status word, cleared on the device by the upload
+  int* const dev_status = reinterpret_cast<int*>(slot.dev);
+  size_t off = BLOB_HEADER;
   auto put = [&](const void* src, size_t bytes, size_t align) -> size_t {
     off = align_up(off, align);
     if (off + bytes > BLOB_BYTES) return (size_t)-1;
@@ -746,7 +819,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
   }
 
   // ---- plan (A1): sweep the kernel kinds until every model's op list is exhausted ----
-  static const int sweep[] = {EPARA_K_GATHER, EPARA_K_ASSEMBLE, EPARA_K_NORM, EPARA_K_GEMM, EPARA_K_ROPE,
+  static const int sweep[] = {EPARA_K_GATHER, EPARA_K_TRACE, EPARA_K_ASSEMBLE, EPARA_K_NORM, EPARA_K_GEMM, EPARA_K_ROPE,
                               EPARA_K_ATTN_DEC, EPARA_K_ATTN_ENC, EPARA_K_OUTPUT};
   std::vector<Launch> launches;
   const bool simt = c->cfg.gemm_impl == EPARA_GEMM_SIMT;
@@ -759,6 +832,18 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
         if (a.cursor < a.m->ops.size() && a.m->ops[a.cursor].kind == kind) who.push_back(&a);
       if (who.empty()) continue;
       more = true;
+      if (kind == EPARA_K_TRACE) {               // debug copies of the residual stream: one plain copy per model
+        for (Active* a : who) {
+          const Op& op = a->m->ops[a->cursor];
+          Launch LL;
+          memset(&LL, 0, sizeof(LL));
+          LL.kind = kind; LL.n_groups = 1;
+          LL.src = op.trace_src; LL.dst = op.trace_dst; LL.bytes = (size_t)a->B * op.trace_row_bytes;
+          launches.push_back(LL);
+          a->cursor++;
+        }
+        continue;
+      }
       // GEMM groups go out in up to three launches: tensor-core tiles (pass 0), the weight-streaming
       // kernel for groups that never exceed 16 rows (pass 1) and 256-row tiles on CTA pairs for the dense
       // bf16-output groups (pass 2); encoder attention in two: the tcgen05 kernel (pass 0) and the
@@ -793,6 +878,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           for (Active* a : same) {
             AttnDecGroup g = a->m->ops[a->cursor].adec;
             g.B = a->B; g.reqs = (const AttnReq*)(slot.dev + a->areq_off); g.req_start = total_B;
+            g.status = dev_status;
             total_B += a->B;
             max_hkv = std::max(max_hkv, g.Hkv); max_hq = std::max(max_hq, g.Hq);
             for (int b = 0; b < a->B; ++b)
@@ -857,12 +943,17 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
             inf.gemm_groups++;
             inf.gemm_flops += 2.0 * rows * g.N * g.K;
             inf.weight_bytes += op.weight_bytes;
+            if (g.stream == 1) {
+              inf.stream_gemm_flops += 2.0 * rows * g.N * g.K;
+              inf.stream_weight_bytes += op.weight_bytes;
+            }
             if (put(&g, sizeof(g), 64) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_ROPE: {
             RopeGroup g = op.rope;
             g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
+            g.status = dev_status;
             mx = std::max(mx, a->B);
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
@@ -896,43 +987,46 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       }
     }
   }
-  if (overflow) {
-    // nothing was launched: give the admitted requests a definite answer
-    for (Active& a : act)
-      for (Request& r : a.reqs) c->tickets[r.ticket].state = T_DROPPED;
+  // Every exit from here on that launches nothing gives the admitted requests a definite answer.
+  auto fail = [&](int result) {
+    fail_tickets(c, admitted_tickets, result);
     if (info) *info = inf;
-    return EPARA_E_RESOURCE;
-  }
-
-  // ---- upload + launch ----
-  if (cudaMemcpyAsync(slot.dev, slot.host, off, cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
+    return result;
+  };
+  if (overflow) return fail(EPARA_E_RESOURCE);     // the step's descriptors do not fit the blob
   const bool prof = c->cfg.profile != 0;
-  slot.profiled = prof;
   if (prof) {
-    if (launches.size() > MAX_PROFILE_LAUNCHES) return EPARA_E_RESOURCE;
+    if ((int)launches.size() > c->max_profile_launches) return fail(EPARA_E_RESOURCE);
     while (slot.prof.size() < 2 * launches.size()) {
       cudaEvent_t e;
-      if (cudaEventCreate(&e) != cudaSuccess) return EPARA_E_CUDA;
+      if (cudaEventCreate(&e) != cudaSuccess) return fail(EPARA_E_CUDA);
       slot.prof.push_back(e);
     }
     slot.prof_kind.clear();
   }
+
+  // ---- upload + launch ----
+  if (cudaMemcpyAsync(slot.dev, slot.host, off, cudaMemcpyHostToDevice, st) != cudaSuccess) return fail(EPARA_E_CUDA);
+  slot.profiled = prof;
   cudaError_t err = cudaSuccess;
   int li = 0, n_kernels = 0;
   for (const Launch& L : launches) {
     n_kernels += 1 + ((L.kind == EPARA_K_ATTN_DEC && L.p2 > 1 &&
                        !attn_decode_fused(L.p0, L.p1 & 0xffff, L.p2, c->sm_count)) ? 1 : 0);
     const unsigned char* gp = slot.dev + L.off;
-    if (prof) { cudaEventRecord(slot.prof[2 * li], st); slot.prof_kind.push_back(L.kind); }
+    if (prof) {
+      cudaEventRecord(slot.prof[2 * li], st);
+      slot.prof_kind.push_back(L.kind == EPARA_K_GEMM && L.p2 == 1 ? (int)EPARA_K_GEMM_STREAM : L.kind);
+    }
     switch (L.kind) {
       case EPARA_K_GATHER: launch_gather((const GatherGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_ASSEMBLE: launch_assemble((const AssembleGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_NORM: launch_norm((const NormGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_GEMM:
         if (L.p2 == 1) err = launch_gemm_stream((const GemmGroup*)gp, L.n_groups, L.p0, L.p1, st);
-        else if (L.p2 == 2) err = launch_gemm_tc_pair((const GemmGroup*)gp, L.n_groups, L.p0, c->dev_status, c->sm_count, st);
+        else if (L.p2 == 2) err = launch_gemm_tc_pair((const GemmGroup*)gp, L.n_groups, L.p0, dev_status, c->sm_count, st);
         else if (simt) launch_gemm_simt((const GemmGroup*)gp, L.n_groups, L.p0, st);
-        else err = launch_gemm_tc((const GemmGroup*)gp, L.n_groups, L.p0, L.p3, c->dev_status, c->sm_count, st);
+        else err = launch_gemm_tc((const GemmGroup*)gp, L.n_groups, L.p0, L.p3, dev_status, c->sm_count, st);
         break;
       case EPARA_K_ROPE: launch_rope_append((const RopeGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_ATTN_DEC:
@@ -940,54 +1034,68 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
                                  L.p3 & 255, attn_decode_fused(L.p0, L.p1 & 0xffff, L.p2, c->sm_count) ? 1 : 0, st);
         break;
       case EPARA_K_ATTN_ENC:
-        if (L.p2 == 0) err = launch_attn_encoder_tc((const AttnEncGroup*)gp, L.n_groups, L.p0, c->dev_status, c->sm_count, st);
+        if (L.p2 == 0) err = launch_attn_encoder_tc((const AttnEncGroup*)gp, L.n_groups, L.p0, dev_status, c->sm_count, st);
         else err = launch_attn_encoder((const AttnEncGroup*)gp, L.n_groups, L.p0, L.p1, st);
         break;
       case EPARA_K_OUTPUT: launch_output((const OutputGroup*)gp, L.n_groups, L.p1, st); break;
+      case EPARA_K_TRACE: err = cudaMemcpyAsync(L.dst, L.src, L.bytes, cudaMemcpyDeviceToDevice, st); break;
     }
     if (prof) cudaEventRecord(slot.prof[2 * li + 1], st);
     ++li;
     if (err != cudaSuccess) break;
   }
   if (err == cudaSuccess) err = cudaGetLastError();
-  cudaMemcpyAsync(slot.status_host, c->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st);
-  cudaEventRecord(slot.done, st);
+  // A launch that failed leaves the step incomplete: the kernels already enqueued still run, the event
+  // still fires, and the step's requests then answer EPARA_E_CUDA instead of EPARA_OK.
+  slot.launch_status = err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
+  *slot.status_host = 0;
+  if (cudaMemcpyAsync(slot.status_host, dev_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaEventRecord(slot.done, st) != cudaSuccess)
+    slot.launch_status = EPARA_E_CUDA;
   slot.busy = true;
   slot.step_id = step_id;
+  slot.tickets = admitted_tickets;
   c->last_step_slot = step_id % N_SLOTS;
   inf.launches = n_kernels;
   if (info) *info = inf;
-  return err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
+  return slot.launch_status;
 }
 
 int epara_collect(epara_ctx* c, uint64_t ticket, epara_output* out) {
   if (!c) return EPARA_E_INVALID;
   auto it = c->tickets.find(ticket);
   if (it == c->tickets.end()) return EPARA_E_INVALID;
-  Ticket& t = it->second;
-  if (t.state == T_QUEUED) return EPARA_PENDING;
-  int result = EPARA_OK;
-  if (t.state == T_DROPPED) {
-    result = EPARA_E_TIMEOUT;
-  } else {
-    Slot& s = c->slots[t.step % N_SLOTS];
-    if (s.step_id == t.step && s.busy) {
+  if (it->second.state == T_QUEUED) return EPARA_PENDING;
+  if (it->second.state == T_INFLIGHT) {
+    Slot& s = c->slots[it->second.step % N_SLOTS];
+    if (s.step_id == it->second.step && s.busy) {
       cudaError_t e = cudaEventQuery(s.done);
       if (e == cudaErrorNotReady) return EPARA_PENDING;
-      if (e != cudaSuccess) return EPARA_E_CUDA;
-      s.busy = false;
+      if (e != cudaSuccess) { s.launch_status = EPARA_E_CUDA; *s.status_host = 0; }
+      finalize_slot(c, s);            // answers every request of that step, this one included
     }
-    if (s.step_id == t.step && *s.status_host != 0) result = EPARA_E_DEVICE;
+    if (it->second.state != T_DONE) {   // (cannot happen: an in-flight ticket's step is always in its slot)
+      it->second.state = T_DONE;
+      it->second.result = EPARA_E_CUDA;
+    }
   }
+  const Ticket t = it->second;
   if (out) {
-    out->status = result;
+    out->status = t.result;
     out->step_id = t.step;
     out->logits = t.out_logits;
     out->argmax = t.out_argmax;
     out->n_out = c->models[t.model]->n_out;
+    out->device_error = t.device_error;
   }
   c->tickets.erase(it);
-  return result;
+  return t.result;
+}
+
+int epara_set_max_profile_launches(epara_ctx* c, int n) {
+  if (!c || n < 0) return EPARA_E_INVALID;
+  c->max_profile_launches = n;
+  return EPARA_OK;
 }
 
 int epara_set_profile(epara_ctx* c, int on) {
@@ -1014,11 +1122,12 @@ int epara_step_profile(epara_ctx* c, float* ms_per_kind, int* launches_per_kind)
 // ---------------------------------------------------------------- single-kernel entry points
 size_t epara_gemm_scratch_bytes(int n) { return (size_t)(n > 0 ? n : 0) * sizeof(GemmGroup) + 256; }
 
-size_t epara_gemm_scratch_bytes_for(const epara_gemm_problem* p, int n) {
+size_t epara_gemm_scratch_bytes_for(int device, const epara_gemm_problem* p, int n) {
+  const int sm_count = device_sm_count(device);
   size_t bytes = epara_gemm_scratch_bytes(n);
   for (int i = 0; i < n && p; ++i) {
     int bn = 128, ks = 1;
-    gemm_tc_config(p[i].M, p[i].N, p[i].K, p[i].epilogue, 148, &bn, &ks);
+    gemm_tc_config(p[i].M, p[i].N, p[i].K, p[i].epilogue, sm_count, &bn, &ks);
     if (ks > 1) {
       const size_t tiles_m = (size_t)(p[i].M + TC_BM - 1) / TC_BM, tiles_n = (size_t)(p[i].N + bn - 1) / bn;
       bytes = align_up(bytes, 256) + (size_t)ks * tiles_m * TC_BM * tiles_n * bn * 4;
@@ -1031,12 +1140,13 @@ size_t epara_gemm_scratch_bytes_for(const epara_gemm_problem* p, int n) {
 int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm_problem* p, int n, void* scratch,
                        size_t scratch_bytes) {
   if (n < 0 || (n > 0 && !p) || !scratch || (reinterpret_cast<uintptr_t>(scratch) & 255)) return EPARA_E_INVALID;
-  if (scratch_bytes < (impl == EPARA_GEMM_SIMT ? epara_gemm_scratch_bytes(n) : epara_gemm_scratch_bytes_for(p, n)))
+  if (scratch_bytes < (impl == EPARA_GEMM_SIMT ? epara_gemm_scratch_bytes(n) : epara_gemm_scratch_bytes_for(device, p, n)))
     return EPARA_E_RESOURCE;
   if (n == 0) return EPARA_OK;
   if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool simt = impl == EPARA_GEMM_SIMT;
+  const int sm_count = device_sm_count(device);
   std::vector<GemmGroup> gs, gs_stream, gs_pair;   // tensor-core (or CUDA-core) groups; weight-streaming groups (M <= 16); CTA-pair groups
   int total = 0, total_stream = 0, max_rows_stream = 0, total_pair = 0;
   size_t soff = epara_gemm_scratch_bytes(n);
@@ -1064,7 +1174,7 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
       gs_stream.push_back(g);
       continue;
     }
-    if (!simt) gemm_tc_config(q.M, q.N, q.K, q.epilogue, 148, &g.bn, &g.ksplit);
+    if (!simt) gemm_tc_config(q.M, q.N, q.K, q.epilogue, sm_count, &g.bn, &g.ksplit);
     if (!simt && gemm_tc_pair_eligible(q.M, q.N, q.K, q.epilogue, g.bn, g.ksplit)) {
       g.stream = 2;
       g.tiles_m = (q.M + 2 * TC_BM - 1) / (2 * TC_BM); g.tiles_n = (q.N + g.bn - 1) / g.bn;
@@ -1116,8 +1226,7 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
     launch_gemm_simt(dev_groups, (int)gs.size(), total, st);
     err = cudaGetLastError();
   } else {
-    int sm = 0;
-    cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device);
+    const int sm = sm_count;
     int max_bn = 0;
     for (const GemmGroup& g : gs) max_bn = std::max(max_bn, g.bn);
     err = launch_gemm_tc(dev_groups, (int)gs.size(), total, max_bn, status, sm, st);
@@ -1136,9 +1245,10 @@ size_t epara_decode_attention_scratch_bytes(int B, int Hq, int hd, int max_len) 
 }
 
 int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_stride, const void* kv_layer,
-                           const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out, int B, int Hq,
-                           int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes) {
-  if (!q || !kv_layer || !kv_lens || !tables || !out || !scratch || B < 0 || Hkv <= 0 || Hq % Hkv || max_len <= 0)
+                           long long kv_pages, const int32_t* kv_lens, const int32_t* tables, int table_stride, void* out,
+                           int B, int Hq, int Hkv, int hd, int max_len, void* scratch, size_t scratch_bytes) {
+  if (!q || !kv_layer || !kv_lens || !tables || !out || !scratch || B < 0 || Hkv <= 0 || Hq % Hkv || max_len <= 0 ||
+      kv_pages <= 0)
     return EPARA_E_INVALID;
   if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(kv_layer) & 15) || (q_stride % 8) ||
       (reinterpret_cast<uintptr_t>(scratch) & 255))
@@ -1148,6 +1258,7 @@ int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_s
   if (cudaSetDevice(device) != cudaSuccess) return EPARA_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   unsigned char* s = (unsigned char*)scratch;
+  static_assert(sizeof(AttnDecGroup) <= DEC_STATUS_OFFSET && DEC_STATUS_OFFSET + sizeof(int) <= 256, "scratch header");
   AttnDecGroup g;
   memset(&g, 0, sizeof(g));
   const int g_chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK;
@@ -1155,12 +1266,13 @@ int epara_decode_attention(int device, void* cuda_stream, const void* q, int q_s
   g.q = (const bf16*)q; g.q_stride = q_stride; g.kv_layer = (const bf16*)kv_layer; g.reqs = reqs; g.out = (bf16*)out;
   g.partial = (float*)(s + 256 + align_up((size_t)B * sizeof(AttnReq), 256));
   g.counters = (int*)((unsigned char*)g.partial + align_up((size_t)B * Hq * g_chunks * (hd + 2) * 4, 256));
-  if (cudaMemsetAsync(g.counters, 0, (size_t)B * Hq * sizeof(int), st) != cudaSuccess) return EPARA_E_CUDA;
-  g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = (max_len + ATTN_CHUNK - 1) / ATTN_CHUNK; g.req_start = 0;
-  if (cudaMemcpyAsync(s, &g, sizeof(g), cudaMemcpyHostToDevice, st) != cudaSuccess) return EPARA_E_CUDA;
-  launch_attn_fill_reqs(reqs, kv_lens, tables, table_stride, B, st);
+  g.B = B; g.Hq = Hq; g.Hkv = Hkv; g.hd = hd; g.max_chunks = g_chunks; g.req_start = 0;
+  g.status = (int*)(s + DEC_STATUS_OFFSET);
+  g.kv_pages = kv_pages;
+  // one set-up kernel writes the descriptor, clears the status word and the counters and fills the request table
+  launch_attn_prepare(g, (AttnDecGroup*)s, reqs, kv_lens, tables, table_stride, max_len, B * Hq, st);
   cudaError_t e = launch_attn_decode((const AttnDecGroup*)s, 1, B, Hkv, Hq, g.max_chunks, hd, Hq / Hkv,
-                                     attn_decode_fused(B, Hkv, g.max_chunks, 148) ? 1 : 0, st);
+                                     attn_decode_fused(B, Hkv, g.max_chunks, device_sm_count(device)) ? 1 : 0, st);
   if (e == cudaErrorInvalidValue) return EPARA_E_UNSUPPORTED;
   return e == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
 }

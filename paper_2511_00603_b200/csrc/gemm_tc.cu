@@ -588,6 +588,10 @@ __device__ __forceinline__ Item decode_item_pair(const G& g, int local, int rank
   return it;
 }
 
+// A producer that gives up cannot await its copies in flight (their bytes are counted on the leader's
+// barrier, which may never complete once the peer has given up too): it sleeps this long instead, far
+// more than a copy takes, before the CTAs meet at the closing cluster barrier.
+constexpr unsigned long long PAIR_DRAIN_NS = 200000ull;
 constexpr int PAIR_W_WARP = 2 + EPI_WARPS;                     // the warp after the epilogue warps loads W
 constexpr int PAIR_THREADS = N_THREADS + 32;
 
@@ -665,7 +669,7 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
           if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) *abort_flag = 1;
+      if (!ok) { *abort_flag = 1; drain_sleep(PAIR_DRAIN_NS); }
     }
   } else if (warp == PAIR_W_WARP) {
     // ------------------------------------------------------------ TMA producer of W (one per CTA)
@@ -692,7 +696,7 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
           if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) *abort_flag = 1;
+      if (!ok) { *abort_flag = 1; drain_sleep(PAIR_DRAIN_NS); }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (rank 0 only)

@@ -44,9 +44,11 @@ constexpr int ATTN_CHUNK = 256;
 bool attn_decode_fused(int total_B, int max_Hkv, int max_chunks, int sm_count);
 cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int total_B, int max_Hkv, int max_Hq,
                                int max_chunks, int hd, int gqa, int fused, cudaStream_t st);
-// Fills AttnReq[b] = {tables + b*stride, kv_lens[b]} on the device.
-void launch_attn_fill_reqs(AttnReq* reqs, const int32_t* kv_lens, const int32_t* tables, int stride, int B,
-                           cudaStream_t st);
+// Set-up of a single-kernel decode-attention call on the stream: writes `g` to `dst`, clears *g.status and
+// g.counters[0 .. n_counters), fills reqs[b] = {tables + b*stride, kv_lens[b] clamped to [0, max_len]}.
+void launch_attn_prepare(const AttnDecGroup& g, AttnDecGroup* dst, AttnReq* reqs, const int32_t* kv_lens,
+                         const int32_t* tables, int stride, int max_len, int n_counters, cudaStream_t st);
+constexpr int DEC_STATUS_OFFSET = 192;   // byte offset of the status word in a single-kernel call's scratch
 
 // Encoder attention on tcgen05 for groups with AttnEncGroup::tc (hd 64, T <= ENC_TC_MAX_T): persistent,
 // one item per (image, head); total_items = sum of B * H.  `status` as for the GEMM.

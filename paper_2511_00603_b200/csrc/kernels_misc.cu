@@ -230,6 +230,7 @@ void launch_norm(const NormGroup* groups, int n_groups, int max_blocks, cudaStre
 // One block per request.  The new token sits at position kv_len: q and k are rotated there
 // (interleaved pairs; cos and sin come from the model's table, computed from fp64 angles when the
 // model was placed), q in place, k and v written to the cache page table[pos/16], slot pos%16.
+// The page id comes from the caller's block table and is checked against the pool's page count.
 __global__ void __launch_bounds__(256) rope_append_kernel(const RopeGroup* __restrict__ groups) {
   const RopeGroup g = groups[blockIdx.y];
   const int b = blockIdx.x;
@@ -240,6 +241,11 @@ __global__ void __launch_bounds__(256) rope_append_kernel(const RopeGroup* __res
   const int pos = r.kv_len, hd = g.hd, half = hd >> 1;
   const float2* cs = g.cs + (size_t)pos * half;
   const int page = r.table[pos / 16], slot = pos % 16;
+  // a page id outside the pool is reported and nothing is written for this request (q stays unrotated)
+  if (page < 0 || page >= g.kv_pages) {
+    if (threadIdx.x == 0) atomicExch(g.status, ERR_PAGE_APPEND);
+    return;
+  }
   bf16* row = g.qkv + (size_t)b * (g.Hq + 2 * g.Hkv) * hd;
   const int n_rot = (g.Hq + g.Hkv) * half;
   for (int e = threadIdx.x; e < n_rot; e += blockDim.x) {

@@ -28,8 +28,10 @@ __device__ __forceinline__ unsigned long long globaltimer() {
 // Bounded wait for the phase with the given parity.  Returns false when it gave up.
 // SLEEP: back off with nanosleep after a few polls (for waits that are long while other warps of the
 // CTA need the issue slots); without it the wait is the hardware's own suspending try_wait in a loop.
+// limit_ns: how long the wait may last (measured from its first check of the clock, about a thousand polls in).
 template <bool SLEEP = true>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
   unsigned long long t0 = 0;
   for (unsigned it = 0;; ++it) {
     uint32_t done;
@@ -44,9 +46,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) return false;
+      else if (now - t0 > limit_ns) return false;
     }
   }
+}
+
+// Used on the give-up path only: lets TMA copies that are still in flight towards this CTA's shared memory
+// land before the CTA leaves (a copy takes microseconds; nothing can be awaited when the barrier that
+// counts it lives in the peer CTA or will never complete).
+__device__ __forceinline__ void drain_sleep(unsigned long long ns) {
+  const unsigned long long t0 = globaltimer();
+  while (globaltimer() - t0 < ns) __nanosleep(1000);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {

@@ -23,7 +23,9 @@ CAT_LS, CAT_FS, CAT_LS_GT1, CAT_FS_GT1 = 0, 1, 2, 3
 MODEL_MLP, MODEL_VIT, MODEL_DECODER = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 EPI_BIAS, EPI_GELU, EPI_SWIGLU, EPI_RESID_F32 = 1, 2, 4, 8
-K_NAMES = ["gather", "norm", "gemm", "rope", "attn_dec", "attn_combine", "attn_enc", "assemble", "output"]
+K_NAMES = ["gather", "norm", "gemm", "rope", "attn_dec", "attn_combine", "attn_enc", "assemble", "output", "gemm_stream", "trace"]
+ERR_PAGE_APPEND, ERR_PAGE_ATTEND, ERR_SELFTEST_WAIT = 101, 102, 90
+DECODE_STATUS_OFFSET = 192
 K_COUNT = len(K_NAMES)
 
 
@@ -38,7 +40,7 @@ class ModelDesc(C.Structure):
                 ("n_kv_heads", C.c_int), ("head_dim", C.c_int), ("ffn", C.c_int), ("vocab", C.c_int),
                 ("img", C.c_int), ("patch", C.c_int), ("mlp_dims", C.POINTER(C.c_int)),
                 ("tensors", C.POINTER(C.c_void_p)), ("n_tensors", C.c_int), ("kv_pool", C.c_void_p),
-                ("kv_pages", C.c_longlong), ("max_kv_len", C.c_int), ("max_batch", C.c_int)]
+                ("kv_pages", C.c_longlong), ("max_kv_len", C.c_int), ("max_batch", C.c_int), ("trace", C.c_void_p)]
 
 
 class Inputs(C.Structure):
@@ -50,12 +52,13 @@ class Inputs(C.Structure):
 class StepInfo(C.Structure):
     _fields_ = [("step_id", C.c_uint64), ("admitted", C.c_int * 2), ("dropped", C.c_int * 2),
                 ("launches", C.c_int), ("gemm_groups", C.c_int), ("gemm_flops", C.c_double),
-                ("weight_bytes", C.c_double), ("kv_bytes", C.c_double), ("device_error", C.c_int)]
+                ("weight_bytes", C.c_double), ("kv_bytes", C.c_double), ("stream_gemm_flops", C.c_double),
+                ("stream_weight_bytes", C.c_double)]
 
 
 class Output(C.Structure):
     _fields_ = [("status", C.c_int), ("step_id", C.c_uint64), ("logits", C.c_void_p), ("n_out", C.c_int),
-                ("argmax", C.c_void_p)]
+                ("argmax", C.c_void_p), ("device_error", C.c_int)]
 
 
 class GemmProblem(C.Structure):
@@ -68,7 +71,8 @@ EXPORTS = ["epara_init", "epara_register_model", "epara_submit", "epara_submit_m
            "epara_step_profile", "epara_set_profile", "epara_destroy", "epara_strerror", "epara_model_workspace_bytes",
            "epara_dp_group_count", "epara_inter_request_count", "epara_admit_queue", "epara_grouped_gemm",
            "epara_gemm_scratch_bytes", "epara_gemm_scratch_bytes_for", "epara_decode_attention", "epara_decode_attention_scratch_bytes",
-           "epara_decode_attention_static", "epara_static_scratch_bytes"]
+           "epara_decode_attention_static", "epara_static_scratch_bytes", "epara_decode_attention_static_status",
+           "epara_set_max_profile_launches", "epara_selftest_bounded_wait"]
 
 lib.epara_init.argtypes = [C.POINTER(Config), C.POINTER(C.c_void_p)]
 lib.epara_register_model.argtypes = [C.c_void_p, C.POINTER(ModelDesc), C.POINTER(C.c_int)]
@@ -93,18 +97,21 @@ lib.epara_grouped_gemm.argtypes = [C.c_int, C.c_void_p, C.c_int, C.POINTER(GemmP
                                    C.c_size_t]
 lib.epara_gemm_scratch_bytes.argtypes = [C.c_int]
 lib.epara_gemm_scratch_bytes.restype = C.c_size_t
-lib.epara_gemm_scratch_bytes_for.argtypes = [C.POINTER(GemmProblem), C.c_int]
+lib.epara_gemm_scratch_bytes_for.argtypes = [C.c_int, C.POINTER(GemmProblem), C.c_int]
 lib.epara_gemm_scratch_bytes_for.restype = C.c_size_t
-lib.epara_decode_attention.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+lib.epara_decode_attention.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_longlong, C.c_void_p,
                                        C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                        C.c_int, C.c_void_p, C.c_size_t]
 lib.epara_decode_attention_scratch_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
 lib.epara_decode_attention_scratch_bytes.restype = C.c_size_t
 
 
-lib.epara_decode_attention_static.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
-                                              C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
-                                              C.c_int]
+lib.epara_decode_attention_static.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_longlong,
+                                              C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                              C.c_int, C.c_int]
+lib.epara_decode_attention_static_status.argtypes = [C.c_int, C.POINTER(C.c_int)]
+lib.epara_set_max_profile_launches.argtypes = [C.c_void_p, C.c_int]
+lib.epara_selftest_bounded_wait.argtypes = [C.c_int, C.c_void_p, C.c_ulonglong, C.c_void_p, C.POINTER(C.c_int)]
 lib.epara_static_scratch_bytes.argtypes = []
 lib.epara_static_scratch_bytes.restype = C.c_size_t
 
@@ -166,8 +173,9 @@ def model_tensors(p: Dict) -> List:
     raise ValueError(k)
 
 
-def make_model_desc(p: Dict, kv_pool=None, max_kv_len: int = 0, max_batch: int = 0):
-    """Returns (ModelDesc, keepalive) for a synth model whose tensors live on the device."""
+def make_model_desc(p: Dict, kv_pool=None, max_kv_len: int = 0, max_batch: int = 0, kv_pages: int = 0, trace=None):
+    """Returns (ModelDesc, keepalive) for a synth model whose tensors live on the device.
+    kv_pages: pages per layer the library may touch (default: all of kv_pool's)."""
     tensors = model_tensors(p)
     for t in tensors:
         assert t.is_cuda and t.is_contiguous()
@@ -187,8 +195,12 @@ def make_model_desc(p: Dict, kv_pool=None, max_kv_len: int = 0, max_batch: int =
     else:
         d.kind, d.n_layers, d.d, d.n_heads = MODEL_DECODER, p["n_layers"], p["d"], p["n_q_heads"]
         d.n_kv_heads, d.head_dim, d.ffn, d.vocab = p["n_kv_heads"], p["head_dim"], p["ffn"], p["vocab"]
-        d.kv_pool, d.kv_pages, d.max_kv_len = kv_pool.data_ptr(), kv_pool.shape[1], max_kv_len
+        d.kv_pool, d.kv_pages, d.max_kv_len = kv_pool.data_ptr(), kv_pages or kv_pool.shape[1], max_kv_len
         keep.append(kv_pool)
+        if trace is not None:
+            assert trace.is_cuda and trace.dtype.itemsize == 4 and trace.numel() >= (p["n_layers"] + 1) * max(max_batch, 1) * p["d"]
+            d.trace = trace.data_ptr()
+            keep.append(trace)
     return d, keep
 
 
@@ -271,8 +283,8 @@ def gemm_problem_array(problems: Sequence[Dict]):
     return arr
 
 
-def epara_gemm_scratch_bytes_for(problems: Sequence[Dict]) -> int:
-    return lib.epara_gemm_scratch_bytes_for(gemm_problem_array(problems), len(problems))
+def epara_gemm_scratch_bytes_for(problems: Sequence[Dict], device: int = 0) -> int:
+    return lib.epara_gemm_scratch_bytes_for(device, gemm_problem_array(problems), len(problems))
 
 
 def epara_grouped_gemm(problems: Sequence[Dict], stream_ptr: int, scratch, impl: int = GEMM_TCGEN05, device: int = 0):
@@ -284,20 +296,35 @@ def epara_grouped_gemm(problems: Sequence[Dict], stream_ptr: int, scratch, impl:
 
 
 def epara_decode_attention(q, kv_layer, kv_lens, tables, out, Hq: int, Hkv: int, hd: int, max_len: int, scratch,
-                           stream_ptr: int, device: int = 0):
+                           stream_ptr: int, device: int = 0, kv_pages: int = 0):
+    """kv_pages: pages of kv_layer the call may touch (default: all of the tensor's)."""
     B = q.shape[0]
     _check(lib.epara_decode_attention(device, C.c_void_p(stream_ptr), q.data_ptr(), q.stride(0), kv_layer.data_ptr(),
-                                      kv_lens.data_ptr(), tables.data_ptr(), tables.stride(0), out.data_ptr(), B, Hq,
+                                      kv_pages or kv_layer.shape[0], kv_lens.data_ptr(), tables.data_ptr(), tables.stride(0), out.data_ptr(), B, Hq,
                                       Hkv, hd, max_len, scratch.data_ptr(),
                                       scratch.numel() * scratch.element_size()), "epara_decode_attention")
 
 
 def epara_decode_attention_static(q, kv_layer, kv_lens, tables, out, Hq: int, Hkv: int, hd: int, max_len: int,
-                                  stream_ptr: int, device: int = 0):
+                                  stream_ptr: int, device: int = 0, kv_pages: int = 0):
     """Decode attention for callers that must not allocate: same arguments as epara_decode_attention
     without the scratch tensor (the library's built-in per-GPU array is used instead)."""
     B = q.shape[0]
     _check(lib.epara_decode_attention_static(device, C.c_void_p(stream_ptr), q.data_ptr(), q.stride(0),
-                                             kv_layer.data_ptr(), kv_lens.data_ptr(), tables.data_ptr(),
-                                             tables.stride(0), out.data_ptr(), B, Hq, Hkv, hd, max_len),
+                                             kv_layer.data_ptr(), kv_pages or kv_layer.shape[0], kv_lens.data_ptr(),
+                                             tables.data_ptr(), tables.stride(0), out.data_ptr(), B, Hq, Hkv, hd,
+                                             max_len),
            "epara_decode_attention_static")
+
+
+def epara_decode_attention_static_status(device: int = 0):
+    """(status, code) of the last allocation-free decode-attention call on the device."""
+    code = C.c_int(0)
+    return lib.epara_decode_attention_static_status(device, C.byref(code)), code.value
+
+
+def epara_selftest_bounded_wait(status_dev, stream_ptr: int, limit_ns: int = 1_000_000, device: int = 0):
+    """(status, code): runs a wait that cannot complete for at most limit_ns; E_DEVICE / 90 is the expected answer."""
+    code = C.c_int(0)
+    s = lib.epara_selftest_bounded_wait(device, C.c_void_p(stream_ptr), limit_ns, status_dev.data_ptr(), C.byref(code))
+    return s, code.value

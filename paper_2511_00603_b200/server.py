@@ -23,11 +23,12 @@ class Server:
 
     # ------------------------------------------------------------- placement
     def add_model(self, p: Dict, kv_pool: Optional[torch.Tensor] = None, max_kv_len: int = 0,
-                  max_batch: int = 0) -> int:
+                  max_batch: int = 0, kv_pages: int = 0, trace: Optional[torch.Tensor] = None) -> int:
         """p: a synth model whose tensors are on this device.  Decoders are packed here."""
         if p["kind"] == "decoder" and "packed_layers" not in p:
             p["packed_layers"] = [synth.pack_decoder_layer(L) for L in p["layers"]]
-        desc, keep = E.make_model_desc(p, kv_pool=kv_pool, max_kv_len=max_kv_len, max_batch=max_batch)
+        desc, keep = E.make_model_desc(p, kv_pool=kv_pool, max_kv_len=max_kv_len, max_batch=max_batch, kv_pages=kv_pages,
+                                       trace=trace)
         mid = self.ctx.epara_register_model(desc, keep)
         n_out = p["dims"][-1] if p["kind"] == "mlp" else (p["n_cls"] if p["kind"] == "vit" else p["vocab"])
         self.models.append({"p": p, "n_out": n_out})

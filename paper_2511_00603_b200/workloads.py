@@ -20,15 +20,8 @@ import torch
 from . import epara as E
 from . import synth
 
-MLP_A = [512, 512, 512, 512, 10]
-VIT_S = dict(d=384, n_layers=12, n_heads=6, mlp=1536, n_cls=1000)
-VIT_B = dict(d=768, n_layers=12, n_heads=12, mlp=3072, n_cls=1000)
-DEC_1B = dict(d=2048, n_layers=16, n_q_heads=32, n_kv_heads=8, head_dim=64, ffn=8192, vocab=32000)
-DEC_8B = dict(d=4096, n_layers=32, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=14336, vocab=32000)
-
-# arrival rates (requests/s) of the 8 instances, fixed table
-MIXED_RATES = {"mlp": [2000.0, 1500.0, 1000.0], "vit": [500.0, 300.0, 200.0], "decoder": [100.0, 50.0]}
-LS_DEADLINE_NS = 20_000_000
+from .configs import (DEC_1B, DEC_8B, LS_DEADLINE_NS, MIXED_RATES, MLP_A, STRESS_DEC_BATCH, STRESS_KV_HI, STRESS_KV_LO,  # noqa: F401
+                      STRESS_VIT_BATCH, STRESS_VITS, VIT_B, VIT_S)
 
 
 class Instance:
@@ -144,9 +137,6 @@ def build_mixed(srv, seed: int = 3, ls_batch: int = 4, fs_batch: int = 256, kv_l
 
 
 # ------------------------------------------------------------------ stress step
-STRESS_VITS, STRESS_VIT_BATCH, STRESS_DEC_BATCH = 16, 32, 256
-STRESS_KV_LO, STRESS_KV_HI = 512, 8192
-
 
 def stress_bytes(kv_hi: int, n_vits: int = STRESS_VITS, vit_batch: int = STRESS_VIT_BATCH,
                  dec_batch: int = STRESS_DEC_BATCH, kv_lo: int = STRESS_KV_LO) -> Dict[str, float]:

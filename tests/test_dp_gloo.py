@@ -1,5 +1,6 @@
 """Two-rank CPU (gloo) test of the replica path: disjoint, complete sharding of requests, sticky
-decoder sequences, Eq. 4, and max-over-ranks throughput aggregation."""
+decoder sequences, Eq. 4, max-over-ranks throughput aggregation, and delivery in frame order of results
+that two replica processes produce at different speeds."""
 import os
 import socket
 
@@ -30,7 +31,27 @@ def _worker(rank, world, port, out):
     sticky_ok = all(dp.replica_of(r["stream"], r["frame"], world, True) == rank for r in mine if r["sticky"])
     # rank 0 takes 10 ms for its share, rank 1 takes 25 ms: the job ran at (n0 + n1) / 25 ms
     thr = dp.whole_job_throughput(len(mine), 10.0 if rank == 0 else 25.0)
-    out.put((rank, len(mine), bool((ids == 1).all()), sticky_ok, thr))
+    # ordered delivery across processes: every rank "serves" its frames (rank 1 reports them in reverse, as a
+    # slower replica would), rank 0 merges the reports through the reorder buffer
+    done = [(r["stream"], r["frame"], r["id"] * 3) for r in mine]
+    if rank == 1:
+        done.reverse()
+    reports = [None] * world
+    dist.all_gather_object(reports, done)
+    ordered_ok = True
+    if rank == 0:
+        od = dp.OrderedDelivery()
+        released = []
+        for i in range(max(len(x) for x in reports)):
+            for rep in reports:
+                if i < len(rep):
+                    released += od.put(*rep[i])
+        per = {}
+        for s, f, val in released:
+            per.setdefault(s, []).append(f)
+            ordered_ok = ordered_ok and val == (f * 5 + s) * 3
+        ordered_ok = ordered_ok and len(released) == 100 and all(per[s] == list(range(20)) for s in range(5))
+    out.put((rank, len(mine), bool((ids == 1).all()), sticky_ok and ordered_ok, thr))
     dist.destroy_process_group()
 
 

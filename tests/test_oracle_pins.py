@@ -94,6 +94,27 @@ def test_gelu_values():
     assert np.allclose(O.gelu(x.numpy()), torch.nn.functional.gelu(x).numpy(), atol=1e-15)
 
 
+def test_device_gelu_formula_stays_within_its_stated_bound_of_the_erf_form():
+    """The CUDA epilogue evaluates GELU as 0.5 x (1 + tanh(x P(x^2))), P(t) = a + b t + c t^2 with t clamped at
+    64 (csrc/common.cuh).  With an exact tanh that formula is within 2.6e-5 of the erf form for every x; the
+    coefficients are read from the source file, so a change there is checked here."""
+    import os
+    import re
+    src = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2511_00603_b200", "csrc",
+                            "common.cuh")).read()
+    body = src[src.index("float gelu_erf(float x)"):]
+    body = body[:body.index("silu_f")]
+    c2, c1 = [float(v) for v in re.search(r"fmaf\(t, (-?[0-9.e+-]+)f, (-?[0-9.e+-]+)f\)", body).groups()]
+    c0 = float(re.search(r"fmaf\(t, p, (-?[0-9.e+-]+)f\)", body).group(1))
+    assert abs(c0 - math.sqrt(2 / math.pi)) < 1e-3            # leading term of erf(x / sqrt 2) ~ tanh(sqrt(2/pi) x)
+    x = np.linspace(-12.0, 12.0, 480001)
+    t = np.minimum(x * x, 64.0)
+    dev = 0.5 * x * (1.0 + np.tanh(x * (c0 + t * (c1 + t * c2))))
+    err = np.abs(dev - O.gelu(x))
+    assert err.max() <= 2.6e-5, err.max()
+    assert err[np.abs(x) > 8].max() <= 1e-10                  # saturated on both sides: x or 0
+
+
 def test_silu_values():
     assert abs(O.silu(np.array([1.0]))[0] - 1.0 / (1.0 + math.exp(-1.0))) < 1e-16
     x = torch.linspace(-8, 8, 77, dtype=torch.float64)
@@ -217,25 +238,31 @@ def test_patchify_index_rule():
     assert np.array_equal(P, ref)
 
 
-def _torch_vit(img, p):
+def _torch_bf16(t):
+    """Storage rounding by the library's own bf16 cast (fp64 -> fp32 -> bf16 -> fp64)."""
+    return t.float().to(torch.bfloat16).double()
+
+
+def _torch_vit(img, p, rnd=lambda t: t):
     """Independent fp64 evaluation with torch library routines (conv patch embedding,
-    layer_norm, scaled_dot_product_attention, gelu)."""
+    layer_norm, scaled_dot_product_attention, gelu).  rnd is applied to every tensor the device
+    contract stores as bf16 (identity: the unrounded evaluation)."""
     F = torch.nn.functional
     f = lambda t: t.double()
     d, H, ps = p["d"], p["n_heads"], p["patch"]
-    x = F.conv2d(f(img)[None], f(p["W_pe"]).reshape(d, 3, ps, ps), f(p["b_pe"]), stride=ps)
+    x = rnd(F.conv2d(f(img)[None], f(p["W_pe"]).reshape(d, 3, ps, ps), f(p["b_pe"]), stride=ps))
     x = x.flatten(2).transpose(1, 2)
     z = torch.cat([f(p["cls"])[None, None], x], dim=1) + f(p["pos"])[None]
     T = z.shape[1]
     for L in p["layers"]:
-        h = F.layer_norm(z, (d,), f(L["ln1_g"]), f(L["ln1_b"]), eps=1e-6)
-        qkv = F.linear(h, f(L["Wqkv"]), f(L["bqkv"])).reshape(1, T, 3, H, d // H).permute(2, 0, 3, 1, 4)
-        o = F.scaled_dot_product_attention(qkv[0], qkv[1], qkv[2]).transpose(1, 2).reshape(1, T, d)
+        h = rnd(F.layer_norm(z, (d,), f(L["ln1_g"]), f(L["ln1_b"]), eps=1e-6))
+        qkv = rnd(F.linear(h, f(L["Wqkv"]), f(L["bqkv"]))).reshape(1, T, 3, H, d // H).permute(2, 0, 3, 1, 4)
+        o = rnd(F.scaled_dot_product_attention(qkv[0], qkv[1], qkv[2]).transpose(1, 2).reshape(1, T, d))
         z = z + F.linear(o, f(L["Wo"]), f(L["bo"]))
-        h = F.layer_norm(z, (d,), f(L["ln2_g"]), f(L["ln2_b"]), eps=1e-6)
-        z = z + F.linear(F.gelu(F.linear(h, f(L["W1"]), f(L["b1"]))), f(L["W2"]), f(L["b2"]))
-    c = F.layer_norm(z[0, 0], (d,), f(p["lnf_g"]), f(p["lnf_b"]), eps=1e-6)
-    return F.linear(c, f(p["Whead"]), f(p["bhead"])).numpy()
+        h = rnd(F.layer_norm(z, (d,), f(L["ln2_g"]), f(L["ln2_b"]), eps=1e-6))
+        z = z + F.linear(rnd(F.gelu(F.linear(h, f(L["W1"]), f(L["b1"])))), f(L["W2"]), f(L["b2"]))
+    c = rnd(F.layer_norm(z[0, 0], (d,), f(p["lnf_g"]), f(p["lnf_b"]), eps=1e-6))
+    return rnd(F.linear(c, f(p["Whead"]), f(p["bhead"]))).numpy()
 
 
 def test_vit_matches_torch_library_evaluation():
@@ -262,9 +289,10 @@ def _pool_fetch(pool_bits):
     return lambda layer, page: pool_bits[layer, page]
 
 
-def _torch_decoder(token, L, table, pool, p):
+def _torch_decoder(token, L, table, pool, p, rnd=lambda t: t):
     """Independent fp64 evaluation: contiguous K/V rebuilt with torch indexing, complex-number
-    RoPE, library rms_norm / sdpa / silu."""
+    RoPE, library rms_norm / sdpa / silu.  rnd is applied to every tensor the device contract stores
+    as bf16 (identity: the unrounded evaluation)."""
     F = torch.nn.functional
     f = lambda t: t.double()
     Hq, Hkv, hd = p["n_q_heads"], p["n_kv_heads"], p["head_dim"]
@@ -278,20 +306,20 @@ def _torch_decoder(token, L, table, pool, p):
 
     tb = torch.as_tensor(table.astype(np.int64))
     for li, Lw in enumerate(p["layers"]):
-        h = F.rms_norm(x, (p["d"],), f(Lw["g1"]), eps=1e-5)
-        q = rope(F.linear(h, f(Lw["Wq"])).reshape(Hq, hd))
-        k = rope(F.linear(h, f(Lw["Wk"])).reshape(Hkv, hd))
-        v = F.linear(h, f(Lw["Wv"])).reshape(Hkv, hd)
+        h = rnd(F.rms_norm(x, (p["d"],), f(Lw["g1"]), eps=1e-5))
+        q = rnd(rope(rnd(F.linear(h, f(Lw["Wq"]))).reshape(Hq, hd)))
+        k = rnd(rope(rnd(F.linear(h, f(Lw["Wk"]))).reshape(Hkv, hd)))
+        v = rnd(F.linear(h, f(Lw["Wv"]))).reshape(Hkv, hd)
         pages = f(pool[li][tb])                               # [n, 2, Hkv, 16, hd]
         Kc = pages[:, 0].permute(1, 0, 2, 3).reshape(Hkv, -1, hd)[:, :L]
         Vc = pages[:, 1].permute(1, 0, 2, 3).reshape(Hkv, -1, hd)[:, :L]
         K = torch.cat([Kc, k[:, None]], dim=1).repeat_interleave(Hq // Hkv, dim=0)
         V = torch.cat([Vc, v[:, None]], dim=1).repeat_interleave(Hq // Hkv, dim=0)
-        o = F.scaled_dot_product_attention(q[:, None], K, V).reshape(-1)
+        o = rnd(F.scaled_dot_product_attention(q[:, None], K, V).reshape(-1))
         x = x + F.linear(o, f(Lw["Wo"]))
-        h = F.rms_norm(x, (p["d"],), f(Lw["g2"]), eps=1e-5)
-        x = x + F.linear(F.silu(F.linear(h, f(Lw["Wg"]))) * F.linear(h, f(Lw["Wu"])), f(Lw["Wd"]))
-    return F.linear(F.rms_norm(x, (p["d"],), f(p["gf"]), eps=1e-5), f(p["Wlm"])).numpy()
+        h = rnd(F.rms_norm(x, (p["d"],), f(Lw["g2"]), eps=1e-5))
+        x = x + F.linear(rnd(F.silu(F.linear(h, f(Lw["Wg"]))) * F.linear(h, f(Lw["Wu"]))), f(Lw["Wd"]))
+    return rnd(F.linear(rnd(F.rms_norm(x, (p["d"],), f(p["gf"]), eps=1e-5)), f(p["Wlm"]))).numpy()
 
 
 def _small_decoder(seed=11, perturb=0.2):
@@ -372,11 +400,52 @@ def test_decoder_paging_invariance_and_gqa():
     assert np.array_equal(base["logits"], r4["logits"])
 
 
-def test_gqa_equal_query_heads_give_equal_outputs():
-    rng = np.random.default_rng(6)
-    K, V = rng.normal(size=(9, 8)), rng.normal(size=(9, 8))
-    q = rng.normal(size=8)
-    assert np.array_equal(O.attention(q, K, V), O.attention(q.copy(), K, V))
+def test_gqa_query_heads_read_their_groups_kv_head():
+    """GQA against a model without it: the decoder with 4 query heads over 2 KV heads must equal the
+    multi-head decoder (4 KV heads) whose K and V projections and cache hold, for query head h, a copy of
+    KV head h // 2.  A wrong head-to-group mapping (h % 2, say) fails: the two KV heads differ."""
+    p = _small_decoder(seed=23)
+    toks, lens, tables, npages = synth.make_decode_batch(2, 20, 45, 50, seed=24)
+    pool = synth.make_kv_pool(2, npages, 2, 16, seed=25)
+    wide = {k: v for k, v in p.items()}
+    wide["n_kv_heads"] = 4
+    wide["layers"] = []
+    for L in p["layers"]:
+        W = dict(L)
+        for name in ("Wk", "Wv"):
+            W[name] = L[name].reshape(2, 16, -1).repeat_interleave(2, dim=0).reshape(64, -1).contiguous()
+        wide["layers"].append(W)
+    pool_wide = pool.repeat_interleave(2, dim=3).contiguous()          # [layer, page, 2, Hkv -> 4, 16, hd]
+    for i in range(2):
+        a = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], _pool_fetch(synth.to_bits(pool)), synth.bits_view(p))
+        b = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], _pool_fetch(synth.to_bits(pool_wide)), synth.bits_view(wide))
+        assert np.allclose(a["logits"], b["logits"], rtol=1e-12, atol=1e-14)
+        # and the mapping matters for this input: swapping the two KV heads changes the answer
+        swapped = synth.to_bits(pool.flip(3).contiguous())
+        c = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], _pool_fetch(swapped), synth.bits_view(p))
+        assert np.max(np.abs(a["logits"] - c["logits"])) > 1e-3
+
+
+def test_bf16_storage_mode_matches_torch_evaluation_with_library_casts():
+    """Mode B (bf16 rounding at the device contract's storage points) is what the decoder parity tests
+    compare with.  It is pinned against the independent torch evaluation with the library's own bf16 cast at
+    those points: norm outputs, q / k / v before and after the rotation, attention output, SwiGLU output,
+    logits; the residual stream stays unrounded.  (An evaluation that rounded somewhere else, or not at all,
+    differs by about 1e-3 relative; agreement here is to 1e-9.)"""
+    p = _small_decoder(seed=26)
+    toks, lens, tables, npages = synth.make_decode_batch(3, 5, 40, 50, seed=27)
+    pool = synth.make_kv_pool(2, npages, 2, 16, seed=28)
+    pb = synth.to_bits(pool)
+    for i in range(3):
+        r = O.decoder_step(int(toks[i]), int(lens[i]), tables[i], _pool_fetch(pb), synth.bits_view(p), round_bf16=True)
+        ref = _torch_decoder(int(toks[i]), int(lens[i]), tables[i], pool, p, rnd=_torch_bf16)
+        assert np.allclose(r["logits"], ref, rtol=1e-9, atol=1e-12)
+        unrounded = _torch_decoder(int(toks[i]), int(lens[i]), tables[i], pool, p)
+        assert np.max(np.abs(unrounded - ref)) > 1e-5
+    pv = synth.make_vit(d=64, n_layers=2, n_heads=4, mlp=128, n_cls=10, seed=29, img=64, std=0.2, perturb=0.3)
+    img = synth.make_images(1, seed=30, img=64)[0]
+    logits, am, _ = O.vit_forward(synth.to_bits(img), synth.bits_view(pv), round_bf16=True)
+    assert np.allclose(logits, _torch_vit(img, pv, rnd=_torch_bf16), rtol=1e-9, atol=1e-12)
 
 
 def test_mode_b_is_close_to_mode_a():
@@ -387,6 +456,31 @@ def test_mode_b_is_close_to_mode_a():
     b = O.decoder_step(int(toks[0]), 30, tables[0], _pool_fetch(pool), synth.bits_view(p), round_bf16=True)["logits"]
     rho = math.sqrt(np.mean(a * a))
     assert 0 < np.max(np.abs(a - b)) < 2e-2 * rho
+
+
+@pytest.mark.parametrize("n_layers,l2_lo,l2_hi,max_hi", [(1, 2e-3, 1.2e-2, 5e-2), (2, 3e-3, 1.5e-2, 6e-2), (16, 8e-3, 4e-2, 1.5e-1)])
+def test_mode_a_vs_mode_b_gap_at_the_1b_layer_shapes(n_layers, l2_lo, l2_hi, max_hi):
+    """How far apart two correct evaluations of one decode request are at the 1B decoder's layer shapes
+    (d 2048, 32 / 8 heads of 64, FFN 8192, vocab 32000): the unrounded fp64 evaluation against the one that
+    rounds to bf16 at the storage points.  This gap, not a kernel, is why a deep random-weight decoder
+    cannot meet 2e-2 element-wise against the unrounded evaluation; the GPU tests bound the device by a
+    fraction of each request's own gap and rely on the ceilings checked here.  Measured (seed 2, KV length
+    600): relative L2 5.9e-3 / 7.3e-3 / 1.8e-2 and worst element 2.5e-2 / 2.9e-2 / 7.9e-2 of the tensor's
+    scale at 1 / 2 / 16 layers."""
+    from paper_2511_00603_b200 import configs
+    from tests.parity import DEEP_GAP_L2_CEIL, DEEP_GAP_MAX_CEIL, max_rel_err, rel_l2_err
+    cfg = dict(configs.DEC_1B, n_layers=n_layers)
+    p = synth.bits_view(synth.make_decoder(seed=2, **cfg))
+    toks, lens, tables, npages = synth.make_decode_batch(1, 600, 600, cfg["vocab"], seed=31)
+    pool = synth.to_bits(synth.make_kv_pool(n_layers, npages, cfg["n_kv_heads"], cfg["head_dim"], seed=32))
+    a = O.decoder_step(int(toks[0]), 600, tables[0], _pool_fetch(pool), p)["logits"]
+    b = O.decoder_step(int(toks[0]), 600, tables[0], _pool_fetch(pool), p, round_bf16=True)["logits"]
+    l2, mx = rel_l2_err(a, b), max_rel_err(a, b)
+    print(f"1B layer shapes, {n_layers} layers: mode A vs mode B relative L2 {l2:.3e}, max relative {mx:.3e}")
+    assert l2_lo <= l2 <= l2_hi and mx <= max_hi
+    assert l2 <= DEEP_GAP_L2_CEIL and mx <= DEEP_GAP_MAX_CEIL
+    if n_layers >= 2:
+        assert mx > 2e-2          # the strict element-wise reading is out of reach for any implementation
 
 
 # ------------------------------------------------------------------- host policy

@@ -65,7 +65,8 @@ def test_static_scratch_entry_rejects_what_does_not_fit(E):
     q, pool, lens_d, tabs_d, max_len = _case(E, 2, [30, 50], 8, 2, 64, 90)
     out = torch.empty_like(q)
     # claim a batch and length whose partials need far more than the built-in array holds
-    s = E.lib.epara_decode_attention_static(0, stream, q.data_ptr(), q.stride(0), pool.data_ptr(), lens_d.data_ptr(),
-                                            tabs_d.data_ptr(), tabs_d.stride(0), out.data_ptr(), 4096, 32, 8, 64, 8192)
+    s = E.lib.epara_decode_attention_static(0, stream, q.data_ptr(), q.stride(0), pool.data_ptr(), pool.shape[0],
+                                            lens_d.data_ptr(), tabs_d.data_ptr(), tabs_d.stride(0), out.data_ptr(), 4096, 32,
+                                            8, 64, 8192)
     assert s == E.E_RESOURCE
-    assert E.lib.epara_decode_attention_static(0, stream, None, 0, None, None, None, 0, None, 1, 8, 2, 64, 16) == E.E_INVALID
+    assert E.lib.epara_decode_attention_static(0, stream, None, 0, None, 1, None, None, 0, None, 1, 8, 2, 64, 16) == E.E_INVALID
