@@ -26,7 +26,8 @@ Parity pins (tests/test_oracle_pins.py): brute-force tiny matmuls, identity weig
 zero inputs, single-token attention equals V, uniform attention equals mean(V),
 norm closed forms, RoPE relative-position property, GQA and paging invariances,
 softmax shift invariance and split/merge, cross-check of every family against an
-independent fp64 torch evaluation.  The host-logic functions (admission, Eq. 4,
+independent fp64 torch evaluation; the prefill against successive decode steps on a growing
+cache, a causal torch evaluation, and causality itself (a later token cannot change an earlier one).  The host-logic functions (admission, Eq. 4,
 Eq. 5, goodput rule) are pinned by the paper's worked example (120 frames,
 60 fps required, 30 fps achieved -> 60 satisfied) and by hand-computed cases.
 No function here is "parity unpinned".
@@ -272,6 +273,52 @@ def decoder_step(token: int, kv_len: int, table: np.ndarray,
         residual.append(x)
         appended.append({"k": k, "v": v, "page": int(table[kv_len // PAGE]), "slot": kv_len % PAGE})
     logits = decoder_head(x, p, round_bf16)
+    return {"logits": logits, "argmax": argmax_lowest(logits), "appended": appended, "residual": residual}
+
+
+def decoder_prefill(tokens: Sequence[int], kv_len: int, table: np.ndarray,
+                    fetch_page: Callable[[int, int], np.ndarray], p: Dict,
+                    round_bf16: bool = False) -> Dict:
+    """A prompt chunk of n tokens through a Llama-style decoder (the prefill phase of an LLM request,
+    Section 4.3; with kv_len > 0 it is one chunk of a chunked prefill).
+
+    Token t of the chunk sits at position kv_len + t.  In every layer each token gets its own q, k, v
+    (rotated at its own position); its k, v go to cache slot kv_len + t; its query attends causally:
+    over the cached positions 0 .. kv_len - 1 and the chunk's tokens 0 .. t.  Everything else is
+    token-wise, exactly as in decoder_layer.  With n = 1 this is decoder_step.
+    Returns the last token's logits and argmax, per layer the chunk's appended k and v
+    (fp64 [n, Hkv, hd]), and the residual stream after the embedding and after every layer ([n, d] each).
+    """
+    D = bf16_to_f64
+    Hq, Hkv, hd = int(p["n_q_heads"]), int(p["n_kv_heads"]), int(p["head_dim"])
+    grp = Hq // Hkv
+    n = len(tokens)
+    X = np.stack([D(p["Emb"][int(t)]) for t in tokens])
+    appended = []
+    residual = [X]
+    for li, L in enumerate(p["layers"]):
+        H = _store(rmsnorm(X, D(L["g1"])), round_bf16)
+        Q = _store(linear(H, D(L["Wq"])), round_bf16).reshape(n, Hq, hd)
+        K = _store(linear(H, D(L["Wk"])), round_bf16).reshape(n, Hkv, hd)
+        V = _store(linear(H, D(L["Wv"])), round_bf16).reshape(n, Hkv, hd)
+        Q = np.stack([_store(rope(Q[t], kv_len + t), round_bf16) for t in range(n)])
+        K = np.stack([_store(rope(K[t], kv_len + t), round_bf16) for t in range(n)])
+        Kc, Vc = gather_kv(fetch_page, li, table, kv_len)
+        Oa = np.empty((n, Hq, hd))
+        for t in range(n):
+            for hq in range(Hq):
+                g = hq // grp
+                Kh = K[:t + 1, g] if Kc is None else np.concatenate([Kc[g], K[:t + 1, g]], axis=0)
+                Vh = V[:t + 1, g] if Vc is None else np.concatenate([Vc[g], V[:t + 1, g]], axis=0)
+                Oa[t, hq] = attention(Q[t, hq], Kh, Vh)
+        Oa = _store(Oa.reshape(n, -1), round_bf16)
+        X = X + linear(Oa, D(L["Wo"]))
+        H = _store(rmsnorm(X, D(L["g2"])), round_bf16)
+        F = _store(silu(linear(H, D(L["Wg"]))) * linear(H, D(L["Wu"])), round_bf16)
+        X = X + linear(F, D(L["Wd"]))
+        residual.append(X)
+        appended.append({"k": K, "v": V})
+    logits = decoder_head(X[n - 1], p, round_bf16)
     return {"logits": logits, "argmax": argmax_lowest(logits), "appended": appended, "residual": residual}
 
 

@@ -483,6 +483,94 @@ def test_mode_a_vs_mode_b_gap_at_the_1b_layer_shapes(n_layers, l2_lo, l2_hi, max
         assert mx > 2e-2          # the strict element-wise reading is out of reach for any implementation
 
 
+# ------------------------------------------------------------------- prefill
+class _GrowingCache:
+    """A paged cache as bf16 bits that decode steps append to: fetch(layer, page) serves the oracle."""
+
+    def __init__(self, pool_bits):
+        self.pool = pool_bits.copy()
+
+    def fetch(self, layer, page):
+        return self.pool[layer, page]
+
+    def append(self, layer, page, slot, k, v):
+        self.pool[layer, page, 0, :, slot, :] = O.f64_to_bf16_bits(k)
+        self.pool[layer, page, 1, :, slot, :] = O.f64_to_bf16_bits(v)
+
+
+def test_prefill_equals_successive_decode_steps_on_a_growing_cache():
+    """The identity that defines prefill: feeding the chunk's tokens one at a time through decoder_step, each
+    step's k, v stored in the cache before the next, gives the same appended k, v, residuals and final
+    logits.  With bf16 storage (mode B) the cache holds exactly what was appended, so the identity is exact
+    up to summation order; both a fresh prompt (kv_len 0) and a chunk after 21 cached tokens."""
+    p = synth.bits_view(_small_decoder(seed=40))
+    for kv0, n in [(0, 9), (21, 14)]:
+        toks, lens, tables, npages = synth.make_decode_batch(1, kv0 + n, kv0 + n, 50, seed=41 + kv0)
+        pool = synth.to_bits(synth.make_kv_pool(2, npages, 2, 16, seed=42))
+        tokens = [int(t) for t in np.random.default_rng(43).integers(0, 50, n)]
+        pre = O.decoder_prefill(tokens, kv0, tables[0], _pool_fetch(pool), p, round_bf16=True)
+        cache = _GrowingCache(pool)
+        for t, tok in enumerate(tokens):
+            r = O.decoder_step(tok, kv0 + t, tables[0], cache.fetch, p, round_bf16=True)
+            for l, ap in enumerate(r["appended"]):
+                assert np.allclose(ap["k"], pre["appended"][l]["k"][t], rtol=1e-12, atol=1e-14)
+                assert np.allclose(ap["v"], pre["appended"][l]["v"][t], rtol=1e-12, atol=1e-14)
+                cache.append(l, ap["page"], ap["slot"], ap["k"], ap["v"])
+            for l in range(3):
+                assert np.allclose(r["residual"][l], pre["residual"][l][t], rtol=1e-11, atol=1e-13)
+        assert np.allclose(r["logits"], pre["logits"], rtol=1e-11, atol=1e-13)
+        assert r["argmax"] == pre["argmax"]
+
+
+def test_prefill_is_causal_and_its_first_token_sees_only_itself():
+    p = synth.bits_view(_small_decoder(seed=44, perturb=0.0))
+    table = np.arange(2, dtype=np.int32)
+    nofetch = lambda l, pg: (_ for _ in ()).throw(AssertionError("no cached token exists"))
+    a = O.decoder_prefill([5, 17, 3, 8], 0, table, nofetch, p)
+    # changing a later token leaves every earlier token's k, v and residual untouched
+    b = O.decoder_prefill([5, 17, 30, 41], 0, table, nofetch, p)
+    for l in range(2):
+        assert np.array_equal(a["appended"][l]["k"][:2], b["appended"][l]["k"][:2])
+        assert np.array_equal(a["residual"][l + 1][:2], b["residual"][l + 1][:2])
+        assert not np.array_equal(a["residual"][l + 1][3], b["residual"][l + 1][3])
+    # the first token attends to itself only: its attention output is its own v (closed form, as for an empty cache)
+    one = O.decoder_step(5, 0, table, nofetch, p)
+    assert np.allclose(a["residual"][2][0], one["residual"][2], rtol=1e-13, atol=1e-15)
+    # and a prompt of one token is a decode step
+    assert np.array_equal(O.decoder_prefill([5], 0, table, nofetch, p)["logits"], one["logits"])
+
+
+def test_prefill_matches_a_causal_torch_evaluation():
+    """Independent route: all tokens at once with the library's causal scaled_dot_product_attention."""
+    F = torch.nn.functional
+    pt = _small_decoder(seed=45)
+    p = synth.bits_view(pt)
+    n, hd, Hq, Hkv, d = 11, 16, 4, 2, 64
+    tokens = [int(t) for t in np.random.default_rng(46).integers(0, 50, n)]
+    got = O.decoder_prefill(tokens, 0, np.arange(1, dtype=np.int32), None, p)
+    f = lambda t: t.double()
+    x = f(pt["Emb"][torch.tensor(tokens)])
+    pos = torch.arange(n, dtype=torch.float64)[:, None]
+    ang = pos * (10000.0 ** (-torch.arange(0, hd, 2, dtype=torch.float64) / hd))[None]
+    rot = torch.polar(torch.ones_like(ang), ang)[:, None, :]                       # [n, 1, hd/2]
+
+    def rope(t):                                                                  # t [n, H, hd]
+        c = torch.view_as_complex(t.reshape(n, -1, hd // 2, 2).contiguous()) * rot
+        return torch.view_as_real(c).reshape(n, -1, hd)
+
+    for Lw in pt["layers"]:
+        h = F.rms_norm(x, (d,), f(Lw["g1"]), eps=1e-5)
+        q = rope(F.linear(h, f(Lw["Wq"])).reshape(n, Hq, hd)).transpose(0, 1)
+        k = rope(F.linear(h, f(Lw["Wk"])).reshape(n, Hkv, hd)).transpose(0, 1).repeat_interleave(Hq // Hkv, dim=0)
+        v = F.linear(h, f(Lw["Wv"])).reshape(n, Hkv, hd).transpose(0, 1).repeat_interleave(Hq // Hkv, dim=0)
+        o = F.scaled_dot_product_attention(q, k, v, is_causal=True).transpose(0, 1).reshape(n, -1)
+        x = x + F.linear(o, f(Lw["Wo"]))
+        h = F.rms_norm(x, (d,), f(Lw["g2"]), eps=1e-5)
+        x = x + F.linear(F.silu(F.linear(h, f(Lw["Wg"]))) * F.linear(h, f(Lw["Wu"])), f(Lw["Wd"]))
+    ref = F.linear(F.rms_norm(x[-1], (d,), f(pt["gf"]), eps=1e-5), f(pt["Wlm"])).numpy()
+    assert np.allclose(got["logits"], ref, rtol=1e-10, atol=1e-12)
+
+
 # ------------------------------------------------------------------- host policy
 def test_eq4_eq5_and_goodput_example():
     assert O.dp_group_count(97, 49) == 2 and O.dp_group_count(98, 49) == 2 and O.dp_group_count(99, 49) == 3
