@@ -101,7 +101,9 @@ typedef struct {
   void* kv_pool;                /* device, decoder only */
   long long kv_pages;
   int max_kv_len;               /* decoder: longest cached length a request may have */
-  int max_batch;                /* rows reserved in the workspace (0 -> cap_ls + cap_fs) */
+  int max_batch;                /* rows reserved in the workspace (0 -> cap_ls + cap_fs): the most requests of a step;
+                                   for a decoder the most TOKENS of a step (a decode request is one, a prompt chunk
+                                   of n tokens is n); requests beyond it wait for the next step */
   void* trace;                  /* device, decoder only, may be NULL: when given, every step copies the model's
                                    residual stream into it after the embedding and after each layer, fp32
                                    [n_layers + 1][max_batch][d] (row = the request's place in its batch).  For
@@ -114,8 +116,15 @@ typedef struct {
   int token;                /* decoder: id of the token being decoded */
   int kv_len;               /* decoder: cached tokens L; the new token is written at slot L and
                                attention runs over L + 1 tokens */
-  const int32_t* block_table; /* device int32 [n_blocks], page ids; needs n_blocks >= L/16 + 1 */
+  const int32_t* block_table; /* device int32 [n_blocks], page ids; needs n_blocks >= (L + n - 1)/16 + 1 */
   int n_blocks;
+  const int32_t* tokens;    /* decoder, HOST, read during epara_submit only: with n_tokens = n > 1 the request is a
+                               prompt chunk (the prefill phase of an LLM request, Section 4.3): token t goes to
+                               position L + t, its k, v are appended there, and it attends causally to positions
+                               0 .. L + t.  L = 0 is a whole prompt, L > 0 a later chunk of a chunked prefill.
+                               The outputs are the LAST token's logits and argmax.  A chunk takes n of the model's
+                               max_batch rows and may share its step with decode requests.  Head sizes 64 and 128. */
+  int n_tokens;             /* 0 or 1: a decode request of `token` (or tokens[0] when given) */
   long long deadline_ns;    /* absolute time after which the request is dropped; 0 = none */
   long long arrival_ns;
   int stream;               /* frequency-sensitive stream id (MF groups frames per stream) */
@@ -134,6 +143,7 @@ typedef struct {
   double kv_bytes;          /* bytes of cached K/V the step reads */
   double stream_gemm_flops;   /* the part of gemm_flops in weight-streaming launches (groups of at most 16 rows) */
   double stream_weight_bytes; /* the part of weight_bytes in those launches */
+  int prefill_tokens;         /* tokens of the step's prompt chunks */
 } epara_step_info;
 
 typedef struct {
@@ -155,7 +165,8 @@ enum {
   EPARA_K_GEMM_STREAM = 9,  /* the weight-streaming GEMM launches (groups of at most 16 rows); EPARA_K_GEMM holds
                                the tensor-core launches */
   EPARA_K_TRACE = 10,       /* copies into epara_model_desc.trace */
-  EPARA_K_COUNT = 11
+  EPARA_K_ATTN_PREFILL = 11, /* causal attention of prompt chunks */
+  EPARA_K_COUNT = 12
 };
 
 /* Creates a context on cfg->device.  Returns INVALID (null/unaligned workspace), CUDA. */
@@ -223,6 +234,68 @@ int epara_inter_request_count(int bs, int mf_max);
 int epara_admit_queue(int n, const uint64_t* tickets, const long long* deadline_ns, const int* streams,
                       long long now_ns, int cap, int mf_max,
                       uint64_t* out_admitted, int* n_admitted, uint64_t* out_dropped, int* n_dropped);
+
+/* ---- host policies around the step (pure host code): request handling, placement, simulation ----
+ *
+ * Model.  Servers n = 0 .. n_servers-1 with gpus[n] identical GPUs; a GPU has compute capacity 1 (a service's MPS
+ * share `a` is a fraction of it) and `vram` GB.  Server index n_servers is the hypothetical server of Algorithm 1,
+ * stage 3: it owns no GPU and places an instance on free GPUs of any real servers.  A placement (service, server)
+ * is one instance; it takes n_gpus GPUs, first fit in (server, gpu) order, `a` and `b` on each.
+ * A service has a category (0 latency-, 1 frequency-sensitive), a batch size, a latency SLO per request or
+ * frame, for frequency-sensitive services the frame rate and the frames of a request (its frames arrive
+ * 1 / fps apart), and the profiled compute time c_ms[k] of a batch of up to 2^k requests (the c_ln table of
+ * Section 3.3, measured by the offline profiler of Section 4.1).
+ * A request reaches `server` at t_ms; u[] are pre-drawn uniform numbers in [0, 1), one per offloading decision. */
+#define EPARA_PROFILE_POINTS 10       /* batch sizes 2^0 .. 2^9 (Section 4.1) */
+#define EPARA_MAX_OFFLOAD_DRAWS 5     /* the default maximum offloading count (Section 4.1, Table 4) */
+typedef struct { int n_servers; const int* gpus; double vram; double sync_ms; double offload_ms; } epara_cluster;
+typedef struct {
+  double a, b;              /* compute share of a GPU, VRAM in GB, per GPU of an instance */
+  int n_gpus;               /* GPUs one instance spans (1 for the "<1 GPU" categories) */
+  int cat;                  /* 0 latency-sensitive, 1 frequency-sensitive */
+  int bs;                   /* batch size */
+  double slo_ms;            /* latency SLO of a request (or of one frame) */
+  double fps;               /* frequency-sensitive: required frame rate */
+  int frames;               /* frequency-sensitive: frames of one request */
+  double c_ms[EPARA_PROFILE_POINTS];
+} epara_service;
+typedef struct { double t_ms; int service; int server; double u[EPARA_MAX_OFFLOAD_DRAWS]; } epara_request;
+typedef struct { int service; int server; } epara_placement;
+typedef struct {
+  double phi;               /* Eq. 2: satisfied requests; a frequency-sensitive request of F frames counts
+                               F x achieved / required frame rate (Section 3.3), at most the frames in time */
+  int served, timeout, offload_exceed, insufficient, late, offloads, instances;   /* per work item (request or frame) */
+} epara_sim_result;
+
+/* Eq. 1: candidate m has idle goodput p_hat[m] - p_act[m] (theoretical minus actual goodput; negative counts
+ * as 0) and is excluded when queued_ms[m] > t_sync_ms[m] + slo_ms; prob[m] = idle / sum of idle (all 0 when no
+ * candidate has idle goodput).  All arrays host, n entries. */
+int epara_offload_probabilities(int n, const double* p_hat, const double* p_act, const double* queued_ms,
+                                const double* t_sync_ms, double slo_ms, double* prob);
+
+/* Event-driven replay (Section 5.2: request scheduling is executed in full, compute latency comes from the
+ * lookup tables, a hop costs offload_ms) of the requests against the placements under the request handler's
+ * decision list (Section 3.2): an item past its deadline answers timeout; else a local instance that would
+ * finish it in time takes it (the server's own first, then the hypothetical server's); else, with max_offload
+ * offloads behind it, offloading exceed; else it moves to a server not yet on its path picked by Eq. 1
+ * (p_hat: sum of bs / c(bs) over the server's instances of the service; p_act: their completions in
+ * [now - 2 sync_ms, now - sync_ms] per second; queued time: the least over those instances), or answers
+ * resource insufficiency when no candidate has idle goodput.  An instance runs one batch at a time: the oldest
+ * bs items still in time, for c(batch).  Placements that do not fit are skipped.  All pointers host. */
+int epara_simulate(const epara_cluster* c, const epara_service* services, int n_services, const epara_request* requests,
+                   int n_requests, const epara_placement* placements, int n_placements, int max_offload,
+                   epara_sim_result* out);
+
+/* Algorithm 1 (state-aware service placement) over Algorithm 2 (submodular placement for full models), with
+ * epara_simulate's phi as the objective: stage 1 places from the priority list (each entry at most once, the
+ * loop goes on while phi does not decrease), stage 2 from the set of all (service, real server) pairs, stage 3
+ * from the set of all (service, hypothetical server) pairs (both while phi strictly grows).  In every round the
+ * candidates that still fit are evaluated, the best ones form the tie set, and its first member in candidate
+ * order is placed.  out receives at most out_cap placements in placement order, *n_out their number
+ * (RESOURCE when out_cap is too small). */
+int epara_place_sssp(const epara_cluster* c, const epara_service* services, int n_services, const epara_request* requests,
+                     int n_requests, const epara_placement* priority, int n_priority, int max_offload,
+                     epara_placement* out, int out_cap, int* n_out);
 
 /* ---- single-kernel entry points (the same kernels a step launches), for parity tests and
  *      roofline measurement.  All pointers device unless named host. ---- */

@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libepara.so")
-SOURCES = ["epara_api.cu", "kernels_misc.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_stream.cu", "attention.cu", "attention_tc.cu",
+SOURCES = ["epara_api.cu", "kernels_misc.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_stream.cu", "gemm_swap.cu", "attention.cu", "attention_tc.cu", "attention_prefill.cu", "policy.cu",
            "selftest.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC"]
 

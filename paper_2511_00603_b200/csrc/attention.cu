@@ -50,7 +50,7 @@ __device__ __forceinline__ float merge_chunks(const float* p, int n_chunks, int 
 // kernel (attn_combine_kernel) does the same merge.  The arithmetic and its order are the same in both
 // cases, so the result depends neither on which block is last nor on the mode.
 template <int HD, int G>
-__device__ __forceinline__ void finish_chunk(const AttnDecGroup& g, int b, int kvh, int chunk, int len, int fused,
+__device__ __forceinline__ void finish_chunk(const AttnDecGroup& g, int b, int row, int kvh, int chunk, int len, int fused,
                                              const float (*sm_m)[G], const float (*sm_l)[G],
                                              const float (*sm_o)[G][HD]) {
   __shared__ int s_last;
@@ -68,7 +68,7 @@ __device__ __forceinline__ void finish_chunk(const AttnDecGroup& g, int b, int k
       oo += sm_o[w][h][e] * a;
     }
     if (n_chunks == 1) {
-      g.out[((size_t)b * g.Hq + (kvh * G + h)) * HD + e] = f2bf(oo / ll);
+      g.out[((size_t)row * g.Hq + (kvh * G + h)) * HD + e] = f2bf(oo / ll);
     } else {
       float* dst = g.partial + (((size_t)b * g.Hq + (kvh * G + h)) * g.max_chunks + chunk) * (HD + 2);
       __stcg(dst + 2 + e, oo);
@@ -90,7 +90,7 @@ __device__ __forceinline__ void finish_chunk(const AttnDecGroup& g, int b, int k
   for (int idx = threadIdx.x; idx < G * HD; idx += 128) {
     const int h = idx / HD, e = idx % HD;
     const float* p = g.partial + ((size_t)b * g.Hq + (kvh * G + h)) * g.max_chunks * (HD + 2);
-    g.out[((size_t)b * g.Hq + (kvh * G + h)) * HD + e] = f2bf(merge_chunks<HD>(p, n_chunks, e));
+    g.out[((size_t)row * g.Hq + (kvh * G + h)) * HD + e] = f2bf(merge_chunks<HD>(p, n_chunks, e));
   }
 }
 
@@ -104,11 +104,12 @@ __global__ void __launch_bounds__(HD) attn_combine_kernel(const AttnDecGroup* __
   const int b = blockIdx.y - g.req_start, hq = blockIdx.x;
   pdl_wait();
   if (hq >= g.Hq) return;
-  const int n_chunks = (g.reqs[b].len + ATTN_CHUNK - 1) / ATTN_CHUNK;
+  const AttnReq rq = g.reqs[b];
+  const int n_chunks = (rq.len + ATTN_CHUNK - 1) / ATTN_CHUNK;
   if (n_chunks == 1) return;            // finished by the attention kernel itself
   const float* p = g.partial + ((size_t)b * g.Hq + hq) * g.max_chunks * (HD + 2);
   const int e = threadIdx.x;
-  g.out[((size_t)b * g.Hq + hq) * HD + e] = f2bf(merge_chunks<HD>(p, n_chunks, e));
+  g.out[((size_t)rq.row * g.Hq + hq) * HD + e] = f2bf(merge_chunks<HD>(p, n_chunks, e));
 }
 
 template <int HD, int G>
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __
   const float scale = LOG2E * rsqrtf((float)HD);
 #pragma unroll
   for (int h = 0; h < G; ++h) {
-    const uint4 u = *reinterpret_cast<const uint4*>(g.q + (size_t)b * g.q_stride + (size_t)(kvh * G + h) * HD + c * 8);
+    const uint4 u = *reinterpret_cast<const uint4*>(g.q + (size_t)rq.row * g.q_stride + (size_t)(kvh * G + h) * HD + c * 8);
     unpack8(u, q[h]);
 #pragma unroll
     for (int e = 0; e < 8; ++e) q[h][e] *= scale;
@@ -243,7 +244,7 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(const AttnDecGroup* __
     }
   }
   __syncthreads();
-  finish_chunk<HD, G>(g, b, kvh, chunk, rq.len, fused, sm_m, sm_l, sm_o);
+  finish_chunk<HD, G>(g, b, rq.row, kvh, chunk, rq.len, fused, sm_m, sm_l, sm_o);
 }
 
 // Tensor-core variant for hd 64 / 128.  Same work split (chunk, kv head, request; 4 warps, warp w
@@ -342,7 +343,7 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
   // ---- Q fragments: rows 0..G-1 of the A operand are the query heads of this kv head
   uint32_t qa[KS][4];
   {
-    const bf16* qrow = g.q + (size_t)b * g.q_stride + (size_t)(kvh * G + gq) * HD;
+    const bf16* qrow = g.q + (size_t)rq.row * g.q_stride + (size_t)(kvh * G + gq) * HD;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
       qa[ks][0] = (gq < G) ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * tq) : 0u;
@@ -445,7 +446,7 @@ __global__ void __launch_bounds__(128) attn_decode_mma_kernel(const AttnDecGroup
     }
   }
   __syncthreads();
-  finish_chunk<HD, G>(g, b, kvh, chunk, rq.len, fused, sm_m, sm_l, sm_o);
+  finish_chunk<HD, G>(g, b, rq.row, kvh, chunk, rq.len, fused, sm_m, sm_l, sm_o);
 }
 
 template <int HD, int G>
@@ -507,7 +508,7 @@ __global__ void attn_prepare_kernel(AttnDecGroup g, AttnDecGroup* dst, AttnReq* 
   if (i < g.B) {
     reqs[i].table = tables + (size_t)i * stride;
     reqs[i].len = min(max(kv_lens[i], 0), max_len);
-    reqs[i].pad = 0;
+    reqs[i].row = i;
   }
   for (int c = i; c < n_counters; c += gridDim.x * blockDim.x) g.counters[c] = 0;
 }

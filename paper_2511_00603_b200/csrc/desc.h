@@ -22,10 +22,18 @@ struct ReqDesc {
   const int32_t* table;  // decoder block table
   void* out_logits;
   int32_t* out_argmax;
-  int token;
+  int token;             // decoder, single-token request: the token being decoded
   int kv_len;            // cached tokens before this step
   int n_blocks;
-  int pad;
+  int row_start;         // decoder: first activation row of the request (a prompt chunk takes n_tok rows)
+  int n_tok;             // decoder: tokens of the request in this step (1 = decode, > 1 = prompt chunk)
+  int pad[3];
+};
+
+// Decoder activations have one row per token.  Row r belongs to request `req`, sits at position `pos` of
+// its sequence and holds token id `token`.
+struct RowDesc {
+  int req, pos, token, pad;
 };
 
 // C = epi(A W^T + bias).  tmA/tmW are the TMA maps of A [rows, K] and W [N, K] (K innermost,
@@ -69,6 +77,7 @@ struct NormGroup {
   bf16* y;               // bf16 [M, d]
   const bf16* gamma;
   const bf16* beta;      // LN only
+  const int* row_index;  // when set, output row m reads input row row_index[m] (a decoder's last-token rows)
   long long x_stride;
   int M, d, kind;
   float eps;
@@ -77,7 +86,8 @@ struct NormGroup {
 enum : int { GATHER_ROWS = 0, GATHER_EMB = 1, GATHER_PATCH = 2 };
 struct GatherGroup {
   const ReqDesc* reqs;
-  void* out;             // ROWS: bf16 [B, ld]; EMB: fp32 [B, d]; PATCH: bf16 [B*np, 3*p*p]
+  const RowDesc* rows;   // EMB: one entry per output row
+  void* out;             // ROWS: bf16 [B, ld]; EMB: fp32 [rows, d]; PATCH: bf16 [B*np, 3*p*p]
   const bf16* emb;       // EMB
   int kind, B, width, ld;
   int img, patch;
@@ -86,9 +96,10 @@ struct GatherGroup {
 };
 
 struct RopeGroup {
-  bf16* qkv;             // [B, (Hq+2Hkv)*hd], q rotated in place
+  bf16* qkv;             // [rows, (Hq+2Hkv)*hd], q rotated in place
   bf16* kv_layer;        // [pages][2][Hkv][16][hd]
   const ReqDesc* reqs;
+  const RowDesc* rows;   // one entry per token row; B counts rows
   const float2* cs;      // [max position + 1][hd/2]: (cos, sin) of position * 10000^(-2j/hd)
   int* status;           // device word: set to ERR_PAGE_APPEND when a block table names a page outside the pool
   long long kv_pages;    // pages of the pool; a page id outside [0, kv_pages) is reported, its write skipped
@@ -98,7 +109,28 @@ struct RopeGroup {
 struct AttnReq {
   const int32_t* table;
   int len;               // tokens to attend (cached + appended)
-  int pad;
+  int row;               // activation row of the request's token (q is read and the output written there)
+};
+
+// Causal attention of prompt chunks (one layer): request i has n_tok query tokens in rows row_start ..,
+// token t at position kv_len + t attends to positions 0 .. kv_len + t of its paged cache (the chunk's own
+// k, v were appended by the kernel before).  One block per (request, query head, tile of 64 tokens).
+struct PrefillReq {
+  const int32_t* table;
+  int row_start, n_tok, kv_len;
+  int blk_start;         // first block of this request within its group
+};
+struct AttnPrefillGroup {
+  const bf16* qkv;       // [rows, q_stride], query head h at column h*hd
+  const bf16* kv_layer;
+  const PrefillReq* reqs;
+  bf16* out;             // [rows, Hq*hd]
+  int* status;
+  long long kv_pages;
+  int q_stride;
+  int n_reqs, Hq, Hkv, hd;
+  int blk_start;         // first block of this group in the launch
+  int n_blocks;
 };
 
 struct AttnDecGroup {
@@ -150,6 +182,7 @@ struct OutputGroup {     // copy logits rows to the requests' buffers and take t
 // Group arrays are packed back to back in the step blob: sizes must keep 8-byte alignment.
 namespace epara {
 static_assert(sizeof(GemmGroup) % 64 == 0, "GemmGroup holds 64-byte aligned TMA maps");
+static_assert(sizeof(AttnPrefillGroup) % 8 == 0 && sizeof(PrefillReq) % 8 == 0 && sizeof(RowDesc) == 16, "descriptor sizes");
 static_assert(sizeof(NormGroup) % 8 == 0 && sizeof(GatherGroup) % 8 == 0 && sizeof(RopeGroup) % 8 == 0 &&
               sizeof(AttnDecGroup) % 8 == 0 && sizeof(AttnEncGroup) % 64 == 0 && sizeof(AssembleGroup) % 8 == 0 &&
               sizeof(OutputGroup) % 8 == 0 && sizeof(ReqDesc) % 16 == 0 && sizeof(AttnReq) % 16 == 0,

@@ -83,7 +83,10 @@ bool make_tmap_c(CUtensorMap* tm, void* C, long long rows, int N, int ldc, int e
 
 struct Op {
   int kind;           // EPARA_K_*
-  int rows_per_req;   // rows of this op = batch * rows_per_req
+  int rows_per_req;   // rows of this op = batch * rows_per_req ...
+  int per_token;      // ... or, for a decoder's token-wise ops, the step's token rows (a prompt chunk has several)
+  int last_rows;      // norm: output row b reads the last token row of request b
+  AttnPrefillGroup apre;
   GemmGroup gemm;
   NormGroup norm;
   GatherGroup gather;
@@ -101,6 +104,8 @@ struct Op {
 struct Request {
   uint64_t ticket;
   epara_inputs in;
+  std::vector<int32_t> toks;   // decoder prompt chunk (n_tokens > 1): a copy of the caller's token ids
+  int n_tok() const { return toks.empty() ? 1 : (int)toks.size(); }
 };
 
 // T_INFLIGHT: admitted to a step whose slot still holds the step's record.  T_DONE: the final answer is
@@ -229,15 +234,22 @@ bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap,
   gemm_tc_config(rows_cap, N, K, g.epi, sm_count, &g.bn, &g.ksplit);
   if (max_rows <= GEMM_STREAM_MAX_ROWS && bl.gemm_impl == EPARA_GEMM_TCGEN05) {
     g.stream = 1; g.bn = 16; g.ksplit = 1;
+  } else if (max_rows <= GEMM_SWAP_MAX_ROWS && bl.gemm_impl == EPARA_GEMM_TCGEN05) {
+    g.stream = 3;                              // W as the MMA's 128-row operand, the batch as its N
+    g.bn = round_up((int)max_rows, 16);
+    g.ksplit = gemm_swap_ksplit(N, K, sm_count);
   } else if (bl.gemm_impl == EPARA_GEMM_TCGEN05 && gemm_tc_pair_eligible(rows_cap, N, K, g.epi, g.bn, g.ksplit)) {
     g.stream = 2;                              // 256-row tiles on CTA pairs
   }
-  if (g.ksplit > 1) {
+  if (g.ksplit > 1 && g.stream == 0) {
     const size_t tiles_m = (size_t)((rows_cap + TC_BM - 1) / TC_BM), tiles_n = (size_t)((N + g.bn - 1) / g.bn);
     m->splitk_bytes = std::max(m->splitk_bytes, (size_t)g.ksplit * tiles_m * TC_BM * tiles_n * g.bn * 4);
     m->splitk_tiles = std::max(m->splitk_tiles, tiles_m * tiles_n);
   }
-  if (bl.c && g.stream != 1) {
+  if (bl.c && g.stream == 3) {
+    if (!make_tmap(&g.tmA, A, rows_cap, K, lda, g.bn)) return false;
+    if (!make_tmap(&g.tmW, W, N, K, K, TC_BM)) return false;
+  } else if (bl.c && g.stream != 1) {
     if (!make_tmap(&g.tmA, A, rows_cap, K, lda, TC_BM)) return false;
     if (!make_tmap(&g.tmW, W, N, K, K, g.stream == 2 ? g.bn / 2 : g.bn)) return false;   // a pair's CTA loads half of the W rows
     if (!make_tmap_c(&g.tmC, C, rows_cap, N, ldc, g.epi)) return false;
@@ -452,6 +464,12 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
     at.adec.Hq = Hq; at.adec.Hkv = Hkv; at.adec.hd = hd; at.adec.max_chunks = m->max_chunks;
     at.adec.reqs_stable = 1; at.adec.kv_pages = d.kv_pages;
     m->ops.push_back(at);
+    Op ap;                                   // causal attention of the step's prompt chunks (none in a pure decode step)
+    memset(&ap, 0, sizeof(ap));
+    ap.kind = EPARA_K_ATTN_PREFILL; ap.rows_per_req = 1;
+    ap.apre.qkv = qkv; ap.apre.q_stride = nq; ap.apre.kv_layer = kv_layer; ap.apre.out = a; ap.apre.kv_pages = d.kv_pages;
+    ap.apre.Hq = Hq; ap.apre.Hkv = Hkv; ap.apre.hd = hd;
+    m->ops.push_back(ap);
     if (!add_gemm(bl, m, a, Hq * hd, Bcap, w[2], dm, Hq * hd, x, dm, nullptr, EPI_RESID_F32, 1)) return EPARA_E_CUDA;
     add_norm(m, x, dm, h, w[3], nullptr, dm, NORM_RMS, 1e-5f, 1);
     if (!add_gemm(bl, m, h, dm, Bcap, w[4], 2 * F, dm, f, F, nullptr, EPI_SWIGLU, 1)) return EPARA_E_CUDA;
@@ -467,6 +485,11 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
   o.outp.logits = logits; o.outp.N = d.vocab; o.outp.ld = ldl;
   m->ops.push_back(o);
   m->n_out = d.vocab;
+  // every op up to the last layer works on token rows; the final norm picks each request's last token row
+  // and the LM head and the output run per request
+  const size_t n_ops = m->ops.size();
+  for (size_t i = 0; i + 3 < n_ops; ++i) m->ops[i].per_token = 1;
+  m->ops[n_ops - 3].last_rows = 1;
   return EPARA_OK;
 }
 
@@ -480,7 +503,7 @@ int finish_model(Builder& bl, Model* m) {
   if (bl.c) {
     if (cudaMemset(counters, 0, m->splitk_tiles * sizeof(int)) != cudaSuccess) return EPARA_E_CUDA;
     for (Op& op : m->ops)
-      if (op.kind == EPARA_K_GEMM && op.gemm.ksplit > 1) { op.gemm.partial = partial; op.gemm.counters = counters; }
+      if (op.kind == EPARA_K_GEMM && op.gemm.ksplit > 1 && op.gemm.stream == 0) { op.gemm.partial = partial; op.gemm.counters = counters; }
   }
   return EPARA_OK;
 }
@@ -696,10 +719,22 @@ int epara_submit(epara_ctx* c, int model_id, int category, const epara_inputs* i
   Model* m = c->models[model_id];
   if (!in->out_logits && !in->out_argmax) return EPARA_E_INVALID;
   if (reinterpret_cast<uintptr_t>(in->out_logits) & 1) return EPARA_E_INVALID;
+  const int n_tok = (m->d.kind == EPARA_MODEL_DECODER && in->n_tokens > 1) ? in->n_tokens : 1;
   if (m->d.kind == EPARA_MODEL_DECODER) {
-    if (!in->block_table || in->kv_len < 0 || in->kv_len > m->d.max_kv_len) return EPARA_E_INVALID;
-    if (in->n_blocks < in->kv_len / EPARA_KV_PAGE + 1) return EPARA_E_INVALID;
-    if (in->token < 0 || in->token >= m->d.vocab) return EPARA_E_INVALID;
+    if (in->n_tokens < 0 || (in->n_tokens > 1 && !in->tokens)) return EPARA_E_INVALID;
+    const long long last_pos = (long long)in->kv_len + n_tok - 1;         // position of the request's last token
+    if (!in->block_table || in->kv_len < 0 || last_pos > m->d.max_kv_len) return EPARA_E_INVALID;
+    if (in->n_blocks < last_pos / EPARA_KV_PAGE + 1) return EPARA_E_INVALID;
+    if (n_tok > m->max_batch) return EPARA_E_RESOURCE;                      // more token rows than the model was placed for
+    if (n_tok > 1) {
+      if (m->d.head_dim != 64 && m->d.head_dim != 128) return EPARA_E_UNSUPPORTED;
+      for (int i = 0; i < n_tok; ++i)
+        if (in->tokens[i] < 0 || in->tokens[i] >= m->d.vocab) return EPARA_E_INVALID;
+    } else if (in->n_tokens == 1 && in->tokens) {
+      if (in->tokens[0] < 0 || in->tokens[0] >= m->d.vocab) return EPARA_E_INVALID;
+    } else if (in->token < 0 || in->token >= m->d.vocab) {
+      return EPARA_E_INVALID;
+    }
   } else {
     if (!in->input || (reinterpret_cast<uintptr_t>(in->input) & 15)) return EPARA_E_INVALID;
   }
@@ -707,7 +742,12 @@ int epara_submit(epara_ctx* c, int model_id, int category, const epara_inputs* i
   Request r;
   r.ticket = c->next_ticket++;
   r.in = *in;
-  m->q[category].push_back(r);
+  if (m->d.kind == EPARA_MODEL_DECODER) {
+    if (n_tok > 1) r.toks.assign(in->tokens, in->tokens + n_tok);
+    else if (in->n_tokens == 1 && in->tokens) r.in.token = in->tokens[0];
+    r.in.tokens = nullptr;                 // the caller's array is not kept
+  }
+  m->q[category].push_back(std::move(r));
   Ticket t;
   t.state = T_QUEUED; t.model = model_id; t.step = 0; t.out_logits = in->out_logits; t.out_argmax = in->out_argmax;
   t.result = EPARA_OK; t.device_error = 0;
@@ -740,12 +780,19 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
   inf.step_id = step_id;
 
   // ---- admission (A0) ----
-  struct Active { Model* m; int B; size_t req_off; size_t areq_off; size_t cursor; std::vector<Request> reqs; };
+  // B requests; `rows` activation rows (one per token for a decoder, B otherwise); n_dec single-token and
+  // n_pre prompt-chunk requests of a decoder, with their descriptor arrays in the blob
+  struct Active {
+    Model* m; int B; int rows; size_t req_off; size_t areq_off; size_t row_off; size_t preq_off; size_t last_off; size_t cursor;
+    int n_dec, n_pre, max_chunks_dec, pre_blocks;
+    std::vector<Request> reqs;
+  };
   std::vector<Active> act;
   for (size_t mi = 0; mi < c->models.size(); ++mi) {
     Model* m = c->models[mi];
     Active a;
-    a.m = m; a.B = 0; a.cursor = 0; a.req_off = 0; a.areq_off = 0;
+    a.m = m; a.B = 0; a.rows = 0; a.cursor = 0; a.req_off = 0; a.areq_off = 0; a.row_off = 0; a.preq_off = 0; a.last_off = 0;
+    a.n_dec = a.n_pre = a.max_chunks_dec = a.pre_blocks = 0;
     for (int cat = 0; cat < 2; ++cat) {
       std::deque<Request>& q = m->q[cat];
       if (q.empty()) continue;
@@ -758,6 +805,16 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       cap = std::min(cap, m->max_batch - a.B);
       std::vector<int> adm, drp;
       admit_impl(n, tk.data(), dl.data(), sid.data(), now_ns, cap, (cat == EPARA_CAT_FS_LT1) ? c->cfg.mf_max : 0, adm, drp);
+      // a request takes one activation row per token: admitted requests beyond the model's rows wait for a later step
+      {
+        size_t keep = 0;
+        for (; keep < adm.size(); ++keep) {
+          const int nt = q[adm[keep]].n_tok();
+          if (a.rows + nt > m->max_batch) break;
+          a.rows += nt;
+        }
+        adm.resize(keep);
+      }
       std::vector<char> gone(n, 0);
       for (int i : adm) { a.reqs.push_back(q[i]); gone[i] = 1; c->tickets[q[i].ticket].state = T_INFLIGHT; c->tickets[q[i].ticket].step = step_id; }
       for (int i : drp) { gone[i] = 1; Ticket& t = c->tickets[q[i].ticket]; t.state = T_DONE; t.result = EPARA_E_TIMEOUT; }
@@ -803,24 +860,62 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
   };
   bool overflow = false;
   for (Active& a : act) {
+    const bool dec = a.m->d.kind == EPARA_MODEL_DECODER;
     std::vector<ReqDesc> rd(a.B);
-    std::vector<AttnReq> ar(a.B);
+    std::vector<AttnReq> ar;
+    std::vector<PrefillReq> pr;
+    std::vector<RowDesc> rows;
+    std::vector<int> last(a.B);
+    int row = 0;
     for (int b = 0; b < a.B; ++b) {
-      const epara_inputs& in = a.reqs[b].in;
+      const Request& rq = a.reqs[b];
+      const epara_inputs& in = rq.in;
+      const int nt = dec ? rq.n_tok() : 1;
+      memset(&rd[b], 0, sizeof(ReqDesc));
       rd[b].input = in.input; rd[b].table = in.block_table; rd[b].out_logits = in.out_logits;
       rd[b].out_argmax = in.out_argmax; rd[b].token = in.token; rd[b].kv_len = in.kv_len;
-      rd[b].n_blocks = in.n_blocks; rd[b].pad = 0;
-      ar[b].table = in.block_table; ar[b].len = in.kv_len + 1; ar[b].pad = 0;
-      if (a.m->d.kind == EPARA_MODEL_DECODER) inf.kv_bytes += a.m->kv_bytes_per_token * in.kv_len;
+      rd[b].n_blocks = in.n_blocks; rd[b].row_start = row; rd[b].n_tok = nt;
+      if (dec) {
+        for (int t = 0; t < nt; ++t) {
+          RowDesc r;
+          r.req = b; r.pos = in.kv_len + t; r.token = nt > 1 ? rq.toks[t] : in.token; r.pad = 0;
+          rows.push_back(r);
+        }
+        if (nt == 1) {
+          AttnReq q1;
+          q1.table = in.block_table; q1.len = in.kv_len + 1; q1.row = row;
+          ar.push_back(q1);
+          a.max_chunks_dec = std::max(a.max_chunks_dec, (in.kv_len + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK);
+        } else {
+          PrefillReq p1;
+          p1.table = in.block_table; p1.row_start = row; p1.n_tok = nt; p1.kv_len = in.kv_len; p1.blk_start = a.pre_blocks;
+          a.pre_blocks += attn_prefill_blocks(nt, a.m->d.n_heads);
+          pr.push_back(p1);
+          inf.prefill_tokens += nt;
+        }
+        // cached bytes the step must read at least once: the request's whole sequence, once per layer
+        inf.kv_bytes += a.m->kv_bytes_per_token * (in.kv_len + (nt > 1 ? nt : 0));
+      }
+      last[b] = row + nt - 1;
+      row += nt;
     }
+    a.rows = dec ? row : a.B;
+    a.n_dec = (int)ar.size(); a.n_pre = (int)pr.size();
     a.req_off = put(rd.data(), rd.size() * sizeof(ReqDesc), 16);
-    if (a.m->d.kind == EPARA_MODEL_DECODER) a.areq_off = put(ar.data(), ar.size() * sizeof(AttnReq), 16);
-    if (a.req_off == (size_t)-1 || a.areq_off == (size_t)-1) overflow = true;
+    if (dec) {
+      a.row_off = put(rows.data(), rows.size() * sizeof(RowDesc), 16);
+      a.last_off = put(last.data(), last.size() * sizeof(int), 16);
+      if (!ar.empty()) a.areq_off = put(ar.data(), ar.size() * sizeof(AttnReq), 16);
+      if (!pr.empty()) a.preq_off = put(pr.data(), pr.size() * sizeof(PrefillReq), 16);
+    }
+    if (a.req_off == (size_t)-1 || a.areq_off == (size_t)-1 || a.row_off == (size_t)-1 || a.preq_off == (size_t)-1 ||
+        a.last_off == (size_t)-1)
+      overflow = true;
   }
 
   // ---- plan (A1): sweep the kernel kinds until every model's op list is exhausted ----
   static const int sweep[] = {EPARA_K_GATHER, EPARA_K_TRACE, EPARA_K_ASSEMBLE, EPARA_K_NORM, EPARA_K_GEMM, EPARA_K_ROPE,
-                              EPARA_K_ATTN_DEC, EPARA_K_ATTN_ENC, EPARA_K_OUTPUT};
+                              EPARA_K_ATTN_DEC, EPARA_K_ATTN_PREFILL, EPARA_K_ATTN_ENC, EPARA_K_OUTPUT};
   std::vector<Launch> launches;
   const bool simt = c->cfg.gemm_impl == EPARA_GEMM_SIMT;
   bool more = true;
@@ -838,7 +933,7 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           Launch LL;
           memset(&LL, 0, sizeof(LL));
           LL.kind = kind; LL.n_groups = 1;
-          LL.src = op.trace_src; LL.dst = op.trace_dst; LL.bytes = (size_t)a->B * op.trace_row_bytes;
+          LL.src = op.trace_src; LL.dst = op.trace_dst; LL.bytes = (size_t)a->rows * op.trace_row_bytes;
           launches.push_back(LL);
           a->cursor++;
         }
@@ -848,7 +943,8 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       // kernel for groups that never exceed 16 rows (pass 1) and 256-row tiles on CTA pairs for the dense
       // bf16-output groups (pass 2); encoder attention in two: the tcgen05 kernel (pass 0) and the
       // mma.sync kernel for shapes it does not take (pass 1)
-      const int n_pass = kind == EPARA_K_GEMM ? 3 : (kind == EPARA_K_ATTN_ENC ? 2 : 1);
+      // (passes 3 to 6: the swapped-operand kernel with 1, 2, 4 and 8 k ranges per tile)
+      const int n_pass = kind == EPARA_K_GEMM ? 7 : (kind == EPARA_K_ATTN_ENC ? 2 : 1);
       for (int pass = 0; pass < n_pass; ++pass) {
       Launch L;
       memset(&L, 0, sizeof(L));
@@ -874,20 +970,45 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           LL.kind = kind; LL.n_groups = (int)same.size();
           off = align_up(off, 64);
           LL.off = off;
-          int total_B = 0, max_hkv = 0, max_hq = 0, max_chunks = 0;
+          int total_B = 0, max_hkv = 0, max_hq = 0, max_chunks = 0, n_put = 0;
           for (Active* a : same) {
+            if (a->n_dec == 0) continue;               // only prompt chunks from this model in this step
             AttnDecGroup g = a->m->ops[a->cursor].adec;
-            g.B = a->B; g.reqs = (const AttnReq*)(slot.dev + a->areq_off); g.req_start = total_B;
+            g.B = a->n_dec; g.reqs = (const AttnReq*)(slot.dev + a->areq_off); g.req_start = total_B;
             g.status = dev_status;
-            total_B += a->B;
+            total_B += a->n_dec;
             max_hkv = std::max(max_hkv, g.Hkv); max_hq = std::max(max_hq, g.Hq);
-            for (int b = 0; b < a->B; ++b)
-              max_chunks = std::max(max_chunks, (a->reqs[b].in.kv_len + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK);
+            max_chunks = std::max(max_chunks, a->max_chunks_dec);
+            ++n_put;
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
           }
+          LL.n_groups = n_put;
           LL.p0 = total_B; LL.p1 = max_hkv | (max_hq << 16); LL.p2 = max_chunks; LL.p3 = (hd << 8) | G;
-          launches.push_back(LL);
+          if (n_put > 0) launches.push_back(LL);
           rest.swap(other);
+        }
+        for (Active* a : who) a->cursor++;
+        continue;
+      }
+      if (kind == EPARA_K_ATTN_PREFILL) {
+        for (int hd : {64, 128}) {
+          Launch LL;
+          memset(&LL, 0, sizeof(LL));
+          LL.kind = kind;
+          off = align_up(off, 64);
+          LL.off = off;
+          int blocks = 0, n_put = 0;
+          for (Active* a : who) {
+            AttnPrefillGroup g = a->m->ops[a->cursor].apre;
+            if (g.hd != hd || a->n_pre == 0) continue;
+            g.reqs = (const PrefillReq*)(slot.dev + a->preq_off); g.n_reqs = a->n_pre; g.status = dev_status;
+            g.blk_start = blocks; g.n_blocks = a->pre_blocks;
+            blocks += a->pre_blocks;
+            ++n_put;
+            if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
+          }
+          LL.n_groups = n_put; LL.p0 = blocks; LL.p1 = hd;
+          if (n_put > 0) launches.push_back(LL);
         }
         for (Active* a : who) a->cursor++;
         continue;
@@ -895,11 +1016,12 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       int total = 0, mx = 0;
       for (Active* a : who) {
         const Op& op = a->m->ops[a->cursor];
-        const int rows = a->B * op.rows_per_req;
+        const int rows = op.per_token ? a->rows : a->B * op.rows_per_req;
         switch (kind) {
           case EPARA_K_GATHER: {
             GatherGroup g = op.gather;
             g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
+            g.rows = (const RowDesc*)(slot.dev + a->row_off);
             g.blocks = g.kind == GATHER_PATCH ? (rows + GATHER_PATCH_ROWS - 1) / GATHER_PATCH_ROWS : rows;
             mx = std::max(mx, g.blocks);
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
@@ -915,15 +1037,22 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           case EPARA_K_NORM: {
             NormGroup g = op.norm;
             g.M = rows;
+            if (op.last_rows) g.row_index = (const int*)(slot.dev + a->last_off);
             mx = std::max(mx, norm_blocks(rows, g.d));
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
           case EPARA_K_GEMM: {
             GemmGroup g = op.gemm;
-            if (g.stream != pass) break;                       // another pass takes it
+            int gpass = g.stream;
+            if (g.stream == 3) gpass = 3 + (g.ksplit >= 8 ? 3 : g.ksplit >= 4 ? 2 : g.ksplit >= 2 ? 1 : 0);
+            if (gpass != pass) break;                          // another pass takes it
             g.M = rows;
-            if (g.stream == 2) {
+            if (g.stream == 3) {
+              g.tiles_m = 1; g.tiles_n = gemm_swap_tiles(g.N);
+              g.tile_start = total;
+              total += g.tiles_n;
+            } else if (g.stream == 2) {
               g.tiles_m = (rows + 2 * TC_BM - 1) / (2 * TC_BM); g.tiles_n = (g.N + g.bn - 1) / g.bn;
               g.tile_start = total;
               total += g.tiles_m * g.tiles_n;
@@ -952,9 +1081,10 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
           }
           case EPARA_K_ROPE: {
             RopeGroup g = op.rope;
-            g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = a->B;
+            g.reqs = (const ReqDesc*)(slot.dev + a->req_off); g.B = rows;
+            g.rows = (const RowDesc*)(slot.dev + a->row_off);
             g.status = dev_status;
-            mx = std::max(mx, a->B);
+            mx = std::max(mx, rows);
             if (put(&g, sizeof(g), 8) == (size_t)-1) overflow = true;
             break;
           }
@@ -1023,7 +1153,8 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       case EPARA_K_ASSEMBLE: launch_assemble((const AssembleGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_NORM: launch_norm((const NormGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_GEMM:
-        if (L.p2 == 1) err = launch_gemm_stream((const GemmGroup*)gp, L.n_groups, L.p0, L.p1, st);
+        if (L.p2 >= 3) err = launch_gemm_swap((const GemmGroup*)gp, L.n_groups, L.p0, 1 << (L.p2 - 3), dev_status, c->sm_count, st);
+        else if (L.p2 == 1) err = launch_gemm_stream((const GemmGroup*)gp, L.n_groups, L.p0, L.p1, st);
         else if (L.p2 == 2) err = launch_gemm_tc_pair((const GemmGroup*)gp, L.n_groups, L.p0, dev_status, c->sm_count, st);
         else if (simt) launch_gemm_simt((const GemmGroup*)gp, L.n_groups, L.p0, st);
         else err = launch_gemm_tc((const GemmGroup*)gp, L.n_groups, L.p0, L.p3, dev_status, c->sm_count, st);
@@ -1039,6 +1170,9 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
         break;
       case EPARA_K_OUTPUT: launch_output((const OutputGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_TRACE: err = cudaMemcpyAsync(L.dst, L.src, L.bytes, cudaMemcpyDeviceToDevice, st); break;
+      case EPARA_K_ATTN_PREFILL:
+        err = launch_attn_prefill((const AttnPrefillGroup*)gp, L.n_groups, L.p0, L.p1, st);
+        break;
     }
     if (prof) cudaEventRecord(slot.prof[2 * li + 1], st);
     ++li;
@@ -1148,6 +1282,8 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
   const bool simt = impl == EPARA_GEMM_SIMT;
   const int sm_count = device_sm_count(device);
   std::vector<GemmGroup> gs, gs_stream, gs_pair;   // tensor-core (or CUDA-core) groups; weight-streaming groups (M <= 16); CTA-pair groups
+  std::vector<GemmGroup> gs_swap[4];               // swapped-operand groups (17 to 128 rows) by k ranges per tile: 1, 2, 4, 8
+  int total_swap[4] = {0, 0, 0, 0};
   int total = 0, total_stream = 0, max_rows_stream = 0, total_pair = 0;
   size_t soff = epara_gemm_scratch_bytes(n);
   for (int i = 0; i < n; ++i) {
@@ -1172,6 +1308,19 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
       if (q.M > 0) total_stream += g.tiles_n;
       max_rows_stream = std::max(max_rows_stream, q.M);
       gs_stream.push_back(g);
+      continue;
+    }
+    if (!simt && q.M <= GEMM_SWAP_MAX_ROWS && q.K % 8 == 0) {
+      g.stream = 3;
+      g.bn = round_up(q.M, 16);
+      g.ksplit = gemm_swap_ksplit(q.N, q.K, sm_count);
+      const int si = g.ksplit >= 8 ? 3 : g.ksplit >= 4 ? 2 : g.ksplit >= 2 ? 1 : 0;
+      g.tiles_m = 1; g.tiles_n = gemm_swap_tiles(q.N);
+      g.tile_start = total_swap[si];
+      total_swap[si] += g.tiles_n;
+      if (!make_tmap(&g.tmA, q.A, q.M, q.K, q.lda, g.bn)) return EPARA_E_CUDA;
+      if (!make_tmap(&g.tmW, q.W, q.N, q.K, q.ldw, TC_BM)) return EPARA_E_CUDA;
+      gs_swap[si].push_back(g);
       continue;
     }
     if (!simt) gemm_tc_config(q.M, q.N, q.K, q.epilogue, sm_count, &g.bn, &g.ksplit);
@@ -1210,6 +1359,13 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
   GemmGroup* dev_groups = (GemmGroup*)((unsigned char*)scratch + 256);
   GemmGroup* dev_stream = dev_groups + gs.size();
   GemmGroup* dev_pair = dev_stream + gs_stream.size();
+  GemmGroup* dev_swap[4];
+  dev_swap[0] = dev_pair + gs_pair.size();
+  for (int i = 1; i < 4; ++i) dev_swap[i] = dev_swap[i - 1] + gs_swap[i - 1].size();
+  for (int i = 0; i < 4; ++i)
+    if (!gs_swap[i].empty() &&
+        cudaMemcpyAsync(dev_swap[i], gs_swap[i].data(), gs_swap[i].size() * sizeof(GemmGroup), cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return EPARA_E_CUDA;
   if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) return EPARA_E_CUDA;
   // (a copy from pageable host memory is staged before cudaMemcpyAsync returns, so the vectors may go out of scope)
   if (!gs.empty() &&
@@ -1234,6 +1390,8 @@ int epara_grouped_gemm(int device, void* cuda_stream, int impl, const epara_gemm
       err = launch_gemm_stream(dev_stream, (int)gs_stream.size(), total_stream, max_rows_stream, st);
     if (err == cudaSuccess)
       err = launch_gemm_tc_pair(dev_pair, (int)gs_pair.size(), total_pair, status, sm, st);
+    for (int i = 0; i < 4 && err == cudaSuccess; ++i)
+      err = launch_gemm_swap(dev_swap[i], (int)gs_swap[i].size(), total_swap[i], 1 << i, status, sm, st);
   }
   return err == cudaSuccess ? EPARA_OK : EPARA_E_CUDA;
 }

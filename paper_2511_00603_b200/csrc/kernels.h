@@ -30,6 +30,16 @@ cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total
 cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int max_bn, int* status,
                            int sm_count, cudaStream_t st);   // max_bn: widest tile among the groups
 
+// Swapped-operand tensor-core GEMM for groups of 17 to 128 rows (GemmGroup::stream == 3): a cluster of `ksplit`
+// CTAs per tile of 128 output columns; all groups of a launch share ksplit.  GemmGroup::bn holds the row capacity
+// rounded up to 16, tmW the weight map (box 128 rows), tmA the activation map (box bn rows); tile_start counts
+// tiles.  total_items = sum of gemm_swap_tiles(N).
+int gemm_swap_ksplit(int N, int K, int sm_count);
+int gemm_swap_tiles(int N);
+cudaError_t launch_gemm_swap(const GemmGroup* groups, int n_groups, int total_items, int ksplit, int* status, int sm_count,
+                             cudaStream_t st);
+constexpr int GEMM_SWAP_MAX_ROWS = 128;
+
 // Weight-streaming GEMM for groups that never exceed 16 rows (GemmGroup::stream): one block per 16
 // rows of W over the whole K, mma.sync, no tensor maps.  total_items = sum of gemm_stream_tiles(N).
 constexpr int GEMM_STREAM_MAX_ROWS = 16;
@@ -49,6 +59,11 @@ cudaError_t launch_attn_decode(const AttnDecGroup* groups, int n_groups, int tot
 void launch_attn_prepare(const AttnDecGroup& g, AttnDecGroup* dst, AttnReq* reqs, const int32_t* kv_lens,
                          const int32_t* tables, int stride, int max_len, int n_counters, cudaStream_t st);
 constexpr int DEC_STATUS_OFFSET = 192;   // byte offset of the status word in a single-kernel call's scratch
+
+// Causal attention of prompt chunks (head size 64 or 128), one block per (request, query head, 64 query tokens).
+constexpr int PREFILL_TILE = 64;
+inline int attn_prefill_blocks(int n_tok, int Hq) { return (n_tok + PREFILL_TILE - 1) / PREFILL_TILE * Hq; }
+cudaError_t launch_attn_prefill(const AttnPrefillGroup* groups, int n_groups, int total_blocks, int hd, cudaStream_t st);
 
 // Encoder attention on tcgen05 for groups with AttnEncGroup::tc (hd 64, T <= ENC_TC_MAX_T): persistent,
 // one item per (image, head); total_items = sum of B * H.  `status` as for the GEMM.

@@ -21,8 +21,8 @@ __global__ void __launch_bounds__(128) gather_kernel(const GatherGroup* __restri
     uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(g.out) + (size_t)b * g.ld);
     for (int i = threadIdx.x; i < g.width / 8; i += blockDim.x) dst[i] = src[i];
   } else if (g.kind == GATHER_EMB) {
-    const int b = blockIdx.x;
-    const int tok = g.reqs[b].token;
+    const int b = blockIdx.x;              // one block per token row
+    const int tok = g.rows[b].token;
     const uint4* src = reinterpret_cast<const uint4*>(g.emb + (size_t)tok * g.width);
     float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(g.out) + (size_t)b * g.width);
     for (int i = threadIdx.x; i < g.width / 8; i += blockDim.x) {
@@ -66,7 +66,7 @@ __device__ __forceinline__ void norm_row(const NormGroup& g, int row, float* red
   constexpr int STRIDE = WARP ? 32 : NORM_THREADS;
   const int t = WARP ? (threadIdx.x & 31) : threadIdx.x;
   const int nvec = g.d >> 2;
-  const float4* x = reinterpret_cast<const float4*>(g.x + (size_t)row * g.x_stride);
+  const float4* x = reinterpret_cast<const float4*>(g.x + (size_t)(g.row_index ? g.row_index[row] : row) * g.x_stride);
   float4 v[8];
   float s = 0.f;
 #pragma unroll
@@ -132,11 +132,12 @@ __device__ __forceinline__ void norm_rows_narrow(const NormGroup& g, int row0) {
   float4 v[NORM_NARROW_ROWS][4];
 #pragma unroll
   for (int r = 0; r < NORM_NARROW_ROWS; ++r) {
-    const float4* x = reinterpret_cast<const float4*>(g.x + (size_t)(row0 + r) * g.x_stride);
+    const bool live = row0 + r < g.M;
+    const float4* x = reinterpret_cast<const float4*>(g.x + (size_t)((live && g.row_index) ? g.row_index[row0 + r] : row0 + r) * g.x_stride);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int c = lane + i * 32;
-      v[r][i] = (row0 + r < g.M && c < nvec) ? x[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      v[r][i] = (live && c < nvec) ? x[c] : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
   const float inv_d = 1.0f / (float)g.d;
@@ -227,21 +228,22 @@ void launch_norm(const NormGroup* groups, int n_groups, int max_blocks, cudaStre
 }
 
 // ------------------------------------------------------------------ RoPE + KV append
-// One block per request.  The new token sits at position kv_len: q and k are rotated there
+// One block per token row (a decode request has one row, a prompt chunk one per token).  The row's token sits
+// at position `pos` of its sequence: q and k are rotated there
 // (interleaved pairs; cos and sin come from the model's table, computed from fp64 angles when the
 // model was placed), q in place, k and v written to the cache page table[pos/16], slot pos%16.
 // The page id comes from the caller's block table and is checked against the pool's page count.
 __global__ void __launch_bounds__(256) rope_append_kernel(const RopeGroup* __restrict__ groups) {
   const RopeGroup g = groups[blockIdx.y];
-  const int b = blockIdx.x;
+  const int b = blockIdx.x;               // token row
   if (b >= g.B) return;
   pdl_launch_dependents();
   pdl_wait();
-  const ReqDesc r = g.reqs[b];
-  const int pos = r.kv_len, hd = g.hd, half = hd >> 1;
+  const RowDesc rd = g.rows[b];
+  const int pos = rd.pos, hd = g.hd, half = hd >> 1;
   const float2* cs = g.cs + (size_t)pos * half;
-  const int page = r.table[pos / 16], slot = pos % 16;
-  // a page id outside the pool is reported and nothing is written for this request (q stays unrotated)
+  const int page = g.reqs[rd.req].table[pos / 16], slot = pos % 16;
+  // a page id outside the pool is reported and nothing is written for this row (q stays unrotated)
   if (page < 0 || page >= g.kv_pages) {
     if (threadIdx.x == 0) atomicExch(g.status, ERR_PAGE_APPEND);
     return;

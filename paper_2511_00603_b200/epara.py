@@ -23,7 +23,7 @@ CAT_LS, CAT_FS, CAT_LS_GT1, CAT_FS_GT1 = 0, 1, 2, 3
 MODEL_MLP, MODEL_VIT, MODEL_DECODER = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 EPI_BIAS, EPI_GELU, EPI_SWIGLU, EPI_RESID_F32 = 1, 2, 4, 8
-K_NAMES = ["gather", "norm", "gemm", "rope", "attn_dec", "attn_combine", "attn_enc", "assemble", "output", "gemm_stream", "trace"]
+K_NAMES = ["gather", "norm", "gemm", "rope", "attn_dec", "attn_combine", "attn_enc", "assemble", "output", "gemm_stream", "trace", "attn_prefill"]
 ERR_PAGE_APPEND, ERR_PAGE_ATTEND, ERR_SELFTEST_WAIT = 101, 102, 90
 DECODE_STATUS_OFFSET = 192
 K_COUNT = len(K_NAMES)
@@ -45,7 +45,7 @@ class ModelDesc(C.Structure):
 
 class Inputs(C.Structure):
     _fields_ = [("input", C.c_void_p), ("token", C.c_int), ("kv_len", C.c_int), ("block_table", C.c_void_p),
-                ("n_blocks", C.c_int), ("deadline_ns", C.c_longlong), ("arrival_ns", C.c_longlong),
+                ("n_blocks", C.c_int), ("tokens", C.POINTER(C.c_int32)), ("n_tokens", C.c_int), ("deadline_ns", C.c_longlong), ("arrival_ns", C.c_longlong),
                 ("stream", C.c_int), ("out_logits", C.c_void_p), ("out_argmax", C.c_void_p)]
 
 
@@ -53,7 +53,7 @@ class StepInfo(C.Structure):
     _fields_ = [("step_id", C.c_uint64), ("admitted", C.c_int * 2), ("dropped", C.c_int * 2),
                 ("launches", C.c_int), ("gemm_groups", C.c_int), ("gemm_flops", C.c_double),
                 ("weight_bytes", C.c_double), ("kv_bytes", C.c_double), ("stream_gemm_flops", C.c_double),
-                ("stream_weight_bytes", C.c_double)]
+                ("stream_weight_bytes", C.c_double), ("prefill_tokens", C.c_int)]
 
 
 class Output(C.Structure):
@@ -72,7 +72,8 @@ EXPORTS = ["epara_init", "epara_register_model", "epara_submit", "epara_submit_m
            "epara_dp_group_count", "epara_inter_request_count", "epara_admit_queue", "epara_grouped_gemm",
            "epara_gemm_scratch_bytes", "epara_gemm_scratch_bytes_for", "epara_decode_attention", "epara_decode_attention_scratch_bytes",
            "epara_decode_attention_static", "epara_static_scratch_bytes", "epara_decode_attention_static_status",
-           "epara_set_max_profile_launches", "epara_selftest_bounded_wait"]
+           "epara_set_max_profile_launches", "epara_selftest_bounded_wait", "epara_offload_probabilities", "epara_simulate",
+           "epara_place_sssp"]
 
 lib.epara_init.argtypes = [C.POINTER(Config), C.POINTER(C.c_void_p)]
 lib.epara_register_model.argtypes = [C.c_void_p, C.POINTER(ModelDesc), C.POINTER(C.c_int)]
@@ -114,6 +115,40 @@ lib.epara_set_max_profile_launches.argtypes = [C.c_void_p, C.c_int]
 lib.epara_selftest_bounded_wait.argtypes = [C.c_int, C.c_void_p, C.c_ulonglong, C.c_void_p, C.POINTER(C.c_int)]
 lib.epara_static_scratch_bytes.argtypes = []
 lib.epara_static_scratch_bytes.restype = C.c_size_t
+
+
+PROFILE_POINTS, MAX_OFFLOAD_DRAWS = 10, 5
+
+
+class Cluster(C.Structure):
+    _fields_ = [("n_servers", C.c_int), ("gpus", C.POINTER(C.c_int)), ("vram", C.c_double), ("sync_ms", C.c_double),
+                ("offload_ms", C.c_double)]
+
+
+class Service(C.Structure):
+    _fields_ = [("a", C.c_double), ("b", C.c_double), ("n_gpus", C.c_int), ("cat", C.c_int), ("bs", C.c_int),
+                ("slo_ms", C.c_double), ("fps", C.c_double), ("frames", C.c_int), ("c_ms", C.c_double * PROFILE_POINTS)]
+
+
+class SimRequest(C.Structure):
+    _fields_ = [("t_ms", C.c_double), ("service", C.c_int), ("server", C.c_int), ("u", C.c_double * MAX_OFFLOAD_DRAWS)]
+
+
+class Placement(C.Structure):
+    _fields_ = [("service", C.c_int), ("server", C.c_int)]
+
+
+class SimResult(C.Structure):
+    _fields_ = [("phi", C.c_double), ("served", C.c_int), ("timeout", C.c_int), ("offload_exceed", C.c_int),
+                ("insufficient", C.c_int), ("late", C.c_int), ("offloads", C.c_int), ("instances", C.c_int)]
+
+
+lib.epara_offload_probabilities.argtypes = [C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                            C.POINTER(C.c_double), C.c_double, C.POINTER(C.c_double)]
+lib.epara_simulate.argtypes = [C.POINTER(Cluster), C.POINTER(Service), C.c_int, C.POINTER(SimRequest), C.c_int,
+                               C.POINTER(Placement), C.c_int, C.c_int, C.POINTER(SimResult)]
+lib.epara_place_sssp.argtypes = [C.POINTER(Cluster), C.POINTER(Service), C.c_int, C.POINTER(SimRequest), C.c_int,
+                                 C.POINTER(Placement), C.c_int, C.c_int, C.POINTER(Placement), C.c_int, C.POINTER(C.c_int)]
 
 
 class EparaError(RuntimeError):
@@ -328,3 +363,50 @@ def epara_selftest_bounded_wait(status_dev, stream_ptr: int, limit_ns: int = 1_0
     code = C.c_int(0)
     s = lib.epara_selftest_bounded_wait(device, C.c_void_p(stream_ptr), limit_ns, status_dev.data_ptr(), C.byref(code))
     return s, code.value
+
+
+# ----------------------------------------------------------------------------- host policies (marshalling only)
+def _policy_args(cluster: Dict, services: Sequence[Dict], requests: Sequence[Dict]):
+    gp = (C.c_int * len(cluster["gpus"]))(*cluster["gpus"])
+    cl = Cluster(len(cluster["gpus"]), C.cast(gp, C.POINTER(C.c_int)), cluster["vram"], cluster["sync_ms"], cluster["offload_ms"])
+    sv = (Service * max(len(services), 1))()
+    for i, s in enumerate(services):
+        sv[i] = Service(s["a"], s["b"], s["n_gpus"], s["cat"], s["bs"], s["slo_ms"], s.get("fps", 0.0), s.get("frames", 0),
+                        (C.c_double * PROFILE_POINTS)(*s["c_ms"]))
+    rq = (SimRequest * max(len(requests), 1))()
+    for i, r in enumerate(requests):
+        rq[i] = SimRequest(r["t_ms"], r["service"], r["server"], (C.c_double * MAX_OFFLOAD_DRAWS)(*r["u"]))
+    return cl, sv, rq, gp
+
+
+def _placements(pl):
+    arr = (Placement * max(len(pl), 1))()
+    for i, (l, n) in enumerate(pl):
+        arr[i] = Placement(l, n)
+    return arr
+
+
+def epara_offload_probabilities(p_hat, p_act, queued_ms, t_sync_ms, slo_ms: float):
+    n = len(p_hat)
+    D = C.c_double * max(n, 1)
+    out = D()
+    _check(lib.epara_offload_probabilities(n, D(*p_hat), D(*p_act), D(*queued_ms), D(*t_sync_ms), slo_ms, out),
+           "epara_offload_probabilities")
+    return list(out[:n])
+
+
+def epara_simulate(cluster: Dict, services, requests, placements, max_offload: int = MAX_OFFLOAD_DRAWS) -> Dict:
+    cl, sv, rq, _keep = _policy_args(cluster, services, requests)
+    res = SimResult()
+    _check(lib.epara_simulate(C.byref(cl), sv, len(services), rq, len(requests), _placements(placements), len(placements),
+                              max_offload, C.byref(res)), "epara_simulate")
+    return {k: getattr(res, k) for k, _ in SimResult._fields_}
+
+
+def epara_place_sssp(cluster: Dict, services, requests, priority, max_offload: int = MAX_OFFLOAD_DRAWS, cap: int = 4096):
+    cl, sv, rq, _keep = _policy_args(cluster, services, requests)
+    out = (Placement * cap)()
+    n = C.c_int(0)
+    _check(lib.epara_place_sssp(C.byref(cl), sv, len(services), rq, len(requests), _placements(priority), len(priority),
+                                max_offload, out, cap, C.byref(n)), "epara_place_sssp")
+    return [(out[i].service, out[i].server) for i in range(n.value)]

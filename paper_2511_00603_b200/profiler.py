@@ -90,6 +90,17 @@ def compute_ms(table: Dict, service: str, batch: int) -> float:
     return float(t[str(sizes[-1])]) * batch / sizes[-1]
 
 
+def service_from_table(table: Dict, name: str, cat: int, slo_ms: float, a: float, b: float, n_gpus: int = 1, fps: float = 0.0,
+                       frames: int = 0) -> Dict:
+    """A service description for epara_simulate / epara_place_sssp whose compute times are the profiled ones:
+    c_ms[k] = step time at batch 2^k (points the sweep could not run take the last measured time scaled by the
+    batch), batch size = the profile's choice."""
+    t = table["services"][name]
+    c_ms = [compute_ms(table, name, 1 << k) for k in range(10)]
+    return {"a": a, "b": b, "n_gpus": n_gpus, "cat": cat, "bs": int(t["best_bs"]), "slo_ms": slo_ms, "fps": fps,
+            "frames": frames, "c_ms": c_ms}
+
+
 class GpuMeasure:
     """measure(service, bs, mt) on the real kernels: places `mt` instances of the service for batch `bs` on one GPU,
     runs `steps` saturated steps after `warmup`, L2 flushed before each, and returns the median device time of a step.
@@ -103,6 +114,10 @@ class GpuMeasure:
         self.torch, self.E, self.server, self.W = torch, E, server, W
         self.services, self.device, self.steps, self.warmup = services, device, steps, warmup
         self.kv_lo, self.kv_hi, self.slack = kv_lo, kv_hi, slack_bytes
+        from . import synth
+        for p in services.values():
+            if p["kind"] == "decoder" and "packed_layers" not in p:
+                p["packed_layers"] = [synth.pack_decoder_layer(L) for L in p["layers"]]
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=torch.device("cuda", device))
 
     def _need_bytes(self, p: Dict, bs: int, mt: int) -> int:

@@ -42,13 +42,17 @@ class Server:
 
     def submit(self, mid: int, category: int, x: Optional[torch.Tensor] = None, token: int = 0, kv_len: int = 0,
                table: Optional[torch.Tensor] = None, deadline_ns: int = 0, arrival_ns: int = 0, stream: int = 0,
-               outs=None) -> int:
+               outs=None, tokens=None) -> int:
+        """tokens: a prompt chunk (sequence of token ids) for a decoder; `token` is then ignored."""
         logits, am = outs if outs is not None else self._outs(mid)
         inp = E.Inputs()
         inp.input = x.data_ptr() if x is not None else None
         inp.token, inp.kv_len = int(token), int(kv_len)
         inp.block_table = table.data_ptr() if table is not None else None
         inp.n_blocks = int(table.numel()) if table is not None else 0
+        if tokens is not None:
+            arr = (E.C.c_int32 * len(tokens))(*[int(t) for t in tokens])     # read by the library during submit only
+            inp.tokens, inp.n_tokens = arr, len(tokens)
         inp.deadline_ns, inp.arrival_ns, inp.stream = int(deadline_ns), int(arrival_ns), int(stream)
         inp.out_logits, inp.out_argmax = logits.data_ptr(), am.data_ptr()
         t = self.ctx.epara_submit(mid, category, inp)

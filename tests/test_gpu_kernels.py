@@ -125,6 +125,37 @@ def test_grouped_gemm_tile_pairs(E):
     assert torch.equal(alone[0]["C"], probs[0]["C"])
 
 
+def test_grouped_gemm_swapped_operands_17_to_128_rows(E):
+    """Problems of 17 to 128 rows run with W as the tensor core's 128-row operand and the batch as its N, a cluster
+    of 1, 2, 4 or 8 CTAs per tile of 128 output columns splitting K (reduced through distributed shared memory in
+    rank order): every epilogue, N below and not a multiple of a tile, K not a multiple of a k-block, batch sizes
+    on both sides of the multiples of 16, one k-block, and the decode shapes of the 1B decoder.  The same problem
+    alone and among others gives the same bits."""
+    cases = [(17, 10, 512, ("bias",)), (128, 3072, 2048, ()), (100, 1000, 776, ("bias",)), (48, 2048, 8192, ("resid",)),
+             (33, 512, 256, ("swiglu",)), (64, 2048, 2048, ("resid", "bias")), (127, 16384, 2048, ("swiglu",)),
+             (32, 1024, 256, ("bias", "gelu")), (96, 136, 64, ("gelu", "bias")), (20, 768, 4096, ("gelu", "bias")),
+             (128, 32000, 2048, ()), (31, 264, 1536, ("bias", "resid")), (80, 4096, 4096, ("swiglu",))]
+    probs, refs = _run_gemm(E, E.GEMM_TCGEN05, cases, seed=11)
+    for p, ref, case in zip(probs, refs, cases):
+        assert_close(p["C"][:ref.shape[0], :ref.shape[1]], ref, what=f"swapped gemm {case}")
+    alone, _ = _run_gemm(E, E.GEMM_TCGEN05, cases[:2], seed=11)
+    assert torch.equal(alone[1]["C"], probs[1]["C"])
+    # fewer live rows than the capacity the tile was sized for leave the other rows' outputs untouched
+    M, N, K = 128, 512, 512
+    g = torch.Generator(device="cuda").manual_seed(12)
+    A = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
+    W = (torch.randn((N, K), generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    full = torch.zeros((M, N), device="cuda", dtype=torch.bfloat16)
+    part = torch.full((M, N), 7.0, device="cuda", dtype=torch.bfloat16)
+    for C_, rows in ((full, M), (part, 40)):
+        pr = [{"A": A, "W": W, "C": C_, "bias": None, "M": rows, "N": N, "K": K, "epilogue": 0}]
+        sc = torch.empty(E.epara_gemm_scratch_bytes_for(pr), dtype=torch.uint8, device="cuda")
+        E.epara_grouped_gemm(pr, _stream(), sc)
+    torch.cuda.synchronize()
+    assert bool((part[40:] == 7.0).all())
+    assert_close(part[:40], to_f64(full[:40]), what="first 40 rows", tol=1e-6)
+
+
 def test_grouped_gemm_rejects_bad_arguments(E):
     dev = torch.device("cuda")
     A = torch.zeros((8, 64), device=dev, dtype=torch.bfloat16)
