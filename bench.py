@@ -415,6 +415,18 @@ def run_gpu(args):
         torch.cuda.synchronize()
         drain()
 
+    check = None
+    if args.check:
+        # sampled parity of the resident step (a test mode: the comparison and its use of the CPU oracle live in
+        # tests/stress_check.py; nothing of it runs inside the timed region)
+        if not stress:
+            raise SystemExit("--check goes with --workload stress (the mixed step has tests/test_gpu_step.py::"
+                             "test_mixed_bench_workload_sampled_parity)")
+        from tests import stress_check
+        if rank == 0:
+            check = stress_check.check_stress_step(insts, n_dec=8, n_img=2, log=lambda m: print(m, file=sys.stderr, flush=True))
+            check["passed"] = True
+
     # ---- timed region: K steps, device-timed; every PROFILE_EVERY-th step (the last one among them)
     # brackets each launch with CUDA events for the per-kernel times.  The events keep a kernel from
     # starting under the tail of the one before it, so a bracketed step is some 7 % slower than a plain
@@ -612,6 +624,8 @@ def run_gpu(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "ms_per_step_unprofiled": ms_plain,
             "ls_latency": poisson, "config_steps": cfg_steps}
+    if check is not None:
+        line["check"] = check
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -776,6 +790,9 @@ def main():
     ap.add_argument("--kv-hi", type=int, default=4096,
                     help="mixed workload: upper bound of the decoders' KV lengths (a short cache keeps a profiler capture small; "
                          "the GEMM launches do not depend on it)")
+    ap.add_argument("--check", action="store_true",
+                    help="stress workload only: compare 8 decode requests and 2 images of the resident step with the "
+                         "CPU oracle before timing (about a quarter of an hour)")
     ap.add_argument("--no-poisson", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-config-steps", action="store_true",

@@ -206,3 +206,30 @@ def test_decode_attention_matches_oracle(E, Hq, Hkv, hd):
         K, V = O.gather_kv(lambda l, pg: pool_ref[pg], 0, tables[b], int(L))
         ref = np.stack([O.attention(qf[b, h], K[h // (Hq // Hkv)], V[h // (Hq // Hkv)]) for h in range(Hq)])
         assert_close(out[b].reshape(Hq, hd), ref, what=f"decode attention b={b} L={L}")
+
+
+@pytest.mark.parametrize("rows", [16, 100, 200, 1024])
+def test_gelu_epilogue_sweep_through_identity_gemm(E, rows):
+    """The device GELU over its whole range: x swept over [-8, 8] (every bf16 value of a fine grid) goes through a
+    GEMM with the identity as weights, so the accumulator holds x exactly and the epilogue alone decides the
+    output.  Bound: the fitted form's 2.6e-5, the hardware tanh's relative error 2^-11 scaled by 0.5 |x|
+    (2.5e-4 |x|), and the rounding of the bf16 store (half an ulp: at most 2^-8 of the result).  The row counts select the
+    weight-streaming kernel, the swapped-operand kernel, the one-CTA tile kernel and the tile-pair kernel."""
+    dev = torch.device("cuda")
+    K = N = 256
+    x = torch.linspace(-8.0, 8.0, rows * K, device=dev).reshape(rows, K)
+    x = x[:, torch.randperm(K, generator=torch.Generator(device=dev).manual_seed(rows), device=dev)].to(torch.bfloat16)
+    W = torch.eye(N, K, device=dev).to(torch.bfloat16)
+    C = torch.full((rows, N), float("nan"), device=dev, dtype=torch.bfloat16)
+    prob = [{"A": x, "W": W, "C": C, "bias": None, "M": rows, "N": N, "K": K, "epilogue": E.EPI_GELU}]
+    scratch = torch.empty(E.epara_gemm_scratch_bytes_for(prob), dtype=torch.uint8, device=dev)
+    E.epara_grouped_gemm(prob, _stream(), scratch, impl=E.GEMM_TCGEN05)
+    torch.cuda.synchronize()
+    assert int(scratch[:4].view(torch.int32).item()) == 0
+    xs = O.bf16_to_f64(synth.to_bits(x))
+    ref = O.gelu(xs)
+    got = to_f64(C)
+    bound = 2.6e-5 + 2.5e-4 * np.abs(xs) + 2.0 ** -8 * np.abs(ref) + 1e-7
+    bad = np.abs(got - ref) > bound
+    assert not bad.any(), f"{int(bad.sum())} of {bad.size} outside the bound; worst excess " \
+                          f"{float(np.max(np.abs(got - ref) - bound)):.3e} at x = {float(xs[np.unravel_index(np.argmax(np.abs(got - ref) - bound), xs.shape)])}"

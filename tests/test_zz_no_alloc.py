@@ -44,17 +44,27 @@ def _case(E, B, lens, Hq, Hkv, hd, seed):
 
 def test_static_scratch_entry_matches_the_ordinary_entry_twice_in_a_row(E):
     stream = torch.cuda.current_stream().cuda_stream
-    # two different problems back to back: the second call finds the first one's leftovers in the array
-    for (B, lens, Hq, Hkv, hd, seed) in [(6, [700, 1, 256, 257, 40, 1023], 8, 2, 64, 70),
-                                        (3, [300, 17, 513], 8, 2, 128, 80)]:
+    # different problems back to back: each call finds the previous one's leftovers in the array; the third
+    # repeats the first (several chunks per request, merged by the last block to arrive) after the second,
+    # so it runs on chunk counters that the earlier calls must have left at zero
+    problems = [(6, [700, 1, 256, 257, 40, 1023], 8, 2, 64, 70), (3, [300, 17, 513], 8, 2, 128, 80),
+                (6, [700, 1, 256, 257, 40, 1023], 8, 2, 64, 70)]
+    for n, (B, lens, Hq, Hkv, hd, seed) in enumerate(problems):
         q, pool, lens_d, tabs_d, max_len = _case(E, B, lens, Hq, Hkv, hd, seed)
         ref = torch.empty_like(q)
         scratch = torch.empty(E.lib.epara_decode_attention_scratch_bytes(B, Hq, hd, max_len), dtype=torch.uint8,
                               device=q.device)
         E.epara_decode_attention(q, pool, lens_d, tabs_d, ref, Hq, Hkv, hd, max_len, scratch, stream)
         got = torch.full_like(q, float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         E.epara_decode_attention_static(q, pool, lens_d, tabs_d, got, Hq, Hkv, hd, max_len, stream)
         torch.cuda.synchronize()
+        free_after = torch.cuda.mem_get_info()[0]
+        if n > 0:
+            # (the first call may load the kernels; from the second on the call must leave the device's free
+            # memory exactly as it found it)
+            assert free_after == free_before, f"call {n}: free device memory changed by {free_before - free_after} bytes"
         assert_close(got, to_f64(ref), what=f"static-scratch decode attention B={B} hd={hd}")
         assert torch.equal(got, ref)          # same kernels, same reduction order
 
