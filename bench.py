@@ -682,6 +682,57 @@ def measure_decode_step(torch, E, server, W, synth, peaks, cfgm, B, lo, hi, step
             "frac_hbm": byt / (ms / 1e3) / 1e9 / peaks["hbm_gbs"], "tokens_per_s": B / (ms / 1e3), "per_kind_ms": kinds}
 
 
+def measure_prefill_step(torch, E, server, synth, peaks, cfgm, n_prompts, n_tok, steps, flush):
+    """Whole prefill steps of one decoder: n_prompts prompts of n_tok tokens each on an empty cache, one step
+    (the prompts' chunks are the step's rows; every layer's GEMMs see n_prompts * n_tok rows).  Work counted:
+    the step's GEMM flops as the library reports them plus the causal attention's 4 * hd * Hq * n (n + 1) / 2
+    per prompt and layer."""
+    import numpy as np
+    dev = torch.device("cuda", torch.cuda.current_device())
+    srv = server.Server(device=dev.index, workspace_bytes=6 << 30)
+    p = synth.make_decoder(seed=2, device=dev, **cfgm)
+    pages_per = (n_tok + 15) // 16
+    pool = synth.make_kv_pool(cfgm["n_layers"], n_prompts * pages_per + 2, cfgm["n_kv_heads"], cfgm["head_dim"], seed=5, device=dev)
+    m = srv.add_model(p, kv_pool=pool, max_kv_len=n_tok, max_batch=n_prompts * n_tok)
+    rng = np.random.default_rng(7)
+    prompts = [[int(t) for t in rng.integers(0, cfgm["vocab"], n_tok)] for _ in range(n_prompts)]
+    perm = rng.permutation(n_prompts * pages_per).astype(np.int32)
+    tables = [torch.as_tensor(perm[i * pages_per:(i + 1) * pages_per], device=dev) for i in range(n_prompts)]
+    stream = torch.cuda.current_stream(dev)
+    times, info = [], None
+    for i in range(steps + 4):
+        if i == steps + 3:
+            srv.ctx.epara_set_profile(True)
+        flush.zero_()
+        ts = [srv.submit(m, E.CAT_FS, tokens=prompts[k], kv_len=0, table=tables[k]) for k in range(n_prompts)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        info = srv.step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        for t in ts:
+            st = srv.collect(t)[0]
+            if st != E.OK:
+                raise RuntimeError(f"prefill request: status {st}")
+        if 3 <= i < steps + 3:
+            times.append(e0.elapsed_time(e1))
+    prof = srv.ctx.epara_step_profile()
+    kinds = {k: round(v[0], 4) for k, v in prof.items() if v[1]}
+    ms = sorted(times)[len(times) // 2]
+    attn = 4.0 * cfgm["head_dim"] * cfgm["n_q_heads"] * n_tok * (n_tok + 1) / 2 * cfgm["n_layers"] * n_prompts
+    fl = info.gemm_flops + attn
+    gemm_ms = kinds.get("gemm", 0.0) + kinds.get("gemm_stream", 0.0)
+    srv.close()
+    return {"kernel": "prefill step", "d": cfgm["d"], "prompts": n_prompts, "tokens_per_prompt": n_tok, "ms": ms,
+            "launches": info.launches, "prefill_tokens": info.prefill_tokens, "tokens_per_s": n_prompts * n_tok / (ms / 1e3),
+            "tflops_step": fl / (ms / 1e3) / 1e12, "frac_tensor_burst": fl / (ms / 1e3) / 1e12 / peaks["bf16_tflops"],
+            "frac_tensor_sustained": fl / (ms / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "gemm_tflops": (info.gemm_flops / (gemm_ms / 1e3) / 1e12) if gemm_ms else None,
+            "gemm_frac_tensor_burst": (info.gemm_flops / (gemm_ms / 1e3) / 1e12 / peaks["bf16_tflops"]) if gemm_ms else None,
+            "attn_prefill_tflops": (attn / (kinds["attn_prefill"] / 1e3) / 1e12) if kinds.get("attn_prefill") else None,
+            "per_kind_ms": kinds}
+
+
 # ------------------------------------------------------------------------------ single-kernel timings
 MICRO_GEMM = {
     "vit_s": [(50432, 1152, 384, "bias"), (50432, 384, 384, "bias,resid"), (50432, 1536, 384, "bias,gelu"),
@@ -768,6 +819,12 @@ def run_micro(args):
         from paper_2511_00603_b200 import server, workloads as W
         print(json.dumps(measure_vit_step(torch, E, server, W, synth, peaks, W.VIT_S if args.case == "vit_s" else W.VIT_B,
                                           args.m or 64, args.steps, flush)))
+    elif args.micro == "prefill_step":
+        from paper_2511_00603_b200 import server, configs
+        big = args.case == "dec_8b"
+        n_prompts, n_tok = (args.m or 4), args.tokens
+        print(json.dumps(measure_prefill_step(torch, E, server, synth, peaks, configs.DEC_8B if big else configs.DEC_1B,
+                                              n_prompts, n_tok, args.steps, flush)))
     elif args.micro == "decode_step":
         from paper_2511_00603_b200 import server, workloads as W
         big = args.case == "dec_8b"
@@ -778,7 +835,7 @@ def run_micro(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["gemm", "attn_dec", "decode_step", "vit_step"], help="time one kernel instead of the step")
+    ap.add_argument("--micro", default=None, choices=["gemm", "attn_dec", "decode_step", "vit_step", "prefill_step"], help="time one kernel instead of the step")
     ap.add_argument("--case", default="vit_s")
     ap.add_argument("--m", type=int, default=0, help="override M (gemm) or B (attn_dec) of the micro case")
     ap.add_argument("--gpus", type=int, default=1)
@@ -790,6 +847,7 @@ def main():
     ap.add_argument("--kv-hi", type=int, default=4096,
                     help="mixed workload: upper bound of the decoders' KV lengths (a short cache keeps a profiler capture small; "
                          "the GEMM launches do not depend on it)")
+    ap.add_argument("--tokens", type=int, default=2048, help="prefill_step micro: tokens per prompt (--m prompts per step)")
     ap.add_argument("--check", action="store_true",
                     help="stress workload only: compare 8 decode requests and 2 images of the resident step with the "
                          "CPU oracle before timing (about a quarter of an hour)")
