@@ -100,7 +100,7 @@ __device__ __forceinline__ Item decode_item(const G& g, int local) {
 // the current group (descriptor reads from global memory are latency the MMA issuer cannot hide).
 struct GroupCache {
   const GemmGroup* g;
-  int start, end, tiles_n, ksplit, bn, kblocks;
+  int start, end, tiles_n, ksplit, bn, kblocks, K;
 };
 __device__ __forceinline__ void group_cache(GroupCache& c, const GemmGroup* groups, int n_groups, int item) {
   if (c.g != nullptr && item >= c.start && item < c.end) return;
@@ -111,7 +111,8 @@ __device__ __forceinline__ void group_cache(GroupCache& c, const GemmGroup* grou
   c.ksplit = g->ksplit;
   c.bn = g->bn;
   c.end = c.start + g->tiles_m * g->tiles_n * g->ksplit;
-  c.kblocks = (g->K + TC_BK - 1) / TC_BK;
+  c.K = g->K;
+  c.kblocks = (c.K + TC_BK - 1) / TC_BK;
 }
 __device__ __forceinline__ Item decode_item(const GroupCache& c, int item) {
   const int local = item - c.start;
@@ -659,7 +660,7 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
       for (int item = pair; item < total_items && ok; item += n_pairs) {
         group_cache(gc, groups, n_groups, item);
         const GemmGroup* g = gc.g;
-        const Item it = decode_item_pair(*g, item - gc.start, rank);
+        const Item it = decode_item_pair(gc, item - gc.start, rank);
         if (g != g_prev) { tensormap_acquire(&g->tmA); g_prev = g; }
         const uint32_t bytes = 2u * (A_BYTES + (uint32_t)(gc.bn >> 1) * TC_BK * 2);   // both CTAs' boxes of a k-block
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
@@ -687,7 +688,7 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
       for (int item = pair; item < total_items && ok; item += n_pairs) {
         group_cache(gc, groups, n_groups, item);
         const GemmGroup* g = gc.g;
-        const Item it = decode_item_pair(*g, item - gc.start, rank);
+        const Item it = decode_item_pair(gc, item - gc.start, rank);
         if (g != g_prev) { tensormap_acquire(&g->tmW); g_prev = g; }
         const int n_half = it.n0 + rank * (gc.bn >> 1);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
