@@ -56,7 +56,11 @@ enum {
 
 enum { EPARA_MODEL_MLP = 0, EPARA_MODEL_VIT = 1, EPARA_MODEL_DECODER = 2 };
 
-enum { EPARA_GEMM_TCGEN05 = 0, EPARA_GEMM_SIMT = 1 };
+/* EPARA_GEMM_TCGEN05: the tensor-core kernels, with an encoder's MLP block (FC1, GELU, FC2, residual) run as one
+ * fused kernel where its shapes allow (d a multiple of 64 up to 384, hidden width a multiple of 128, more than
+ * 128 rows at capacity).  EPARA_GEMM_TCGEN05_UNFUSED: the same kernels, every GEMM its own launch.  Both round
+ * at the same points and reduce in the same order.  EPARA_GEMM_SIMT: plain CUDA-core comparator. */
+enum { EPARA_GEMM_TCGEN05 = 0, EPARA_GEMM_SIMT = 1, EPARA_GEMM_TCGEN05_UNFUSED = 2 };
 
 #define EPARA_KV_PAGE 16 /* tokens per KV page */
 
@@ -67,7 +71,7 @@ typedef struct {
   int cap_ls;             /* BS cap of a latency-sensitive group per model per step (0 -> 4) */
   int cap_fs;             /* BS cap of a frequency-sensitive group (0 -> 256) */
   int mf_max;             /* MF: max inter-frame count per stream; 0 = plain oldest-first batching */
-  int gemm_impl;          /* EPARA_GEMM_TCGEN05 (default) or EPARA_GEMM_SIMT (plain CUDA-core comparator) */
+  int gemm_impl;          /* EPARA_GEMM_TCGEN05 (default), EPARA_GEMM_TCGEN05_UNFUSED or EPARA_GEMM_SIMT */
   int max_queue;          /* queued requests per (model, category) before RESOURCE (0 -> 4096) */
   int profile;            /* 1: bracket every launch with CUDA events (see epara_step_profile) */
 } epara_config;

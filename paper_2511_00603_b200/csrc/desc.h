@@ -163,6 +163,24 @@ struct alignas(64) AttnEncGroup {
   int pad[8];
 };
 
+// One transformer MLP block of an encoder as a single work unit of the fused kernel:
+// z += GELU(h W1^T + b1) W2^T + b2 with h bf16 [rows, d], W1 [F, d], W2 [d, F], z fp32 [rows, d].
+// d is a multiple of 64 and at most 384 (the output accumulator of a 128-row tile must fit the tensor memory
+// beside one 128-column chunk of the hidden layer), F a multiple of 128.
+struct alignas(64) MlpGroup {
+  CUtensorMap tmX;       // h [rows, d] bf16, box 64 columns x 128 rows, 128-byte swizzle
+  CUtensorMap tmW1;      // W1 [F, d] bf16, box 64 x 64 rows (one CTA of a pair loads half of a chunk's 128 rows)
+  CUtensorMap tmW2;      // W2 [d, F] bf16, box 64 x n2/2 rows (n2 = d, or d / 2 when d > 256: two MMAs per k step)
+  CUtensorMap tmC;       // z [rows, d] fp32, box 16 columns x 32 rows (TMA reduce-add of the epilogue)
+  const bf16* b1;        // [F] or null
+  const bf16* b2;        // [d] or null
+  int M, d, F;
+  int tile_start;        // first work item (256-row tile) of this group in the launch
+  int tiles_m;
+  int c_rows;            // row extent of tmC
+  int pad[8];
+};
+
 struct AssembleGroup {   // z[b, 0] = cls + pos[0]; z[b, 1+p] = E[b*np + p] + pos[1+p]
   const bf16* E;
   const bf16* cls;
@@ -184,7 +202,7 @@ namespace epara {
 static_assert(sizeof(GemmGroup) % 64 == 0, "GemmGroup holds 64-byte aligned TMA maps");
 static_assert(sizeof(AttnPrefillGroup) % 8 == 0 && sizeof(PrefillReq) % 8 == 0 && sizeof(RowDesc) == 16, "descriptor sizes");
 static_assert(sizeof(NormGroup) % 8 == 0 && sizeof(GatherGroup) % 8 == 0 && sizeof(RopeGroup) % 8 == 0 &&
-              sizeof(AttnDecGroup) % 8 == 0 && sizeof(AttnEncGroup) % 64 == 0 && sizeof(AssembleGroup) % 8 == 0 &&
+              sizeof(AttnDecGroup) % 8 == 0 && sizeof(AttnEncGroup) % 64 == 0 && sizeof(MlpGroup) % 64 == 0 && sizeof(AssembleGroup) % 8 == 0 &&
               sizeof(OutputGroup) % 8 == 0 && sizeof(ReqDesc) % 16 == 0 && sizeof(AttnReq) % 16 == 0,
               "descriptor sizes");
 }  // namespace epara

@@ -88,6 +88,7 @@ struct Op {
   int last_rows;      // norm: output row b reads the last token row of request b
   AttnPrefillGroup apre;
   GemmGroup gemm;
+  MlpGroup mlp;          // EPARA_K_GEMM with gemm.stream == 4: FC1, GELU, FC2 and the residual update in one kernel
   NormGroup norm;
   GatherGroup gather;
   RopeGroup rope;
@@ -232,13 +233,13 @@ bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap,
   g.N = N; g.K = K; g.lda = lda; g.ldw = K; g.ldc = ldc; g.epi = epi | (bias ? EPI_BIAS : 0);
   op.weight_bytes = 2.0 * N * K;
   gemm_tc_config(rows_cap, N, K, g.epi, sm_count, &g.bn, &g.ksplit);
-  if (max_rows <= GEMM_STREAM_MAX_ROWS && bl.gemm_impl == EPARA_GEMM_TCGEN05) {
+  if (max_rows <= GEMM_STREAM_MAX_ROWS && bl.gemm_impl != EPARA_GEMM_SIMT) {
     g.stream = 1; g.bn = 16; g.ksplit = 1;
-  } else if (max_rows <= GEMM_SWAP_MAX_ROWS && bl.gemm_impl == EPARA_GEMM_TCGEN05) {
+  } else if (max_rows <= GEMM_SWAP_MAX_ROWS && bl.gemm_impl != EPARA_GEMM_SIMT) {
     g.stream = 3;                              // W as the MMA's 128-row operand, the batch as its N
     g.bn = round_up((int)max_rows, 16);
     g.ksplit = gemm_swap_ksplit(N, K, sm_count);
-  } else if (bl.gemm_impl == EPARA_GEMM_TCGEN05 && gemm_tc_pair_eligible(rows_cap, N, K, g.epi, g.bn, g.ksplit)) {
+  } else if (bl.gemm_impl != EPARA_GEMM_SIMT && gemm_tc_pair_eligible(rows_cap, N, K, g.epi, g.bn, g.ksplit)) {
     g.stream = 2;                              // 256-row tiles on CTA pairs
   }
   if (g.ksplit > 1 && g.stream == 0) {
@@ -255,6 +256,29 @@ bool add_gemm(Builder& bl, Model* m, const void* A, int lda, long long rows_cap,
     if (!make_tmap_c(&g.tmC, C, rows_cap, N, ldc, g.epi)) return false;
   }
   g.c_rows = (int)rows_cap;
+  m->ops.push_back(op);
+  return true;
+}
+
+// An encoder's MLP block as one fused op (see MlpGroup).  gemm.N / gemm.K carry the shapes for the step's
+// flop and byte accounting; gemm.stream == 4 routes the op to the fused kernel's launch.
+bool add_mlp(Builder& bl, Model* m, const void* X, long long rows_cap, const void* W1, const void* b1, const void* W2,
+             const void* b2, float* Z, int d, int F, int rows_per_req) {
+  Op op;
+  memset(&op, 0, sizeof(op));
+  op.kind = EPARA_K_GEMM;
+  op.rows_per_req = rows_per_req;
+  op.gemm.stream = 4; op.gemm.N = d; op.gemm.K = F; op.gemm.ksplit = 1; op.gemm.bn = d;
+  op.weight_bytes = 2.0 * 2.0 * d * F;
+  MlpGroup& g = op.mlp;
+  g.b1 = (const bf16*)b1; g.b2 = (const bf16*)b2; g.d = d; g.F = F; g.c_rows = (int)rows_cap;
+  if (bl.c) {
+    const int n2 = d > 256 ? d / 2 : d;
+    if (!make_tmap(&g.tmX, X, rows_cap, d, d, TC_BM)) return false;
+    if (!make_tmap(&g.tmW1, W1, F, d, d, 64)) return false;
+    if (!make_tmap(&g.tmW2, W2, d, F, F, n2 / 2)) return false;
+    if (!make_tmap_c(&g.tmC, Z, rows_cap, d, d, EPI_RESID_F32)) return false;
+  }
   m->ops.push_back(op);
   return true;
 }
@@ -377,7 +401,7 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
       at.kind = EPARA_K_ATTN_ENC; at.rows_per_req = T;
       at.aenc.qkv = qkv; at.aenc.out = a; at.aenc.T = T; at.aenc.H = d.n_heads; at.aenc.hd = d.head_dim;
       at.aenc.KP = round_up(T, 16);
-      at.aenc.tc = (d.head_dim == 64 && T <= ENC_TC_MAX_T && bl.gemm_impl == EPARA_GEMM_TCGEN05) ? 1 : 0;
+      at.aenc.tc = (d.head_dim == 64 && T <= ENC_TC_MAX_T && bl.gemm_impl != EPARA_GEMM_SIMT) ? 1 : 0;
       if (at.aenc.tc && bl.c) {
         if (!make_tmap(&at.aenc.tmQ, qkv, Mcap, 3 * dm, 3 * dm, 128)) return EPARA_E_CUDA;
         if (!make_tmap(&at.aenc.tmKV, qkv, Mcap, 3 * dm, 3 * dm, at.aenc.KP)) return EPARA_E_CUDA;
@@ -385,8 +409,12 @@ int build_model(Builder& bl, Model* m, const epara_config& cfg) {
       m->ops.push_back(at);
       if (!add_gemm(bl, m, a, dm, Mcap, w[4], dm, dm, z, dm, w[5], EPI_RESID_F32, T)) return EPARA_E_CUDA;
       add_norm(m, z, dm, h, w[6], w[7], dm, NORM_LN, 1e-6f, T);
-      if (!add_gemm(bl, m, h, dm, Mcap, w[8], d.ffn, dm, f, d.ffn, w[9], EPI_GELU, T)) return EPARA_E_CUDA;
-      if (!add_gemm(bl, m, f, d.ffn, Mcap, w[10], dm, d.ffn, z, dm, w[11], EPI_RESID_F32, T)) return EPARA_E_CUDA;
+      if (bl.gemm_impl == EPARA_GEMM_TCGEN05 && gemm_mlp_eligible(Mcap, dm, d.ffn)) {
+        if (!add_mlp(bl, m, h, Mcap, w[8], w[9], w[10], w[11], z, dm, d.ffn, T)) return EPARA_E_CUDA;
+      } else {
+        if (!add_gemm(bl, m, h, dm, Mcap, w[8], d.ffn, dm, f, d.ffn, w[9], EPI_GELU, T)) return EPARA_E_CUDA;
+        if (!add_gemm(bl, m, f, d.ffn, Mcap, w[10], dm, d.ffn, z, dm, w[11], EPI_RESID_F32, T)) return EPARA_E_CUDA;
+      }
     }
     const void* const* w = t + 4 + 12 * d.n_layers;
     add_norm(m, z, (long long)T * dm, cvec, w[0], w[1], dm, NORM_LN, 1e-6f, 1);
@@ -944,7 +972,8 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       // bf16-output groups (pass 2); encoder attention in two: the tcgen05 kernel (pass 0) and the
       // mma.sync kernel for shapes it does not take (pass 1)
       // (passes 3 to 6: the swapped-operand kernel with 1, 2, 4 and 8 k ranges per tile)
-      const int n_pass = kind == EPARA_K_GEMM ? 7 : (kind == EPARA_K_ATTN_ENC ? 2 : 1);
+      // (pass 7: encoder MLP blocks in the fused kernel)
+      const int n_pass = kind == EPARA_K_GEMM ? 8 : (kind == EPARA_K_ATTN_ENC ? 2 : 1);
       for (int pass = 0; pass < n_pass; ++pass) {
       Launch L;
       memset(&L, 0, sizeof(L));
@@ -1046,7 +1075,21 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
             GemmGroup g = op.gemm;
             int gpass = g.stream;
             if (g.stream == 3) gpass = 3 + (g.ksplit >= 8 ? 3 : g.ksplit >= 4 ? 2 : g.ksplit >= 2 ? 1 : 0);
+            if (g.stream == 4) gpass = 7;
             if (gpass != pass) break;                          // another pass takes it
+            if (g.stream == 4) {
+              MlpGroup mg = op.mlp;
+              mg.M = rows;
+              mg.tiles_m = (rows + 2 * TC_BM - 1) / (2 * TC_BM);
+              mg.tile_start = total;
+              total += mg.tiles_m;
+              ++n_put;
+              inf.gemm_groups++;
+              inf.gemm_flops += 2.0 * 2.0 * rows * mg.d * mg.F;
+              inf.weight_bytes += op.weight_bytes;
+              if (put(&mg, sizeof(mg), 64) == (size_t)-1) overflow = true;
+              break;
+            }
             g.M = rows;
             if (g.stream == 3) {
               g.tiles_m = 1; g.tiles_n = gemm_swap_tiles(g.N);
@@ -1153,7 +1196,8 @@ int epara_step(epara_ctx* c, void* cuda_stream, long long now_ns, epara_step_inf
       case EPARA_K_ASSEMBLE: launch_assemble((const AssembleGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_NORM: launch_norm((const NormGroup*)gp, L.n_groups, L.p1, st); break;
       case EPARA_K_GEMM:
-        if (L.p2 >= 3) err = launch_gemm_swap((const GemmGroup*)gp, L.n_groups, L.p0, 1 << (L.p2 - 3), dev_status, c->sm_count, st);
+        if (L.p2 == 7) err = launch_gemm_mlp_pair((const MlpGroup*)gp, L.n_groups, L.p0, dev_status, c->sm_count, st);
+        else if (L.p2 >= 3) err = launch_gemm_swap((const GemmGroup*)gp, L.n_groups, L.p0, 1 << (L.p2 - 3), dev_status, c->sm_count, st);
         else if (L.p2 == 1) err = launch_gemm_stream((const GemmGroup*)gp, L.n_groups, L.p0, L.p1, st);
         else if (L.p2 == 2) err = launch_gemm_tc_pair((const GemmGroup*)gp, L.n_groups, L.p0, dev_status, c->sm_count, st);
         else if (simt) launch_gemm_simt((const GemmGroup*)gp, L.n_groups, L.p0, st);

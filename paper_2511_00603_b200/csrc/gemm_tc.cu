@@ -785,6 +785,336 @@ gemm_tc_pair_kernel(const GemmGroup* __restrict__ groups, int n_groups, int tota
   }
 }
 
+// ---------------------------------------------------------------------------------- fused MLP block
+// z += GELU(h W1^T + b1) W2^T + b2 for encoder blocks with d <= 384: the 4d-wide hidden tensor never leaves
+// the SM.  A cluster of two CTAs works one 256-row tile (cta_group::2, as in the tile-pair kernel).  Per tile
+// the CTA's 128 rows of h stay in shared memory (d / 64 k-blocks of 16 KB); the hidden layer is taken in chunks
+// of 128 columns:
+//   S = h W1_c^T         (M 256, N 128, K d)  into tensor-memory columns 384..511,
+//   P = bf16(GELU(S + b1_c)) by the 16 epilogue warps, written to shared memory in the K-major 128-byte-swizzled
+//                        layout an A operand has (two blocks of 128 rows x 64 columns),
+//   O += P W2_c^T        (M 256, N d, K 128)  into columns 0..d-1 (two MMAs of N = d / 2 per k step when d > 256),
+// and after the last chunk O + b2 is added to z through the same TMA reduce-add epilogue as any fp32-residual
+// GEMM.  The rounding points are those of the unfused pair of GEMMs (the hidden tensor is rounded to bf16 once,
+// the k order of both contractions is ascending), so a request's bits do not change with the kernel.
+// The two contractions have an issuing thread each (warp 1 for S, the last warp for O): the chains only meet
+// through the epilogue warps (S -> P), so the tensor core works on the next chunk's S while this chunk's GELU is
+// computed and on this chunk's O while the next S is read out, and neither thread's issue time (some 80 cycles
+// per tcgen05.mma) delays the other chain.  Weights stream through two rings of two 24 KB slots (W1: three k-blocks
+// of a chunk half per slot; W2: one k-block of a chunk half per slot), each with its own producer thread.
+// P's 32 KB double as the staging area of the final epilogue (P is idle by then).
+constexpr int MLP_SLOT_BYTES = 24 * 1024;
+constexpr int MLP_SLOTS = 4;                                   // two for W1 (0, 1), two for W2 (2, 3)
+constexpr int MLP_O_WARP = PAIR_W_WARP + 1;                    // issues the second contraction
+constexpr int MLP_THREADS = PAIR_THREADS + 32;
+constexpr int MLP_X_BYTES = 6 * A_BYTES;                       // d <= 384: at most six k-blocks of 128 x 64
+constexpr int MLP_P_BYTES = 2 * A_BYTES;                       // 128 rows x 128 hidden columns, bf16
+constexpr int MLP_OFF_P = MLP_X_BYTES;
+constexpr int MLP_OFF_RING = MLP_OFF_P + MLP_P_BYTES;
+constexpr int MLP_OFF_BAR = MLP_OFF_RING + MLP_SLOTS * MLP_SLOT_BYTES;
+constexpr size_t MLP_SMEM_BYTES = 1024 + (size_t)MLP_OFF_BAR + 256;
+static_assert(MLP_SMEM_BYTES <= 227 * 1024, "shared memory of one SM");
+static_assert(STAGE_OUT_BYTES <= MLP_P_BYTES, "the final epilogue stages its boxes in P");
+constexpr int MLP_S_COL = 384;                                 // S behind the output accumulator
+constexpr int MLP_CHUNK = 128;
+enum { MB_W_FULL = 0, MB_W_EMPTY = MLP_SLOTS, MB_X_FULL = 2 * MLP_SLOTS, MB_X_EMPTY, MB_S_FULL, MB_S_EMPTY, MB_P_FULL,
+       MB_P_EMPTY, MB_O_FULL, MB_O_EMPTY, MB_STAGE_FREE, MB_COUNT };
+static_assert(8 * MB_COUNT + 16 <= 256, "barrier area");
+
+__device__ __forceinline__ int find_group_mlp(const MlpGroup* groups, int n, int item) {
+  int gi = 0;
+  for (int i = 1; i < n; ++i) if (groups[i].tile_start <= item) gi = i;
+  return gi;
+}
+// Geometry of a group in registers (the single-thread roles cannot hide descriptor loads).
+struct MlpGeo {
+  const MlpGroup* g;
+  int start, end, kb1, nc, n2, n2i, slots1;
+};
+__device__ __forceinline__ void mlp_geo(MlpGeo& c, const MlpGroup* groups, int n_groups, int item) {
+  if (c.g != nullptr && item >= c.start && item < c.end) return;
+  const MlpGroup* g = groups + find_group_mlp(groups, n_groups, item);
+  c.g = g;
+  c.start = g->tile_start;
+  c.end = c.start + g->tiles_m;
+  const int d = g->d;
+  c.kb1 = d >> 6;                       // k-blocks of the first contraction
+  c.nc = g->F / MLP_CHUNK;              // chunks of the hidden layer
+  c.n2i = d > 256 ? 2 : 1;              // MMAs per k step of the second contraction
+  c.n2 = d / c.n2i;                     // and their N
+  c.slots1 = (c.kb1 + 2) / 3;           // ring slots of one W1 chunk (three k-blocks of 64 rows each per slot)
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MLP_THREADS, 1)
+gemm_mlp_pair_kernel(const MlpGroup* __restrict__ groups, int n_groups, int total_items, int* __restrict__ status) {
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t bars = base + MLP_OFF_BAR;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + MLP_OFF_BAR + 8 * MB_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < MLP_SLOTS; ++s) { mbar_init(bar(MB_W_FULL + s), 1); mbar_init(bar(MB_W_EMPTY + s), 1); }
+    mbar_init(bar(MB_X_FULL), 1); mbar_init(bar(MB_X_EMPTY), 1);
+    mbar_init(bar(MB_S_FULL), 1); mbar_init(bar(MB_S_EMPTY), 2 * EPI_WARPS);
+    mbar_init(bar(MB_P_FULL), 2 * EPI_WARPS); mbar_init(bar(MB_P_EMPTY), 1);
+    mbar_init(bar(MB_O_FULL), 1); mbar_init(bar(MB_O_EMPTY), 2 * EPI_WARPS);
+    mbar_init(bar(MB_STAGE_FREE), EPI_WARPS);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                        // the peer's barriers exist before anything is reported to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer of h and W1 (one per CTA)
+    // Per tile: the CTA's rows of h (once the tile before has been used by its last S), then W1 chunk by chunk.
+    if (lane == 0) {
+      bool ok = true;
+      bool waited = false;
+      const MlpGroup* g_prev = nullptr;
+      MlpGeo gc;
+      gc.g = nullptr;
+      int slot = 0;
+      uint32_t phase = 0, t = 0;
+      for (int item = pair; item < total_items && ok; item += n_pairs, ++t) {
+        mlp_geo(gc, groups, n_groups, item);
+        const MlpGroup* g = gc.g;
+        if (g != g_prev) { tensormap_acquire(&g->tmX); tensormap_acquire(&g->tmW1); g_prev = g; }
+        const int m0 = (item - gc.start) * (2 * TC_BM) + rank * TC_BM;
+        if (!mbar_wait(bar(MB_X_EMPTY), (t & 1u) ^ 1u, abort_flag)) { ok = false; atomicExch(status, 41); break; }
+        if (!waited) { pdl_wait(); waited = true; }   // h is written by the kernel before this one
+        if (rank == 0) mbar_expect_tx(bar(MB_X_FULL), 2u * (uint32_t)gc.kb1 * A_BYTES);
+        for (int kb = 0; kb < gc.kb1; ++kb)
+          tma_load_2d_pair(base + kb * A_BYTES, &g->tmX, kb * TC_BK, m0, mapa_shared(bar(MB_X_FULL), 0));
+        for (int c = 0; c < gc.nc && ok; ++c) {
+          for (int s1 = 0; s1 < gc.slots1; ++s1) {
+            if (!mbar_wait(bar(MB_W_EMPTY + slot), phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 42); break; }
+            const int kb_lo = s1 * 3, kb_hi = min(gc.kb1, kb_lo + 3);
+            if (rank == 0) mbar_expect_tx(bar(MB_W_FULL + slot), 2u * (uint32_t)(kb_hi - kb_lo) * (64 * 128));
+            for (int kb = kb_lo; kb < kb_hi; ++kb)
+              tma_load_2d_pair(base + MLP_OFF_RING + slot * MLP_SLOT_BYTES + (kb - kb_lo) * (64 * 128), &g->tmW1, kb * TC_BK,
+                               c * MLP_CHUNK + rank * 64, mapa_shared(bar(MB_W_FULL + slot), 0));
+            if (++slot == 2) { slot = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) { *abort_flag = 1; drain_sleep(PAIR_DRAIN_NS); }
+    }
+  } else if (warp == PAIR_W_WARP) {
+    // ------------------------------------------------------------ TMA producer of W2 (one per CTA)
+    // (Weights are never written by a kernel: no wait for earlier kernels.)
+    if (lane == 0) {
+      int slot = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const MlpGroup* g_prev = nullptr;
+      MlpGeo gc;
+      gc.g = nullptr;
+      for (int item = pair; item < total_items && ok; item += n_pairs) {
+        mlp_geo(gc, groups, n_groups, item);
+        const MlpGroup* g = gc.g;
+        if (g != g_prev) { tensormap_acquire(&g->tmW2); g_prev = g; }
+        const int half = gc.n2 >> 1;                         // rows of one MMA's B operand held by this CTA
+        for (int c = 0; c < gc.nc && ok; ++c) {
+          for (int j = 0; j < 2; ++j) {                      // the chunk's two k-blocks
+            if (!mbar_wait(bar(MB_W_EMPTY + 2 + slot), phase ^ 1u, abort_flag)) { ok = false; atomicExch(status, 43); break; }
+            if (rank == 0) mbar_expect_tx(bar(MB_W_FULL + 2 + slot), 2u * (uint32_t)gc.n2i * (uint32_t)half * 128u);
+            for (int i = 0; i < gc.n2i; ++i)
+              tma_load_2d_pair(base + MLP_OFF_RING + (2 + slot) * MLP_SLOT_BYTES + i * half * 128, &g->tmW2, (2 * c + j) * TC_BK,
+                               i * gc.n2 + rank * half, mapa_shared(bar(MB_W_FULL + 2 + slot), 0));
+            if (++slot == 2) { slot = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) { *abort_flag = 1; drain_sleep(PAIR_DRAIN_NS); }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer of S = h W1_c^T (rank 0 only)
+    if (lane == 0 && rank == 0) {
+      int slot = 0;
+      uint32_t phase = 0;
+      uint32_t n_s = 0, t = 0;                // chunks issued, tiles started
+      bool ok = true;
+      MlpGeo gc;
+      gc.g = nullptr;
+      const uint32_t idesc_s = make_idesc_pair(MLP_CHUNK);
+      for (int item = pair; item < total_items && ok; item += n_pairs, ++t) {
+        mlp_geo(gc, groups, n_groups, item);
+        if (!mbar_wait(bar(MB_X_FULL), t & 1u, abort_flag)) { ok = false; atomicExch(status, 49); break; }
+        for (int c = 0; c < gc.nc && ok; ++c, ++n_s) {
+          // S is free once the epilogue warps have read the chunk before out of it
+          if (n_s > 0 && !mbar_wait(bar(MB_S_EMPTY), (n_s - 1) & 1u, abort_flag)) { ok = false; atomicExch(status, 44); break; }
+          tc_fence_after();
+          for (int s1 = 0; s1 < gc.slots1; ++s1) {
+            if (!mbar_wait(bar(MB_W_FULL + slot), phase, abort_flag)) { ok = false; atomicExch(status, 45); break; }
+            tc_fence_after();
+            const int kb_lo = s1 * 3, kb_hi = min(gc.kb1, kb_lo + 3);
+            for (int kb = kb_lo; kb < kb_hi; ++kb) {
+              const uint64_t da = make_smem_desc(base + kb * A_BYTES);
+              const uint64_t db = make_smem_desc(base + MLP_OFF_RING + slot * MLP_SLOT_BYTES + (kb - kb_lo) * (64 * 128));
+#pragma unroll
+              for (int k = 0; k < TC_BK / 16; ++k)
+                mma_f16_pair(tmem_base + MLP_S_COL, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc_s, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            mma_commit_pair(bar(MB_W_EMPTY + slot));
+            if (++slot == 2) { slot = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          mma_commit_pair(bar(MB_S_FULL));
+          if (c == gc.nc - 1) mma_commit_pair(bar(MB_X_EMPTY));     // the tile's rows of h are no longer needed
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp == MLP_O_WARP) {
+    // ------------------------------------------------------------ MMA issuer of O += P W2_c^T (rank 0 only)
+    if (lane == 0 && rank == 0) {
+      int slot = 0;
+      uint32_t phase = 0;
+      uint32_t n_o = 0, t = 0;
+      bool ok = true;
+      MlpGeo gc;
+      gc.g = nullptr;
+      for (int item = pair; item < total_items && ok; item += n_pairs, ++t) {
+        mlp_geo(gc, groups, n_groups, item);
+        const uint32_t idesc_o = make_idesc_pair(gc.n2);
+        const int half = gc.n2 >> 1;
+        for (int c = 0; c < gc.nc && ok; ++c, ++n_o) {
+          if (!mbar_wait(bar(MB_P_FULL), n_o & 1u, abort_flag)) { ok = false; atomicExch(status, 46); break; }
+          // the first chunk overwrites O: the tile before must have been read out of it
+          if (c == 0 && t > 0 && !mbar_wait(bar(MB_O_EMPTY), (t - 1) & 1u, abort_flag)) { ok = false; atomicExch(status, 47); break; }
+          tc_fence_after();
+          for (int j = 0; j < 2; ++j) {
+            if (!mbar_wait(bar(MB_W_FULL + 2 + slot), phase, abort_flag)) { ok = false; atomicExch(status, 48); break; }
+            tc_fence_after();
+            const uint64_t da = make_smem_desc(base + MLP_OFF_P + j * A_BYTES);
+#pragma unroll
+            for (int k = 0; k < TC_BK / 16; ++k)
+              for (int i = 0; i < gc.n2i; ++i) {
+                const uint64_t db = make_smem_desc(base + MLP_OFF_RING + (2 + slot) * MLP_SLOT_BYTES + i * half * 128);
+                mma_f16_pair(tmem_base + (uint32_t)(i * gc.n2), da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc_o,
+                             (c > 0 || j > 0 || k > 0) ? 1u : 0u);
+              }
+            mma_commit_pair(bar(MB_W_EMPTY + 2 + slot));
+            if (++slot == 2) { slot = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          mma_commit_pair(bar(MB_P_EMPTY));
+          if (c == gc.nc - 1) mma_commit_pair(bar(MB_O_FULL));
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps (2..17 of both CTAs)
+    pdl_wait();
+    const int ew = warp - 2;
+    const int quarter = warp & 3;
+    const int part = ew >> 2;
+    const int row = quarter * 32 + lane;
+    bool ok = true;
+    uint32_t n_c = 0, t = 0;                  // chunks and tiles done by this warp
+    const MlpGroup* g = nullptr;
+    int g_start = 0, g_end = -1, nc = 0, d = 0, c_rows = 0;
+    const bf16 *b1 = nullptr, *b2 = nullptr;
+    const uint32_t s_taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(MLP_S_COL + part * 32);
+    unsigned char* prow = base_ptr + MLP_OFF_P + (part >> 1) * A_BYTES + row * 128;
+    const int piece0 = (part & 1) * 4, sw = row & 7;
+    const uint32_t s_empty_r = mapa_shared(bar(MB_S_EMPTY), 0), p_full_r = mapa_shared(bar(MB_P_FULL), 0);
+    const uint32_t o_empty_r = mapa_shared(bar(MB_O_EMPTY), 0);
+    for (int item = pair; item < total_items && ok; item += n_pairs, ++t) {
+      if (item >= g_end || item < g_start) {
+        g = groups + find_group_mlp(groups, n_groups, item);
+        g_start = g->tile_start; g_end = g_start + g->tiles_m;
+        nc = g->F / MLP_CHUNK; d = g->d; c_rows = g->c_rows; b1 = g->b1; b2 = g->b2;
+        if (lane == 0) tensormap_acquire(&g->tmC);
+      }
+      for (int c = 0; c < nc && ok; ++c, ++n_c) {
+        // this warp's 32 hidden columns of the chunk: bias values four per lane in lanes 0..7
+        uint2 bias_reg = make_uint2(0u, 0u);
+        if (b1 != nullptr && lane < 8) bias_reg = __ldg(reinterpret_cast<const uint2*>(b1 + c * MLP_CHUNK + part * 32 + lane * 4));
+        if (!mbar_wait(bar(MB_S_FULL), n_c & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 50); break; }
+        tc_fence_after();
+        float v[32];
+        {
+          uint32_t r[32];
+          tmem_ld32(s_taddr, r);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(s_empty_r);       // the next chunk's S may be issued
+        if (b1 != nullptr) {
+#pragma unroll
+          for (int jj = 0; jj < 16; ++jj) {
+            const uint32_t w = __shfl_sync(0xffffffffu, (jj & 1) ? bias_reg.y : bias_reg.x, jj >> 1);
+            v[2 * jj] += __uint_as_float(w << 16);
+            v[2 * jj + 1] += __uint_as_float(w & 0xffff0000u);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+        // P still feeds the second contraction of the chunk before; at a tile's first chunk it also was the
+        // staging area of the final epilogue of the tile before, which every warp of this CTA must have left
+        if (n_c > 0 && !mbar_wait(bar(MB_P_EMPTY), (n_c - 1) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 51); break; }
+        if (c == 0 && t > 0 && !mbar_wait(bar(MB_STAGE_FREE), (t - 1) & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 52); break; }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          uint4 o;
+          o.x = pack2(v[8 * k], v[8 * k + 1]); o.y = pack2(v[8 * k + 2], v[8 * k + 3]);
+          o.z = pack2(v[8 * k + 4], v[8 * k + 5]); o.w = pack2(v[8 * k + 6], v[8 * k + 7]);
+          *reinterpret_cast<uint4*>(prow + (((piece0 + k) ^ sw) << 4)) = o;
+        }
+        fence_async_smem();                     // P must be visible to the tensor core's reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(p_full_r);
+      }
+      if (!ok) break;
+      // ---- the tile's output: O + b2 added to z (TMA reduce-add), staged in P
+      GView gv;
+      gv.bias = b2; gv.C = nullptr; gv.partial = nullptr; gv.counters = nullptr; gv.tmC = &g->tmC;
+      gv.M = g->M; gv.N = d; gv.K = g->F; gv.ldc = d; gv.epi = EPI_RESID_F32 | (b2 != nullptr ? EPI_BIAS : 0);
+      gv.tile_start = g_start; gv.tiles_m = g_end - g_start; gv.tiles_n = 1; gv.bn = d; gv.ksplit = 1; gv.c_rows = c_rows;
+      Item it;
+      it.split = 0; it.tile = item - g_start; it.m0 = it.tile * (2 * TC_BM) + rank * TC_BM; it.n0 = 0; it.kb0 = 0; it.kb1 = 0;
+      uint2 bias_reg = make_uint2(0u, 0u);
+      if (b2 != nullptr) {
+        const int nb = part * (d >> 2) + lane * 4;
+        if (lane * 4 < (d >> 2)) bias_reg = __ldg(reinterpret_cast<const uint2*>(b2 + nb));
+      }
+      if (!mbar_wait(bar(MB_O_FULL), t & 1u, abort_flag)) { ok = false; if (lane == 0) atomicExch(status, 53); break; }
+      tc_fence_after();
+      const uint32_t o_taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      epi_direct<2, true>(gv, it, o_taddr, base_ptr + MLP_OFF_P + ew * 2048, quarter, part, lane, bias_reg, o_empty_r);
+      if (lane == 0) { bulk_wait_read0(); mbar_arrive(bar(MB_STAGE_FREE)); }   // this warp's boxes have left P
+    }
+    if (lane == 0) bulk_wait_done0();
+    if (!ok) *abort_flag = 1;
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                        // neither CTA leaves while the other may still read its operands or signal it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+  }
+}
+
 }  // namespace
 
 // Tile width and k-split of a GEMM whose row capacity is rows_cap (fixed when the model is placed,
@@ -847,6 +1177,21 @@ cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total
   if (e != cudaSuccess) return e;
   const int pairs = total_items < sm_count / 2 ? total_items : sm_count / 2;
   return launch_pdl(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(PAIR_THREADS), SMEM_BYTES, st, groups, n_groups, total_items, status);
+}
+
+// The fused MLP kernel takes an encoder block when its accumulators fit the tensor memory (d <= 384 beside one
+// 128-column chunk of S), the shapes tile evenly, and the model has more than one 128-row tile at capacity.
+bool gemm_mlp_eligible(long long rows_cap, int d, int F) {
+  return rows_cap > TC_BM && d >= 64 && d <= 384 && d % 64 == 0 && F >= 128 && F % 128 == 0;
+}
+
+cudaError_t launch_gemm_mlp_pair(const MlpGroup* groups, int n_groups, int total_items, int* status, int sm_count,
+                                 cudaStream_t st) {
+  if (n_groups == 0 || total_items == 0) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(gemm_mlp_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MLP_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int pairs = total_items < sm_count / 2 ? total_items : sm_count / 2;
+  return launch_pdl(gemm_mlp_pair_kernel, dim3(2 * pairs), dim3(MLP_THREADS), MLP_SMEM_BYTES, st, groups, n_groups, total_items, status);
 }
 
 }  // namespace epara

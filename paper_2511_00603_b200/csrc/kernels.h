@@ -25,6 +25,9 @@ constexpr int TC_BN_MAX = 256;
 constexpr int TC_BK = 64;
 void gemm_tc_config(long long rows_cap, int N, int K, int epi, int sm_count, int* bn, int* ksplit);
 bool gemm_tc_pair_eligible(long long rows_cap, int N, int K, int epi, int bn, int ksplit);
+bool gemm_mlp_eligible(long long rows_cap, int d, int F);
+cudaError_t launch_gemm_mlp_pair(const MlpGroup* groups, int n_groups, int total_items, int* status, int sm_count,
+                                 cudaStream_t st);
 cudaError_t launch_gemm_tc_pair(const GemmGroup* groups, int n_groups, int total_items, int* status, int sm_count,
                                 cudaStream_t st);
 cudaError_t launch_gemm_tc(const GemmGroup* groups, int n_groups, int total_items, int max_bn, int* status,

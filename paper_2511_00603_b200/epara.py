@@ -21,7 +21,7 @@ OK, PENDING = 0, 1
 E_INVALID, E_UNSUPPORTED, E_TIMEOUT, E_RESOURCE, E_DEVICE, E_CUDA = -1, -2, -3, -4, -5, -6
 CAT_LS, CAT_FS, CAT_LS_GT1, CAT_FS_GT1 = 0, 1, 2, 3
 MODEL_MLP, MODEL_VIT, MODEL_DECODER = 0, 1, 2
-GEMM_TCGEN05, GEMM_SIMT = 0, 1
+GEMM_TCGEN05, GEMM_SIMT, GEMM_TCGEN05_UNFUSED = 0, 1, 2
 EPI_BIAS, EPI_GELU, EPI_SWIGLU, EPI_RESID_F32 = 1, 2, 4, 8
 K_NAMES = ["gather", "norm", "gemm", "rope", "attn_dec", "attn_combine", "attn_enc", "assemble", "output", "gemm_stream", "trace", "attn_prefill"]
 ERR_PAGE_APPEND, ERR_PAGE_ATTEND, ERR_SELFTEST_WAIT = 101, 102, 90

@@ -418,3 +418,39 @@ def test_workspace_too_small_is_resource_insufficiency(mods):
         srv.add_model(p, max_batch=64)
     assert ei.value.status == E.E_RESOURCE
     srv.close()
+
+
+@pytest.mark.parametrize("shape", [(384, 6, 1536, 2, 3, 224), (128, 2, 256, 2, 5, 96), (256, 4, 512, 1, 4, 128),
+                                   (320, 5, 1280, 1, 2, 224)])
+def test_fused_encoder_mlp_block_equals_the_unfused_kernels_and_the_oracle(mods, shape):
+    """The fused FC1 -> GELU -> FC2 -> residual kernel (default placement of encoder blocks with d <= 384 and more than
+    128 rows) against the same model placed with every GEMM as its own launch: same rounding points, same
+    reduction order, so the logits must be bit-identical; and against the oracle for the first and last image.
+    Shapes: ViT-S (two MMAs of N = 192 per k step), d 128 and 256 (one MMA), d 320 (two of 160; five k-blocks: a
+    partly filled second ring slot), with row counts that leave a ragged last pair."""
+    E, server = mods
+    d, heads, mlp, layers, B, img = shape
+    p = synth.make_vit(d=d, n_layers=layers, n_heads=heads, mlp=mlp, n_cls=100, seed=5, device=DEV, img=img, std=0.05,
+                       perturb=0.2)
+    imgs = synth.make_images(B, seed=6, device=DEV, img=img)
+
+    def run(impl):
+        srv = server.Server(workspace_bytes=1 << 30, gemm_impl=impl)
+        m = srv.add_model(p, max_batch=B)
+        ts = [srv.submit(m, E.CAT_FS, x=imgs[i]) for i in range(B)]
+        info = srv.step()
+        res = _finish(srv, E, ts)
+        srv.close()
+        return info, res
+
+    fused_info, fused = run(E.GEMM_TCGEN05)
+    plain_info, plain = run(E.GEMM_TCGEN05_UNFUSED)
+    assert plain_info.launches - fused_info.launches == layers          # one launch less per block
+    assert fused_info.gemm_flops == plain_info.gemm_flops
+    for i in range(B):
+        assert torch.equal(fused[i][0], plain[i][0]) and fused[i][1] == plain[i][1]
+    v = synth.bits_view(p)
+    for i in (0, B - 1):
+        ref, _, _ = O.vit_forward(synth.to_bits(imgs[i]), v)
+        assert_close(fused[i][0], ref, what=f"fused MLP block, d={d}, image {i}")
+        check_argmax(fused[i][1], fused[i][0], ref)
