@@ -24,10 +24,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # DRAM bytes (read + write) per tensor-core GEMM launch of the mixed step, from one ncu pass over the GEMM
-# launches of a step (65 tile-pair launches: 15.92 GB read + 8.54 GB written; the 65 weight-streaming
-# launches moved 2.08 GB).  Not measured by this run: the profile it comes from is named beside it in the
-# JSON line.  Set to None when the GEMM kernels change.
-GEMM_TC_TRAFFIC_PER_LAUNCH_MIXED = (15922343680 + 8536922368) / 65
+# launches of a step (65 tile-pair launches: 7.72 GB read + 3.69 GB written; 12 fused MLP-block launches:
+# 2.90 GB read + 1.18 GB written; the 65 weight-streaming launches moved 2.08 GB).  Not measured by this run:
+# the profile it comes from is named beside it in the JSON line.  Set to None when the GEMM kernels change.
+GEMM_TC_TRAFFIC_PER_LAUNCH_MIXED = 15488294144 / 77
 GEMM_TRAFFIC_SOURCE = "profiles/gemm_kernels_mixed_step_dram_traffic.md (one ncu pass, dram__bytes_read.sum + dram__bytes_write.sum)"
 
 E2E_BUFS = 4          # device input buffers per instance in the end-to-end loop
@@ -569,7 +569,7 @@ def run_gpu(args):
     if dom == "gemm":
         ach = per_step(flops - sflops) / (tc_ms / 1e3) / 1e12
         peak = peaks["bf16_tflops"] if near_max else peaks["bf16_tflops_sustained"]
-        roof = {"kernel": "gemm_tc_pair_kernel + gemm_tc_kernel (the tensor-core GEMM launches of a step)", "bound": "tensor",
+        roof = {"kernel": "gemm_tc_pair_kernel + gemm_mlp_pair_kernel (the tensor-core GEMM launches of a step)", "bound": "tensor",
                 "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
                 "frac_of_burst_peak": ach / peaks["bf16_tflops"], "frac_of_sustained_peak": ach / peaks["bf16_tflops_sustained"],
                 "sm_mhz_median": clocks.get("sm_mhz"), "launches_per_step": prof["gemm"][1], "ms_per_step": tc_ms,
